@@ -1,0 +1,62 @@
+"""Pins for the oracle's staging model (D6): the sink is the concatenation, chunk count and sizes,
+stage-in inverts stage-out, resume, budget rule, completion order."""
+import numpy as np
+import pytest
+
+import oracle
+
+
+def _bufs(sizes, seed=0):
+    rng = np.random.default_rng(seed)
+    return [rng.integers(0, 256, size=n, dtype=np.uint64).astype(np.uint8) for n in sizes]
+
+
+@pytest.mark.parametrize("sizes,budget,chunk", [
+    ((10000, 10000), 8192, 0),          # default chunk = budget/2; a chunk straddles the boundary
+    ((12345, 1, 777), 3000, 1000),      # three slots, ragged tail
+    ((4096,), 8192, 4096),              # exactly one chunk
+    ((5000, 0, 5000), 8192, 4096),      # an empty buffer in the middle
+])
+def test_stage_out_is_concatenation_and_stage_in_inverts_it(sizes, budget, chunk):
+    bufs = _bufs(sizes)
+    sink, csz = oracle.stage_out(bufs, budget, chunk)
+    cat = np.concatenate(bufs)
+    assert np.array_equal(sink, cat)
+    c = chunk or budget // 2 // 4096 * 4096
+    assert len(csz) == -(-cat.size // c)
+    assert (csz[:-1] == c).all() and csz[-1] == cat.size - c * (len(csz) - 1)
+    back = [np.zeros_like(b) for b in bufs]
+    order = list(range(len(bufs)))[::-1]
+    pieces, done = oracle.stage_in(back, sink, budget, chunk, order)
+    assert all(np.array_equal(a, b) for a, b in zip(back, bufs))
+    assert done == order
+    assert pieces == sum(-(-n // c) for n in sizes)
+
+
+def test_tiny_workload_chunking_matches_the_quoted_figures():
+    # Adam m and v of rank 0's shard of the tiny model, 1 MiB budget: 16 chunks, last of 38 912 bytes,
+    # chunk 7 straddles the m | v boundary.
+    shard_bytes = 987_904 * 4
+    bufs = _bufs((shard_bytes, shard_bytes), 1)
+    sink, csz = oracle.stage_out(bufs, 1 << 20)
+    assert len(csz) == 16 and csz[-1] == 38_912 and (csz[:-1] == 512 * 1024).all()
+    assert 7 * 512 * 1024 < shard_bytes < 8 * 512 * 1024
+    assert np.array_equal(sink, np.concatenate(bufs))
+
+
+def test_resume_from_a_failed_chunk_gives_the_same_bytes():
+    bufs = _bufs((9000, 7000), 3)
+    full, csz = oracle.stage_out(bufs, 4096, 1024)
+    k = 5
+    partial = np.zeros_like(full)
+    partial[:k * 1024] = full[:k * 1024]          # chunks < k were delivered before the failure
+    sink, _ = oracle.stage_out(bufs, 4096, 1024, first_chunk=k, sink=partial)
+    assert np.array_equal(sink, full)
+
+
+def test_budget_must_hold_two_slots():
+    bufs = _bufs((100,))
+    with pytest.raises(ValueError):
+        oracle.stage_out(bufs, 1000, 600)
+    with pytest.raises(ValueError):
+        oracle.stage_out(bufs, 4096)  # default chunk rounds down to 0
