@@ -1,0 +1,247 @@
+/*
+ * dynaresize.h -- C ABI of the per-GPU role-switch state transform for sm_100a (B200).
+ *
+ * When runtime GPU reallocation turns a Training GPU into a Rollout GPU (or back), the GPU must
+ * "flush old parameters and ingest new weights and optimizer states" (paper Sec. 1, challenge 2) and
+ * "reload the states required by the new topology" (Sec. 3.3).  This library is that per-GPU step:
+ *
+ *   Training -> Rollout : read the FSDP-style flat fp32 master buffer, un-flatten it, fuse Q/K/V and
+ *                         gate/up, slice for a tensor-parallel degree and rank, cast to bf16
+ *                         (round to nearest, ties to even) into a contiguous rollout arena;
+ *   Rollout -> Training : the inverse layout map (bf16 widened exactly to fp32);
+ *   both directions     : stream optimizer state (fp32 master, Adam m, Adam v) to and from host
+ *                         memory in fixed chunks through a bounded pinned ring (the "chunked
+ *                         streaming ... through host-memory buffers" of Sec. 3.3), weights first
+ *                         on the way back (the deferred optimizer reload of Sec. 3.3).
+ *
+ * Conventions
+ *   - Every function returns an int status: DR_OK (0) or a negative dr_status.  Nothing throws,
+ *     aborts or exits.  dr_last_error() gives a thread-local detail string for the last failure.
+ *   - "dev" pointers are CUDA device pointers of the current device; "host" pointers are ordinary
+ *     host pointers.  The caller owns every buffer it passes.  A plan owns only its device segment
+ *     table, its pinned staging ring and two internal streams.
+ *   - Streams and events are passed as void* holding a cudaStream_t / cudaEvent_t (NULL stream =
+ *     the legacy default stream).
+ *   - There is no CPU fallback: without a CUDA device every compute call fails with DR_ERR_CUDA.
+ *   - Matrices are [out_features, in_features], row-major.
+ */
+#ifndef DYNARESIZE_H
+#define DYNARESIZE_H
+
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+#define DR_VERSION 1u
+#define DR_MAX_STAGE_BUFS 8u
+
+typedef enum dr_status {
+    DR_OK = 0,
+    DR_ERR_INVALID = -1,     /* NULL pointer, bad struct_size/version, value out of range          */
+    DR_ERR_UNSUPPORTED = -2, /* shapes not divisible by tp, moe_tp != 1, unknown kind/dtype         */
+    DR_ERR_SIZE = -3,        /* a buffer is smaller than the plan needs                             */
+    DR_ERR_ALIGN = -4,       /* a base pointer is not 16-byte aligned                               */
+    DR_ERR_NOMEM = -5,       /* host, pinned or device allocation failed                            */
+    DR_ERR_CUDA = -6,        /* a CUDA runtime call failed (detail in dr_last_error)                */
+    DR_ERR_BUDGET = -7,      /* staging budget cannot hold two chunk slots                          */
+    DR_ERR_SINK = -8,        /* the chunk callback returned non-zero                                */
+    DR_ERR_TIMEOUT = -9,     /* a bounded host-side wait ran out                                    */
+    DR_ERR_STATE = -10       /* call not valid for this plan (e.g. reshard on a host-only plan)     */
+} dr_status;
+
+enum { DR_SRC_FSDP_FLAT = 1 };
+enum { DR_DST_ROLLOUT_FUSED = 1 };
+enum { DR_F32 = 1, DR_BF16 = 2 };
+
+/* Decoder shape.  Dense when n_experts == 0 (SwiGLU of width ffn), else every layer holds a router
+ * [n_experts, hidden] and n_experts SwiGLU experts of width moe_ffn (ffn is ignored). */
+typedef struct dr_model_spec {
+    uint32_t struct_size, version; /* sizeof(dr_model_spec), DR_VERSION */
+    uint32_t n_layers, hidden, n_q_heads, n_kv_heads, head_dim, ffn, vocab;
+    uint32_t n_experts, moe_ffn;
+    uint8_t tied_embeddings; /* 1: no separate lm_head; the rollout lm_head aliases embed            */
+    uint8_t qk_norm;         /* 1: per-layer q_norm[head_dim], k_norm[head_dim] vectors exist        */
+    uint8_t pad[2];
+} dr_model_spec;
+
+/* Training-side layout: all parameters flattened in canonical order
+ *   embed; per layer: in_norm, q, k, v, (q_norm, k_norm), o, post_norm,
+ *   dense: gate, up, down | MoE: router, then per expert gate_e, up_e, down_e;
+ *   final_norm; lm_head unless tied
+ * each starting at a multiple of align_elems; N elements in all, S = ceil(N / world) per rank.
+ * gathered = 1: the source buffer holds world * S elements (the whole flat buffer);
+ * gathered = 0: it holds rank `rank`'s S elements only, and only elements inside that shard move. */
+typedef struct dr_src_layout {
+    uint32_t struct_size, kind /* DR_SRC_FSDP_FLAT */, dtype /* DR_F32 */;
+    uint32_t world, rank, gathered, align_elems /* >= 1 */;
+} dr_src_layout;
+
+/* Rollout-side layout at (tp, rank): tensors in arena order, each start aligned to arena_align_bytes:
+ *   embed rows of this rank; per layer: in_norm, qkv = [q_t; k_t; v_t], (q_norm, k_norm),
+ *   o columns of this rank, post_norm, dense: gate_up = [gate_t; up_t], down columns of this rank |
+ *   MoE: router, w13[e] = [gate_e; up_e] for every expert, w2[e] = down_e;
+ *   final_norm; lm_head rows of this rank (an alias of embed when tied).
+ * Norms and the router are replicated on every rank; experts are not sliced (moe_tp must be 1). */
+typedef struct dr_dst_layout {
+    uint32_t struct_size, kind /* DR_DST_ROLLOUT_FUSED */, dtype /* DR_BF16 or DR_F32 */;
+    uint32_t moe_tp /* 1 */, arena_align_bytes /* power of two >= 16, e.g. 256 */;
+} dr_dst_layout;
+
+typedef struct dr_plan dr_plan;
+
+typedef struct dr_plan_info {
+    uint64_t flat_elems;      /* N                                                                   */
+    uint64_t shard_elems;     /* S                                                                   */
+    uint64_t src_bytes;       /* bytes the source (flat) buffer must hold: 4*W*S or 4*S              */
+    uint64_t dst_bytes;       /* bytes the rollout arena must hold                                   */
+    uint64_t n_tensors;       /* rollout tensors (aliases included)                                  */
+    uint64_t n_segments;      /* entries of the device segment table                                 */
+    uint64_t n_tiles;         /* work tiles one launch processes                                     */
+    uint64_t elems_moved;     /* elements one dr_reshard / dr_reshard_inverse moves                  */
+    uint64_t bytes_moved_fwd; /* algorithmic bytes of dr_reshard: (4 + dst element size) * elems     */
+    uint64_t bytes_moved_inv; /* the same for dr_reshard_inverse                                     */
+} dr_plan_info;
+
+typedef struct dr_tensor_desc {
+    char name[64];
+    uint64_t arena_off; /* byte offset of the tensor inside the rollout arena                       */
+    uint64_t rows, cols;
+    int64_t alias_of;   /* >= 0: index of the rollout tensor whose storage this one shares           */
+} dr_tensor_desc;
+
+/* One entry of the compiled map: rows x row_len elements, row i read from source element
+ * src_off + i * src_row_stride and written at arena byte dst_off + i * dst_row_stride * elem size.
+ * Exposed so that the planner can be checked without a GPU. */
+typedef struct dr_segment_desc {
+    uint64_t dst_off;  /* bytes, relative to the arena base                                         */
+    uint64_t src_off;  /* elements, relative to the source buffer the call receives                 */
+    uint64_t rows, row_len, src_row_stride, dst_row_stride; /* elements                              */
+    uint32_t vector_bytes; /* 32 / 16: source access width the kernel may use; 0: scalar path        */
+    uint32_t tensor;       /* rollout tensor it belongs to                                           */
+} dr_segment_desc;
+
+/*
+ * dr_plan_create -- compile the un-flatten / fuse / slice map for (spec, src, dst, tp, rank) into a
+ * segment table and upload it to the current device (one small H2D copy; synchronous).  This is the
+ * metadata a resize prepares ahead of the switch (Sec. 3.2 applies the same idea to communicators).
+ * Errors: DR_ERR_INVALID, DR_ERR_UNSUPPORTED (n_q_heads, n_kv_heads, ffn or vocab not divisible by
+ * tp; moe_tp != 1), DR_ERR_NOMEM, DR_ERR_CUDA.  *out is NULL on failure.
+ */
+int dr_plan_create(const dr_model_spec* spec, const dr_src_layout* src, const dr_dst_layout* dst, uint32_t tp,
+                   uint32_t rank, dr_plan** out);
+
+/* Same planner, no device work: the plan answers queries only; reshard and staging calls on it
+ * return DR_ERR_STATE.  For checking the planner where no GPU exists. */
+int dr_plan_create_host(const dr_model_spec* spec, const dr_src_layout* src, const dr_dst_layout* dst, uint32_t tp,
+                        uint32_t rank, dr_plan** out);
+
+int dr_plan_query(const dr_plan* plan, dr_plan_info* out);
+int dr_plan_tensor(const dr_plan* plan, uint32_t i, dr_tensor_desc* out);   /* DR_ERR_INVALID if i >= n_tensors  */
+int dr_plan_segment(const dr_plan* plan, uint64_t i, dr_segment_desc* out); /* DR_ERR_INVALID if i >= n_segments */
+
+/*
+ * dr_reshard -- Training -> Rollout (Sec. 1 challenge 2: "ingest new weights").  Enqueues the
+ * gather / cast kernel on cuda_stream and returns; nothing is synchronised.
+ *   src_dev : fp32 flat buffer (whole, or this rank's shard when gathered = 0), read only
+ *   dst_dev : rollout arena; only mapped elements are written, gaps and (for gathered = 0) elements
+ *             whose source lies in another shard keep their bytes
+ * Every rollout element is the bf16 round-to-nearest-even cast of its source element (NaN -> 0x7FFF;
+ * subnormals are rounded, not flushed), or a bit copy when the plan's dst dtype is DR_F32.
+ * Errors (all found before launch): DR_ERR_SIZE if src_bytes / dst_bytes are below the plan's
+ * requirement, DR_ERR_ALIGN if a base pointer is not 16-byte aligned, DR_ERR_STATE, DR_ERR_CUDA.
+ * The plan is not modified: concurrent calls on different streams are allowed.
+ */
+int dr_reshard(const dr_plan* plan, const void* src_dev, uint64_t src_bytes, void* dst_dev, uint64_t dst_bytes,
+               void* cuda_stream);
+
+/*
+ * dr_reshard_inverse -- Rollout -> Training (Sec. 3.3: "reload the states required by the new
+ * topology").  Scatters the rollout arena back to the flat positions it was taken from, widening
+ * bf16 to fp32 exactly (bits << 16).  Only positions covered by this TP rank (and, for gathered = 0,
+ * lying in this shard) are written; padding and everything else keep their bytes.  Asynchronous on
+ * cuda_stream; same errors as dr_reshard.
+ */
+int dr_reshard_inverse(const dr_plan* plan, const void* rollout_dev, uint64_t rollout_bytes, void* flat_dev,
+                       uint64_t flat_bytes, void* cuda_stream);
+
+/* Chunk callback: stage-out hands chunk `chunk_idx` (bytes [stream_off, stream_off + n) of the
+ * stream) in `pinned`; stage-in asks the callback to fill `pinned` with those bytes.  The pointer is
+ * valid only during the call.  A non-zero return stops the transfer with DR_ERR_SINK. */
+typedef int (*dr_chunk_fn)(void* user, uint64_t chunk_idx, uint64_t stream_off, void* pinned, uint64_t n);
+
+/*
+ * Staging descriptor.  The state buffers form one logical byte stream X = buf_0 | buf_1 | ... of B
+ * bytes.  Stage-out cuts X into chunks of chunk_bytes (chunk k = X[k C, min((k+1) C, B)); a chunk
+ * that straddles a buffer boundary is one chunk made of two copies) and delivers them in increasing
+ * k.  Stage-in restores the buffers in `order` (weights first); each buffer is cut into pieces of at
+ * most chunk_bytes, numbered consecutively in that order.
+ * At most budget_bytes of pinned ring memory are held: slots = floor(budget / chunk) >= 2.
+ * Where the bytes rest (exactly one of):
+ *   callback   != NULL : every chunk goes to / comes from the callback
+ *   relay_dev[0] != NULL (stage-out only): every chunk is copied straight on to relay_dev[i], the
+ *                        old-rank -> new-rank pipeline of Sec. 3.3, never resting on the host
+ *   host_arena != NULL : arena[0, B) is the stream image; a pinned arena is copied to directly
+ *                        (still chunk by chunk), a pageable one through the ring by worker threads
+ */
+typedef struct dr_stage_desc {
+    uint32_t struct_size, n_bufs;       /* sizeof(dr_stage_desc); 1..DR_MAX_STAGE_BUFS                */
+    void* dev_ptr[DR_MAX_STAGE_BUFS];   /* device buffers, in stream order                            */
+    uint64_t bytes[DR_MAX_STAGE_BUFS];
+    uint32_t order[DR_MAX_STAGE_BUFS];  /* stage-in priority, a permutation of 0..n_bufs-1            */
+    uint64_t budget_bytes;
+    uint64_t chunk_bytes;               /* 0: budget / 2 rounded down to a multiple of 4096           */
+    void* host_arena;
+    uint64_t host_arena_bytes;
+    dr_chunk_fn callback;
+    void* user;
+    void* relay_dev[DR_MAX_STAGE_BUFS];
+    uint64_t first_chunk;               /* resume: chunks / pieces below this index are skipped       */
+    void* wait_event;                   /* cudaEvent_t the first copy waits for (producer), or NULL   */
+    void* ready_events[DR_MAX_STAGE_BUFS]; /* stage-in: caller's cudaEvent_t recorded on the copy
+                                              stream right after buffer i's last copy; NULL = none   */
+    uint32_t timeout_ms;                /* bound on every internal wait; 0 = 60 000                   */
+    uint32_t flags;                     /* 0                                                          */
+} dr_stage_desc;
+
+typedef struct dr_stage_stats {
+    uint64_t bytes;                    /* bytes moved by this call                                    */
+    uint64_t chunks_done;              /* chunks (stage-out) / pieces (stage-in) complete, counted
+                                          from 0: on failure, resume with first_chunk = chunks_done  */
+    uint64_t n_chunks;                 /* total for the whole stream                                  */
+    double elapsed_ms;
+    double link_gbs;                   /* bytes / elapsed, 1e9 bytes per second                       */
+    uint64_t pinned_high_water_bytes;  /* pinned ring bytes held (0 when a pinned arena is used)      */
+    double ready_ms[DR_MAX_STAGE_BUFS];/* stage-in: time from call start until buffer i was resident  */
+} dr_stage_stats;
+
+/*
+ * dr_stage_out -- device -> host in bounded chunks (Sec. 3.3: the states are partitioned into
+ * chunks and streamed through host-memory buffers, store and reload pipelined chunk by chunk).
+ * Blocking pump on the calling thread; copies run on the plan's side stream so that a dr_reshard
+ * enqueued before it overlaps (both only read the master buffer).  On return every delivered chunk
+ * is complete and byte-exact.  Errors: DR_ERR_INVALID, DR_ERR_BUDGET, DR_ERR_SIZE (arena too small),
+ * DR_ERR_NOMEM (pinned ring), DR_ERR_SINK, DR_ERR_TIMEOUT, DR_ERR_CUDA, DR_ERR_STATE.
+ * Calls on one plan must not overlap in time (they share the ring).
+ */
+int dr_stage_out(dr_plan* plan, const dr_stage_desc* desc, dr_stage_stats* stats);
+
+/*
+ * dr_stage_in -- host -> device, buffers in desc->order so that the weights are resident first and
+ * the optimizer state follows (Sec. 3.3: only the weights are loaded during the transition, the
+ * optimizer states are deferred to the first step on the new topology).  stats->ready_ms[i] and
+ * ready_events[i] tell when buffer i became usable.  Same pump, errors and threading as above.
+ */
+int dr_stage_in(dr_plan* plan, const dr_stage_desc* desc, dr_stage_stats* stats);
+
+/* Synchronises the plan's own streams, frees its ring, table and streams.  NULL is accepted. */
+int dr_plan_destroy(dr_plan* plan);
+
+const char* dr_strerror(int status);
+const char* dr_last_error(void);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* DYNARESIZE_H */

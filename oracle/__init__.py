@@ -41,6 +41,8 @@ def _l():
         u64, i64, p = ctypes.c_uint64, ctypes.c_int64, ctypes.c_void_p
         lib.orc_cast_bf16.restype = ctypes.c_uint16
         lib.orc_cast_bf16.argtypes = [ctypes.c_uint32]
+        lib.orc_cast_bf16_many.restype = None
+        lib.orc_cast_bf16_many.argtypes = [p, p, u64]
         lib.orc_widen_bf16.restype = ctypes.c_uint32
         lib.orc_widen_bf16.argtypes = [ctypes.c_uint16]
         lib.orc_model_create.restype = p
@@ -82,8 +84,9 @@ def widen_bf16(b: int) -> int:
 def cast_bf16_array(u: np.ndarray) -> np.ndarray:
     """D5 element by element (the scalar C function called in a loop)."""
     u = np.ascontiguousarray(u, dtype=np.uint32)
-    f = _l().orc_cast_bf16
-    return np.fromiter((f(int(x)) for x in u.ravel()), dtype=np.uint16, count=u.size).reshape(u.shape)
+    out = np.empty(u.shape, dtype=np.uint16)
+    _l().orc_cast_bf16_many(u.ctypes.data, out.ctypes.data, u.size)
+    return out
 
 
 @dataclass(frozen=True)

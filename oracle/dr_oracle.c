@@ -86,6 +86,13 @@ uint16_t orc_cast_bf16(uint32_t u)
     return (uint16_t)((u + 0x7FFFu + ((u >> 16) & 1u)) >> 16);
 }
 
+/* The same cast over an array: the scalar function, one element at a time. */
+void orc_cast_bf16_many(const uint32_t *u, uint16_t *out, uint64_t n)
+{
+    uint64_t i;
+    for (i = 0; i < n; ++i) out[i] = orc_cast_bf16(u[i]);
+}
+
 /* bf16 -> fp32 is exact: the 16 bits become the high half. */
 uint32_t orc_widen_bf16(uint16_t b) { return (uint32_t)b << 16; }
 

@@ -1,0 +1,282 @@
+"""ctypes binding for ``libdynaresize.so``: structures and functions named as in ``dynaresize.h``."""
+from __future__ import annotations
+
+import ctypes as C
+import os
+
+_DIR = os.path.dirname(os.path.abspath(__file__))
+lib_path = os.path.join(_DIR, "libdynaresize.so")
+
+DR_OK = 0
+DR_ERR_INVALID, DR_ERR_UNSUPPORTED, DR_ERR_SIZE, DR_ERR_ALIGN, DR_ERR_NOMEM = -1, -2, -3, -4, -5
+DR_ERR_CUDA, DR_ERR_BUDGET, DR_ERR_SINK, DR_ERR_TIMEOUT, DR_ERR_STATE = -6, -7, -8, -9, -10
+DR_VERSION = 1
+DR_SRC_FSDP_FLAT = 1
+DR_DST_ROLLOUT_FUSED = 1
+DR_F32, DR_BF16 = 1, 2
+DR_MAX_STAGE_BUFS = 8
+
+EXPORTS = ["dr_plan_create", "dr_plan_create_host", "dr_plan_query", "dr_plan_tensor", "dr_plan_segment",
+           "dr_reshard", "dr_reshard_inverse", "dr_stage_out", "dr_stage_in", "dr_plan_destroy", "dr_strerror",
+           "dr_last_error"]
+
+u8, u32, u64, i64, vp = C.c_uint8, C.c_uint32, C.c_uint64, C.c_int64, C.c_void_p
+
+
+class dr_model_spec(C.Structure):
+    _fields_ = [("struct_size", u32), ("version", u32), ("n_layers", u32), ("hidden", u32), ("n_q_heads", u32),
+                ("n_kv_heads", u32), ("head_dim", u32), ("ffn", u32), ("vocab", u32), ("n_experts", u32),
+                ("moe_ffn", u32), ("tied_embeddings", u8), ("qk_norm", u8), ("pad", u8 * 2)]
+
+
+class dr_src_layout(C.Structure):
+    _fields_ = [("struct_size", u32), ("kind", u32), ("dtype", u32), ("world", u32), ("rank", u32),
+                ("gathered", u32), ("align_elems", u32)]
+
+
+class dr_dst_layout(C.Structure):
+    _fields_ = [("struct_size", u32), ("kind", u32), ("dtype", u32), ("moe_tp", u32), ("arena_align_bytes", u32)]
+
+
+class dr_plan_info(C.Structure):
+    _fields_ = [(n, u64) for n in ("flat_elems", "shard_elems", "src_bytes", "dst_bytes", "n_tensors", "n_segments",
+                                   "n_tiles", "elems_moved", "bytes_moved_fwd", "bytes_moved_inv")]
+
+
+class dr_tensor_desc(C.Structure):
+    _fields_ = [("name", C.c_char * 64), ("arena_off", u64), ("rows", u64), ("cols", u64), ("alias_of", i64)]
+
+
+class dr_segment_desc(C.Structure):
+    _fields_ = [("dst_off", u64), ("src_off", u64), ("rows", u64), ("row_len", u64), ("src_row_stride", u64),
+                ("dst_row_stride", u64), ("vector_bytes", u32), ("tensor", u32)]
+
+
+dr_chunk_fn = C.CFUNCTYPE(C.c_int, vp, u64, u64, vp, u64)
+
+
+class dr_stage_desc(C.Structure):
+    _fields_ = [("struct_size", u32), ("n_bufs", u32), ("dev_ptr", vp * 8), ("bytes", u64 * 8), ("order", u32 * 8),
+                ("budget_bytes", u64), ("chunk_bytes", u64), ("host_arena", vp), ("host_arena_bytes", u64),
+                ("callback", dr_chunk_fn), ("user", vp), ("relay_dev", vp * 8), ("first_chunk", u64),
+                ("wait_event", vp), ("ready_events", vp * 8), ("timeout_ms", u32), ("flags", u32)]
+
+
+class dr_stage_stats(C.Structure):
+    _fields_ = [("bytes", u64), ("chunks_done", u64), ("n_chunks", u64), ("elapsed_ms", C.c_double),
+                ("link_gbs", C.c_double), ("pinned_high_water_bytes", u64), ("ready_ms", C.c_double * 8)]
+
+
+class DrError(RuntimeError):
+    def __init__(self, status: int, where: str):
+        self.status = status
+        super().__init__(f"{where}: {dr_strerror(status)} ({status}): {dr_last_error()}")
+
+
+_lib = None
+
+
+def lib() -> C.CDLL:
+    """The loaded C-ABI library.  Raises if it has not been built: there is no other code path."""
+    global _lib
+    if _lib is None:
+        if not os.path.exists(lib_path):
+            raise ImportError(f"{lib_path} is missing: run `python -m paper_2607_22614_b200.build` "
+                              "(the CUDA library is the only implementation)")
+        L = C.CDLL(lib_path)
+        P = C.POINTER
+        L.dr_plan_create.argtypes = [P(dr_model_spec), P(dr_src_layout), P(dr_dst_layout), u32, u32, P(vp)]
+        L.dr_plan_create_host.argtypes = L.dr_plan_create.argtypes
+        L.dr_plan_query.argtypes = [vp, P(dr_plan_info)]
+        L.dr_plan_tensor.argtypes = [vp, u32, P(dr_tensor_desc)]
+        L.dr_plan_segment.argtypes = [vp, u64, P(dr_segment_desc)]
+        L.dr_reshard.argtypes = [vp, vp, u64, vp, u64, vp]
+        L.dr_reshard_inverse.argtypes = [vp, vp, u64, vp, u64, vp]
+        L.dr_stage_out.argtypes = [vp, P(dr_stage_desc), P(dr_stage_stats)]
+        L.dr_stage_in.argtypes = [vp, P(dr_stage_desc), P(dr_stage_stats)]
+        L.dr_plan_destroy.argtypes = [vp]
+        for n in EXPORTS:
+            getattr(L, n).restype = C.c_int
+        L.dr_strerror.argtypes = [C.c_int]
+        L.dr_strerror.restype = C.c_char_p
+        L.dr_last_error.argtypes = []
+        L.dr_last_error.restype = C.c_char_p
+        _lib = L
+    return _lib
+
+
+# ---- struct helpers ----------------------------------------------------------------------------
+def model_spec(spec: dict) -> dr_model_spec:
+    return dr_model_spec(struct_size=C.sizeof(dr_model_spec), version=DR_VERSION, n_layers=spec["n_layers"],
+                         hidden=spec["hidden"], n_q_heads=spec["n_q_heads"], n_kv_heads=spec["n_kv_heads"],
+                         head_dim=spec["head_dim"], ffn=spec.get("ffn", 0), vocab=spec["vocab"],
+                         n_experts=spec.get("n_experts", 0), moe_ffn=spec.get("moe_ffn", 0),
+                         tied_embeddings=int(spec.get("tied", 0)), qk_norm=int(spec.get("qk_norm", 1)))
+
+
+def src_layout(world=1, rank=0, gathered=True, align_elems=1) -> dr_src_layout:
+    return dr_src_layout(struct_size=C.sizeof(dr_src_layout), kind=DR_SRC_FSDP_FLAT, dtype=DR_F32, world=world,
+                         rank=rank, gathered=int(gathered), align_elems=align_elems)
+
+
+def dst_layout(dtype=DR_BF16, arena_align_bytes=256, moe_tp=1) -> dr_dst_layout:
+    return dr_dst_layout(struct_size=C.sizeof(dr_dst_layout), kind=DR_DST_ROLLOUT_FUSED, dtype=dtype, moe_tp=moe_tp,
+                         arena_align_bytes=arena_align_bytes)
+
+
+def stage_desc(dev_ptrs, sizes, budget, chunk=0, order=None, host_arena=None, host_arena_bytes=0, callback=None,
+               relay_dev=None, first_chunk=0, wait_event=None, ready_events=None, timeout_ms=0) -> dr_stage_desc:
+    d = dr_stage_desc()
+    d.struct_size = C.sizeof(dr_stage_desc)
+    d.n_bufs = len(dev_ptrs)
+    for i, (p, n) in enumerate(zip(dev_ptrs, sizes)):
+        d.dev_ptr[i] = p
+        d.bytes[i] = n
+    for i, o in enumerate(order if order is not None else range(len(dev_ptrs))):
+        d.order[i] = o
+    d.budget_bytes, d.chunk_bytes, d.first_chunk, d.timeout_ms = budget, chunk, first_chunk, timeout_ms
+    d.host_arena, d.host_arena_bytes = host_arena, host_arena_bytes
+    if callback is not None:
+        d.callback = callback
+    for i, p in enumerate(relay_dev or []):
+        d.relay_dev[i] = p
+    d.wait_event = wait_event
+    for i, e in enumerate(ready_events or []):
+        d.ready_events[i] = e
+    return d
+
+
+# ---- the C calls, same names, status codes returned as-is ---------------------------------------
+def dr_plan_create(spec, src, dst, tp, rank):
+    h = vp()
+    rc = lib().dr_plan_create(C.byref(spec), C.byref(src), C.byref(dst), tp, rank, C.byref(h))
+    return rc, h
+
+
+def dr_plan_create_host(spec, src, dst, tp, rank):
+    h = vp()
+    rc = lib().dr_plan_create_host(C.byref(spec), C.byref(src), C.byref(dst), tp, rank, C.byref(h))
+    return rc, h
+
+
+def dr_plan_query(plan):
+    info = dr_plan_info()
+    return lib().dr_plan_query(plan, C.byref(info)), info
+
+
+def dr_plan_tensor(plan, i):
+    t = dr_tensor_desc()
+    return lib().dr_plan_tensor(plan, i, C.byref(t)), t
+
+
+def dr_plan_segment(plan, i):
+    s = dr_segment_desc()
+    return lib().dr_plan_segment(plan, i, C.byref(s)), s
+
+
+def dr_reshard(plan, src_dev, src_bytes, dst_dev, dst_bytes, cuda_stream):
+    return lib().dr_reshard(plan, src_dev, src_bytes, dst_dev, dst_bytes, cuda_stream)
+
+
+def dr_reshard_inverse(plan, rollout_dev, rollout_bytes, flat_dev, flat_bytes, cuda_stream):
+    return lib().dr_reshard_inverse(plan, rollout_dev, rollout_bytes, flat_dev, flat_bytes, cuda_stream)
+
+
+def dr_stage_out(plan, desc):
+    st = dr_stage_stats()
+    return lib().dr_stage_out(plan, C.byref(desc), C.byref(st)), st
+
+
+def dr_stage_in(plan, desc):
+    st = dr_stage_stats()
+    return lib().dr_stage_in(plan, C.byref(desc), C.byref(st)), st
+
+
+def dr_plan_destroy(plan):
+    return lib().dr_plan_destroy(plan)
+
+
+def dr_strerror(status: int) -> str:
+    return lib().dr_strerror(status).decode()
+
+
+def dr_last_error() -> str:
+    return lib().dr_last_error().decode()
+
+
+# ---- convenience wrapper (raises instead of returning codes; still marshalling only) -------------
+class Plan:
+    """Owns one ``dr_plan``.  ``host_only=True`` builds the planner's tables without touching CUDA."""
+
+    def __init__(self, spec: dict, *, world=1, rank=0, gathered=True, align_elems=1, tp=1, tp_rank=0,
+                 dtype=DR_BF16, arena_align_bytes=256, host_only=False):
+        create = dr_plan_create_host if host_only else dr_plan_create
+        rc, self.handle = create(model_spec(spec), src_layout(world, rank, gathered, align_elems),
+                                 dst_layout(dtype, arena_align_bytes), tp, tp_rank)
+        if rc:
+            self.handle = None
+            raise DrError(rc, "dr_plan_create")
+        rc, self.info = dr_plan_query(self.handle)
+        if rc:
+            raise DrError(rc, "dr_plan_query")
+
+    def close(self):
+        if getattr(self, "handle", None):
+            dr_plan_destroy(self.handle)
+            self.handle = None
+
+    __del__ = close
+
+    def tensors(self):
+        out = []
+        for i in range(self.info.n_tensors):
+            rc, t = dr_plan_tensor(self.handle, i)
+            if rc:
+                raise DrError(rc, "dr_plan_tensor")
+            out.append(t)
+        return out
+
+    def segments(self):
+        out = []
+        for i in range(self.info.n_segments):
+            rc, s = dr_plan_segment(self.handle, i)
+            if rc:
+                raise DrError(rc, "dr_plan_segment")
+            out.append(s)
+        return out
+
+    @staticmethod
+    def _stream(stream):
+        if stream is None:
+            import torch
+            return torch.cuda.current_stream().cuda_stream
+        return getattr(stream, "cuda_stream", stream)
+
+    def reshard(self, src, dst, stream=None):
+        """src: CUDA tensor holding the flat fp32 buffer; dst: CUDA tensor holding the rollout arena."""
+        rc = dr_reshard(self.handle, src.data_ptr(), src.numel() * src.element_size(), dst.data_ptr(),
+                        dst.numel() * dst.element_size(), self._stream(stream))
+        if rc:
+            raise DrError(rc, "dr_reshard")
+
+    def reshard_inverse(self, rollout, flat, stream=None):
+        rc = dr_reshard_inverse(self.handle, rollout.data_ptr(), rollout.numel() * rollout.element_size(),
+                                flat.data_ptr(), flat.numel() * flat.element_size(), self._stream(stream))
+        if rc:
+            raise DrError(rc, "dr_reshard_inverse")
+
+    def stage_out(self, desc):
+        rc, st = dr_stage_out(self.handle, desc)
+        if rc:
+            e = DrError(rc, "dr_stage_out")
+            e.stats = st
+            raise e
+        return st
+
+    def stage_in(self, desc):
+        rc, st = dr_stage_in(self.handle, desc)
+        if rc:
+            e = DrError(rc, "dr_stage_in")
+            e.stats = st
+            raise e
+        return st

@@ -1,0 +1,246 @@
+// C ABI entry points: argument validation, plan lifetime, reshard enqueue.
+#include <cuda_runtime.h>
+
+#include <cstdarg>
+#include <cstring>
+#include <new>
+
+#include "dr_internal.h"
+
+namespace dr {
+
+static thread_local char g_err[512] = "";
+
+void set_error(const char* fmt, ...)
+{
+    va_list ap;
+    va_start(ap, fmt);
+    vsnprintf(g_err, sizeof g_err, fmt, ap);
+    va_end(ap);
+}
+
+namespace {
+
+int validate(const dr_model_spec* s, const dr_src_layout* a, const dr_dst_layout* b, uint32_t tp, uint32_t rank)
+{
+    if (!s || !a || !b) {
+        set_error("NULL spec or layout");
+        return DR_ERR_INVALID;
+    }
+    if (s->struct_size != sizeof(dr_model_spec) || s->version != DR_VERSION || a->struct_size != sizeof(dr_src_layout) ||
+        b->struct_size != sizeof(dr_dst_layout)) {
+        set_error("struct_size / version mismatch");
+        return DR_ERR_INVALID;
+    }
+    if (a->kind != DR_SRC_FSDP_FLAT || a->dtype != DR_F32 || b->kind != DR_DST_ROLLOUT_FUSED ||
+        (b->dtype != DR_BF16 && b->dtype != DR_F32)) {
+        set_error("unknown layout kind or dtype");
+        return DR_ERR_UNSUPPORTED;
+    }
+    if (!s->hidden || !s->n_q_heads || !s->n_kv_heads || !s->head_dim || !s->vocab ||
+        (s->n_experts == 0 ? !s->ffn : !s->moe_ffn)) {
+        set_error("zero model dimension");
+        return DR_ERR_INVALID;
+    }
+    if (!a->world || a->rank >= a->world || !a->align_elems || a->gathered > 1 || !tp || rank >= tp) {
+        set_error("world/rank/tp/align out of range");
+        return DR_ERR_INVALID;
+    }
+    uint32_t al = b->arena_align_bytes;
+    if (al < 16 || (al & (al - 1))) {
+        set_error("arena_align_bytes must be a power of two >= 16");
+        return DR_ERR_INVALID;
+    }
+    if (b->moe_tp != 1) {
+        set_error("moe_tp must be 1 (experts are not sliced)");
+        return DR_ERR_UNSUPPORTED;
+    }
+    if (s->n_q_heads % tp || s->n_kv_heads % tp || s->vocab % tp || (s->n_experts == 0 && s->ffn % tp)) {
+        set_error("n_q_heads, n_kv_heads, ffn and vocab must be divisible by tp (no replication or padding)");
+        return DR_ERR_UNSUPPORTED;
+    }
+    return DR_OK;
+}
+
+int create(const dr_model_spec* s, const dr_src_layout* a, const dr_dst_layout* b, uint32_t tp, uint32_t rank,
+           bool host_only, dr_plan** out)
+{
+    if (!out) {
+        set_error("NULL out");
+        return DR_ERR_INVALID;
+    }
+    *out = nullptr;
+    int rc = validate(s, a, b, tp, rank);
+    if (rc) return rc;
+    dr_plan* p = new (std::nothrow) dr_plan();
+    if (!p) return DR_ERR_NOMEM;
+    p->spec = *s;
+    p->src = *a;
+    p->dst = *b;
+    p->tp = tp;
+    p->tp_rank = rank;
+    p->elem_size = b->dtype == DR_BF16 ? 2 : 4;
+    p->host_only = host_only;
+    try {
+        rc = compile_plan(p);
+    } catch (const std::bad_alloc&) {
+        rc = DR_ERR_NOMEM;
+    }
+    if (rc == DR_OK && !host_only) {
+        cudaError_t e = cudaGetDevice(&p->device);
+        size_t bytes = p->dev_segs.size() * sizeof(DevSeg);
+        if (e == cudaSuccess && bytes) e = cudaMalloc((void**)&p->d_segs, bytes);
+        if (e == cudaSuccess && bytes) e = cudaMemcpy(p->d_segs, p->dev_segs.data(), bytes, cudaMemcpyHostToDevice);
+        if (e == cudaSuccess) p->grid = choose_grid(p->device, p->elem_size);
+        if (e != cudaSuccess || p->grid <= 0) {
+            set_error("plan upload: %s", cudaGetErrorString(e));
+            rc = e == cudaErrorMemoryAllocation ? DR_ERR_NOMEM : DR_ERR_CUDA;
+        }
+    }
+    if (rc) {
+        dr_plan_destroy(p);
+        return rc;
+    }
+    *out = p;
+    return DR_OK;
+}
+
+int check_call(const dr_plan* p, const void* a, uint64_t a_bytes, uint64_t a_need, const void* b, uint64_t b_bytes,
+               uint64_t b_need)
+{
+    if (!p || (!a && a_need) || (!b && b_need)) {
+        set_error("NULL plan or buffer");
+        return DR_ERR_INVALID;
+    }
+    if (p->host_only) {
+        set_error("host-only plan cannot launch");
+        return DR_ERR_STATE;
+    }
+    if (a_bytes < a_need || b_bytes < b_need) {
+        set_error("buffer too small: have %llu / %llu bytes, need %llu / %llu", (unsigned long long)a_bytes,
+                  (unsigned long long)b_bytes, (unsigned long long)a_need, (unsigned long long)b_need);
+        return DR_ERR_SIZE;
+    }
+    if (((uintptr_t)a | (uintptr_t)b) & 15) {
+        set_error("base pointers must be 16-byte aligned");
+        return DR_ERR_ALIGN;
+    }
+    int dev = -1;
+    if (cudaGetDevice(&dev) != cudaSuccess || dev != p->device) {
+        set_error("current device differs from the plan's device");
+        return DR_ERR_STATE;
+    }
+    return DR_OK;
+}
+
+}  // namespace
+}  // namespace dr
+
+using namespace dr;
+
+extern "C" {
+
+int dr_plan_create(const dr_model_spec* spec, const dr_src_layout* src, const dr_dst_layout* dst, uint32_t tp,
+                   uint32_t rank, dr_plan** out)
+{
+    return create(spec, src, dst, tp, rank, false, out);
+}
+
+int dr_plan_create_host(const dr_model_spec* spec, const dr_src_layout* src, const dr_dst_layout* dst, uint32_t tp,
+                        uint32_t rank, dr_plan** out)
+{
+    return create(spec, src, dst, tp, rank, true, out);
+}
+
+int dr_plan_query(const dr_plan* plan, dr_plan_info* out)
+{
+    if (!plan || !out) {
+        set_error("NULL argument");
+        return DR_ERR_INVALID;
+    }
+    *out = plan->info;
+    return DR_OK;
+}
+
+int dr_plan_tensor(const dr_plan* plan, uint32_t i, dr_tensor_desc* out)
+{
+    if (!plan || !out || i >= plan->tensors.size()) {
+        set_error("bad tensor index");
+        return DR_ERR_INVALID;
+    }
+    const Tensor& t = plan->tensors[i];
+    memset(out, 0, sizeof *out);
+    snprintf(out->name, sizeof out->name, "%s", t.name.c_str());
+    out->arena_off = t.arena_off;
+    out->rows = t.rows;
+    out->cols = t.cols;
+    out->alias_of = t.alias_of;
+    return DR_OK;
+}
+
+int dr_plan_segment(const dr_plan* plan, uint64_t i, dr_segment_desc* out)
+{
+    if (!plan || !out || i >= plan->segs.size()) {
+        set_error("bad segment index");
+        return DR_ERR_INVALID;
+    }
+    const HostSeg& g = plan->segs[i];
+    out->dst_off = g.dst_off;
+    out->src_off = g.src_off;
+    out->rows = g.rows;
+    out->row_len = g.row_len;
+    out->src_row_stride = g.src_stride;
+    out->dst_row_stride = g.dst_stride;
+    out->vector_bytes = (g.flags & kSegVec32) ? 32 : (g.flags & kSegVec16) ? 16 : 0;
+    out->tensor = g.tensor;
+    return DR_OK;
+}
+
+int dr_reshard(const dr_plan* plan, const void* src_dev, uint64_t src_bytes, void* dst_dev, uint64_t dst_bytes,
+               void* cuda_stream)
+{
+    int rc = check_call(plan, src_dev, src_bytes, plan ? plan->info.src_bytes : 0, dst_dev, dst_bytes,
+                        plan ? plan->info.dst_bytes : 0);
+    if (rc) return rc;
+    return launch_reshard(plan, false, src_dev, dst_dev, nullptr, cuda_stream);
+}
+
+int dr_reshard_inverse(const dr_plan* plan, const void* rollout_dev, uint64_t rollout_bytes, void* flat_dev,
+                       uint64_t flat_bytes, void* cuda_stream)
+{
+    int rc = check_call(plan, rollout_dev, rollout_bytes, plan ? plan->info.dst_bytes : 0, flat_dev, flat_bytes,
+                        plan ? plan->info.src_bytes : 0);
+    if (rc) return rc;
+    return launch_reshard(plan, true, nullptr, flat_dev, rollout_dev, cuda_stream);
+}
+
+int dr_plan_destroy(dr_plan* plan)
+{
+    if (!plan) return DR_OK;
+    if (plan->ring) ring_destroy(plan->ring);
+    if (plan->d_segs) cudaFree(plan->d_segs);
+    delete plan;
+    return DR_OK;
+}
+
+const char* dr_strerror(int status)
+{
+    switch (status) {
+    case DR_OK: return "ok";
+    case DR_ERR_INVALID: return "invalid argument";
+    case DR_ERR_UNSUPPORTED: return "unsupported layout";
+    case DR_ERR_SIZE: return "buffer too small";
+    case DR_ERR_ALIGN: return "misaligned base pointer";
+    case DR_ERR_NOMEM: return "out of memory";
+    case DR_ERR_CUDA: return "CUDA error";
+    case DR_ERR_BUDGET: return "staging budget cannot hold two chunk slots";
+    case DR_ERR_SINK: return "chunk callback failed";
+    case DR_ERR_TIMEOUT: return "wait timed out";
+    case DR_ERR_STATE: return "call not valid in this state";
+    default: return "unknown status";
+    }
+}
+
+const char* dr_last_error(void) { return g_err; }
+
+}  // extern "C"

@@ -1,0 +1,85 @@
+// Internal declarations shared by the planner, the kernels and the staging engine.
+#pragma once
+#include <cstdint>
+#include <cstdio>
+#include <memory>
+#include <mutex>
+#include <string>
+#include <vector>
+
+#include "dynaresize.h"
+
+namespace dr {
+
+// A work unit is 8 consecutive elements of one row (32 B of fp32, 16 B of bf16); a tile is
+// kTileUnits consecutive units of one segment.  One CTA iteration processes one tile.
+constexpr uint32_t kUnitElems = 8;
+constexpr uint32_t kTileUnits = 1024;
+// Contiguous runs are cut so that a segment's unit count fits 32 bits with room to spare.
+constexpr uint64_t kMaxSegElems = 1ull << 31;
+
+enum SegFlags : uint32_t {
+    kSegVec32 = 1u,      // flat-side addresses 32-byte aligned: 256-bit accesses allowed
+    kSegVec16 = 2u,      // flat-side addresses 16-byte aligned: 128-bit accesses
+    kSegContiguous = 4u  // rows == 1: no row/column split needed
+};
+
+// Device segment table entry (48 bytes).
+struct DevSeg {
+    uint64_t dst_off;        // bytes from the arena base
+    uint64_t src_off;        // elements from the flat buffer base
+    uint64_t tile0;          // index of this segment's first tile
+    uint32_t n_units;        // rows * units_per_row
+    uint32_t units_per_row;  // ceil(row_len / 8)
+    uint32_t row_len;        // elements
+    uint32_t src_stride;     // elements
+    uint32_t dst_stride;     // elements
+    uint32_t flags;
+};
+static_assert(sizeof(DevSeg) == 48, "DevSeg layout");
+
+struct HostSeg {
+    uint64_t dst_off, src_off, rows, row_len, src_stride, dst_stride;
+    uint32_t flags, tensor;
+};
+
+struct Tensor {
+    std::string name;
+    uint64_t arena_off = 0, rows = 0, cols = 0;
+    int64_t alias_of = -1;
+};
+
+struct Ring;  // pinned staging ring + worker pool (staging.cu)
+
+}  // namespace dr
+
+struct dr_plan {
+    dr_model_spec spec{};
+    dr_src_layout src{};
+    dr_dst_layout dst{};
+    uint32_t tp = 1, tp_rank = 0;
+    uint32_t elem_size = 2;  // rollout element size in bytes
+    dr_plan_info info{};
+    std::vector<dr::Tensor> tensors;
+    std::vector<dr::HostSeg> segs;
+    std::vector<dr::DevSeg> dev_segs;  // host copy of the device table
+    // device side (absent on a host-only plan)
+    bool host_only = true;
+    int device = -1;
+    dr::DevSeg* d_segs = nullptr;
+    int grid = 0;
+    // staging
+    std::mutex stage_mu;
+    dr::Ring* ring = nullptr;
+};
+
+namespace dr {
+
+void set_error(const char* fmt, ...);
+int compile_plan(dr_plan* p);  // planner.cpp: fills tensors, segs, dev_segs, info
+int launch_reshard(const dr_plan* p, bool inverse, const void* flat, void* arena_or_flat_out, const void* arena_in,
+                   void* stream);
+int choose_grid(int device, uint32_t elem_size);  // resident CTAs of the reshard kernel on the whole GPU
+void ring_destroy(Ring* r);
+
+}  // namespace dr

@@ -1,0 +1,301 @@
+// Gather / permute / cast kernels for sm_100a.
+//
+// The transform is pure data movement (4 B read + 2 B written per element, no contraction), so the
+// design goal is HBM bandwidth: every thread keeps several 256-bit loads in flight, each warp-level
+// access is one fully coalesced 1 KB (load) or 512 B (store) request, the flat buffer and the arena are
+// streamed past L1, and the grid is persistent (a multiple of the SM count) with a cheap walk through
+// the segment table instead of a per-element lookup.
+#include <cuda_runtime.h>
+
+#include "dr_internal.h"
+
+namespace dr {
+namespace {
+
+constexpr int kThreads = 256;
+constexpr int kUnroll = kTileUnits / kThreads;  // units per thread per tile
+static_assert(kTileUnits % kThreads == 0, "tile must be a whole number of thread sweeps");
+
+// ---- memory access helpers (inline PTX: 256-bit accesses and cache hints) ----------------------
+struct V8 {
+    uint32_t w[8];
+};
+struct V4 {
+    uint32_t w[4];
+};
+
+__device__ __forceinline__ V8 ld256(const void* p)
+{
+    V8 v;
+    asm volatile("ld.global.nc.L1::no_allocate.v8.b32 {%0,%1,%2,%3,%4,%5,%6,%7}, [%8];"
+                 : "=r"(v.w[0]), "=r"(v.w[1]), "=r"(v.w[2]), "=r"(v.w[3]), "=r"(v.w[4]), "=r"(v.w[5]), "=r"(v.w[6]),
+                   "=r"(v.w[7])
+                 : "l"(p));
+    return v;
+}
+__device__ __forceinline__ V4 ld128(const void* p)
+{
+    V4 v;
+    asm volatile("ld.global.nc.L1::no_allocate.v4.b32 {%0,%1,%2,%3}, [%4];"
+                 : "=r"(v.w[0]), "=r"(v.w[1]), "=r"(v.w[2]), "=r"(v.w[3])
+                 : "l"(p));
+    return v;
+}
+__device__ __forceinline__ uint32_t ld32(const void* p)
+{
+    uint32_t v;
+    asm volatile("ld.global.nc.L1::no_allocate.b32 %0, [%1];" : "=r"(v) : "l"(p));
+    return v;
+}
+__device__ __forceinline__ uint16_t ld16(const void* p)
+{
+    uint16_t v;
+    asm volatile("ld.global.nc.L1::no_allocate.b16 %0, [%1];" : "=h"(v) : "l"(p));
+    return v;
+}
+__device__ __forceinline__ void st256(void* p, const V8& v)
+{
+    asm volatile("st.global.L1::no_allocate.v8.b32 [%0], {%1,%2,%3,%4,%5,%6,%7,%8};" ::"l"(p), "r"(v.w[0]), "r"(v.w[1]),
+                 "r"(v.w[2]), "r"(v.w[3]), "r"(v.w[4]), "r"(v.w[5]), "r"(v.w[6]), "r"(v.w[7])
+                 : "memory");
+}
+__device__ __forceinline__ void st128(void* p, const V4& v)
+{
+    asm volatile("st.global.L1::no_allocate.v4.b32 [%0], {%1,%2,%3,%4};" ::"l"(p), "r"(v.w[0]), "r"(v.w[1]),
+                 "r"(v.w[2]), "r"(v.w[3])
+                 : "memory");
+}
+__device__ __forceinline__ void st32(void* p, uint32_t v)
+{
+    asm volatile("st.global.L1::no_allocate.b32 [%0], %1;" ::"l"(p), "r"(v) : "memory");
+}
+__device__ __forceinline__ void st16(void* p, uint16_t v)
+{
+    asm volatile("st.global.L1::no_allocate.b16 [%0], %1;" ::"l"(p), "h"(v) : "memory");
+}
+
+// fp32 -> bf16, round to nearest even, in hardware: NaN becomes 0x7FFF, subnormals are rounded (the
+// instruction has no flush-to-zero form), overflow goes to infinity.
+__device__ __forceinline__ uint32_t cvt_pair(uint32_t lo, uint32_t hi)
+{
+    uint32_t d;
+    asm("cvt.rn.bf16x2.f32 %0, %1, %2;" : "=r"(d) : "f"(__uint_as_float(hi)), "f"(__uint_as_float(lo)));
+    return d;
+}
+__device__ __forceinline__ uint16_t cvt_one(uint32_t x)
+{
+    uint16_t d;
+    asm("cvt.rn.bf16.f32 %0, %1;" : "=h"(d) : "f"(__uint_as_float(x)));
+    return d;
+}
+__device__ __forceinline__ V4 narrow(const V8& v)
+{
+    V4 o;
+    o.w[0] = cvt_pair(v.w[0], v.w[1]);
+    o.w[1] = cvt_pair(v.w[2], v.w[3]);
+    o.w[2] = cvt_pair(v.w[4], v.w[5]);
+    o.w[3] = cvt_pair(v.w[6], v.w[7]);
+    return o;
+}
+__device__ __forceinline__ V8 widen(const V4& v)
+{
+    V8 o;
+#pragma unroll
+    for (int i = 0; i < 4; ++i) {
+        o.w[2 * i] = v.w[i] << 16;
+        o.w[2 * i + 1] = v.w[i] & 0xFFFF0000u;
+    }
+    return o;
+}
+
+// flat side: fp32 at 16- or 32-byte aligned addresses
+__device__ __forceinline__ V8 load_flat(const char* p, bool wide)
+{
+    if (wide) return ld256(p);
+    V4 a = ld128(p), b = ld128(p + 16);
+    return V8{{a.w[0], a.w[1], a.w[2], a.w[3], b.w[0], b.w[1], b.w[2], b.w[3]}};
+}
+__device__ __forceinline__ void store_flat(char* p, const V8& v, bool wide)
+{
+    if (wide) {
+        st256(p, v);
+    } else {
+        st128(p, V4{{v.w[0], v.w[1], v.w[2], v.w[3]}});
+        st128(p + 16, V4{{v.w[4], v.w[5], v.w[6], v.w[7]}});
+    }
+}
+
+// Last segment whose first tile is <= tile, searching upward from `from`.
+__device__ __forceinline__ uint32_t find_segment(const DevSeg* __restrict__ segs, uint32_t n_segs, uint32_t from,
+                                                 uint64_t tile)
+{
+    // the common case is one of the next few entries
+    uint32_t s = from;
+#pragma unroll 1
+    for (int probe = 0; probe < 4; ++probe) {
+        if (s + 1 >= n_segs || segs[s + 1].tile0 > tile) return s;
+        ++s;
+    }
+    uint32_t lo = s, hi = n_segs;  // invariant: segs[lo].tile0 <= tile, (hi == n_segs or segs[hi].tile0 > tile)
+    while (hi - lo > 1) {
+        uint32_t mid = lo + (hi - lo) / 2;
+        if (segs[mid].tile0 <= tile) lo = mid; else hi = mid;
+    }
+    return lo;
+}
+
+// ES: rollout element size (2 = bf16, 4 = fp32).  INV: false = flat -> arena, true = arena -> flat.
+// BLOCKED: each CTA takes one contiguous range of tiles; otherwise tiles are dealt round-robin.
+template <int ES, bool INV, bool BLOCKED>
+__global__ void __launch_bounds__(kThreads) reshard_kernel(const DevSeg* __restrict__ segs, uint32_t n_segs,
+                                                          uint64_t n_tiles, char* __restrict__ flat,
+                                                          char* __restrict__ arena, int allow256)
+{
+    uint64_t tile, last, step;
+    if (BLOCKED) {
+        uint64_t per = (n_tiles + gridDim.x - 1) / gridDim.x;
+        tile = per * blockIdx.x;
+        last = tile + per < n_tiles ? tile + per : n_tiles;
+        step = 1;
+    } else {
+        tile = blockIdx.x;
+        last = n_tiles;
+        step = gridDim.x;
+    }
+    if (tile >= last) return;
+
+    uint32_t si = find_segment(segs, n_segs, 0, tile);
+    DevSeg g = segs[si];
+    uint64_t seg_end = si + 1 < n_segs ? segs[si + 1].tile0 : n_tiles;
+
+    for (; tile < last; tile += step) {
+        if (tile >= seg_end) {
+            si = find_segment(segs, n_segs, si, tile);
+            g = segs[si];
+            seg_end = si + 1 < n_segs ? segs[si + 1].tile0 : n_tiles;
+        }
+        const uint32_t u0 = (uint32_t)(tile - g.tile0) * kTileUnits + threadIdx.x;
+        const char* fbase = flat + g.src_off * 4;
+        char* abase = arena + g.dst_off;
+        const bool contiguous = g.flags & kSegContiguous;
+
+        if (g.flags & (kSegVec32 | kSegVec16)) {
+            const bool wide = (g.flags & kSegVec32) && allow256;
+            uint64_t fo[kUnroll], ao[kUnroll];
+            bool ok[kUnroll];
+#pragma unroll
+            for (int j = 0; j < kUnroll; ++j) {
+                uint32_t u = u0 + j * kThreads;
+                ok[j] = u < g.n_units;
+                if (contiguous) {
+                    fo[j] = (uint64_t)u * 8;
+                    ao[j] = (uint64_t)u * 8;
+                } else {
+                    uint32_t row = u / g.units_per_row;
+                    uint32_t col = (u - row * g.units_per_row) * 8;
+                    fo[j] = (uint64_t)row * g.src_stride + col;
+                    ao[j] = (uint64_t)row * g.dst_stride + col;
+                }
+            }
+            if (!INV) {
+                V8 v[kUnroll];
+#pragma unroll
+                for (int j = 0; j < kUnroll; ++j)
+                    if (ok[j]) v[j] = load_flat(fbase + fo[j] * 4, wide);
+#pragma unroll
+                for (int j = 0; j < kUnroll; ++j) {
+                    if (!ok[j]) continue;
+                    if (ES == 2) st128(abase + ao[j] * 2, narrow(v[j]));
+                    else store_flat(abase + ao[j] * 4, v[j], allow256);
+                }
+            } else if (ES == 2) {
+                V4 v[kUnroll];
+#pragma unroll
+                for (int j = 0; j < kUnroll; ++j)
+                    if (ok[j]) v[j] = ld128(abase + ao[j] * 2);
+#pragma unroll
+                for (int j = 0; j < kUnroll; ++j)
+                    if (ok[j]) store_flat((char*)fbase + fo[j] * 4, widen(v[j]), wide);
+            } else {
+                V8 v[kUnroll];
+#pragma unroll
+                for (int j = 0; j < kUnroll; ++j)
+                    if (ok[j]) v[j] = load_flat(abase + ao[j] * 4, allow256);
+#pragma unroll
+                for (int j = 0; j < kUnroll; ++j)
+                    if (ok[j]) store_flat((char*)fbase + fo[j] * 4, v[j], wide);
+            }
+        } else {
+            // Scalar path for runs that start or end off the vector grid (odd shapes, shard cuts):
+            // element e of the tile is handled by thread e % 256, so accesses stay coalesced.
+            const uint64_t e0 = (uint64_t)(tile - g.tile0) * kTileUnits * 8;
+#pragma unroll 1
+            for (uint32_t k = threadIdx.x; k < kTileUnits * 8; k += kThreads) {
+                uint64_t e = e0 + k;  // element index in the segment's padded unit space
+                uint64_t row, col;
+                if (contiguous) {
+                    row = 0;
+                    col = e;
+                } else {
+                    uint64_t per_row = (uint64_t)g.units_per_row * 8;
+                    row = e / per_row;
+                    col = e - row * per_row;
+                }
+                if (col >= g.row_len || row * g.units_per_row >= g.n_units) continue;
+                const char* fp = fbase + (row * g.src_stride + col) * 4;
+                char* ap = abase + (row * g.dst_stride + col) * ES;
+                if (!INV) {
+                    uint32_t x = ld32(fp);
+                    if (ES == 2) st16(ap, cvt_one(x)); else st32(ap, x);
+                } else {
+                    uint32_t x = ES == 2 ? (uint32_t)ld16(ap) << 16 : ld32(ap);
+                    st32((char*)fp, x);
+                }
+            }
+        }
+    }
+}
+
+}  // namespace
+
+int choose_grid(int device, uint32_t elem_size)
+{
+    int sms = 0, per_sm = 0;
+    if (cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, device) != cudaSuccess || sms <= 0) return 0;
+    cudaError_t e = elem_size == 2
+        ? cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, reshard_kernel<2, false, false>, kThreads, 0)
+        : cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, reshard_kernel<4, false, false>, kThreads, 0);
+    if (e != cudaSuccess || per_sm <= 0) return 0;
+    return sms * per_sm;  // one wave of resident CTAs: the kernel is persistent
+}
+
+int launch_reshard(const dr_plan* p, bool inverse, const void* flat, void* arena_or_flat_out, const void* arena_in,
+                   void* stream)
+{
+    // forward: flat = source, arena_or_flat_out = arena.  inverse: arena_in = source, arena_or_flat_out = flat.
+    char* f = inverse ? (char*)arena_or_flat_out : (char*)flat;
+    char* a = inverse ? (char*)arena_in : (char*)arena_or_flat_out;
+    const uint64_t n_tiles = p->info.n_tiles;
+    if (n_tiles == 0) return DR_OK;
+    const int allow256 = (((uintptr_t)f | (uintptr_t)a) & 31) == 0;
+    uint64_t g64 = n_tiles < (uint64_t)p->grid ? n_tiles : (uint64_t)p->grid;
+    dim3 grid((unsigned)g64), block(kThreads);
+    cudaStream_t s = (cudaStream_t)stream;
+    const uint32_t n_segs = (uint32_t)p->dev_segs.size();
+#define DR_LAUNCH(ES, INV) \
+    reshard_kernel<ES, INV, false><<<grid, block, 0, s>>>(p->d_segs, n_segs, n_tiles, f, a, allow256)
+    if (p->elem_size == 2) {
+        if (inverse) DR_LAUNCH(2, true); else DR_LAUNCH(2, false);
+    } else {
+        if (inverse) DR_LAUNCH(4, true); else DR_LAUNCH(4, false);
+    }
+#undef DR_LAUNCH
+    cudaError_t e = cudaGetLastError();
+    if (e != cudaSuccess) {
+        set_error("reshard kernel launch: %s", cudaGetErrorString(e));
+        return DR_ERR_CUDA;
+    }
+    return DR_OK;
+}
+
+}  // namespace dr

@@ -1,0 +1,437 @@
+// Bounded chunked host staging: a pinned ring of chunk slots, a copy stream and a relay stream,
+// and a small worker pool that moves chunks between the ring and a pageable host arena.
+// Every wait is a bounded host-side poll; there is no device-side waiting anywhere.
+#include <cuda_runtime.h>
+
+#include <algorithm>
+#include <atomic>
+#include <chrono>
+#include <condition_variable>
+#include <cstring>
+#include <functional>
+#include <thread>
+
+#include "dr_internal.h"
+
+namespace dr {
+
+namespace {
+
+using Clock = std::chrono::steady_clock;
+
+double ms_since(Clock::time_point t0) { return std::chrono::duration<double, std::milli>(Clock::now() - t0).count(); }
+
+// Splits one memcpy over a few threads: a single core cannot keep up with the host link.
+class CopyPool {
+public:
+    explicit CopyPool(unsigned n) : n_(n ? n : 1)
+    {
+        for (unsigned i = 1; i < n_; ++i) th_.emplace_back([this, i] { loop(i); });
+    }
+    ~CopyPool()
+    {
+        {
+            std::lock_guard<std::mutex> l(mu_);
+            stop_ = true;
+            ++gen_;
+        }
+        cv_.notify_all();
+        for (auto& t : th_) t.join();
+    }
+    void copy(void* dst, const void* src, uint64_t n)
+    {
+        if (n_ == 1 || n < (1u << 20)) {
+            memcpy(dst, src, n);
+            return;
+        }
+        {
+            std::lock_guard<std::mutex> l(mu_);
+            dst_ = (char*)dst;
+            src_ = (const char*)src;
+            len_ = n;
+            pending_ = n_ - 1;
+            ++gen_;
+        }
+        cv_.notify_all();
+        part(0);
+        std::unique_lock<std::mutex> l(mu_);
+        done_.wait(l, [this] { return pending_ == 0; });
+    }
+
+private:
+    void part(unsigned i)
+    {
+        uint64_t per = (len_ / n_ + 63) / 64 * 64;
+        uint64_t a = std::min<uint64_t>(len_, per * i), b = std::min<uint64_t>(len_, a + per);
+        if (i == n_ - 1) b = len_;
+        if (b > a) memcpy(dst_ + a, src_ + a, b - a);
+    }
+    void loop(unsigned i)
+    {
+        uint64_t seen = 0;
+        for (;;) {
+            {
+                std::unique_lock<std::mutex> l(mu_);
+                cv_.wait(l, [&] { return gen_ != seen; });
+                seen = gen_;
+                if (stop_) return;
+            }
+            part(i);
+            {
+                std::lock_guard<std::mutex> l(mu_);
+                --pending_;
+            }
+            done_.notify_one();
+        }
+    }
+    unsigned n_;
+    std::vector<std::thread> th_;
+    std::mutex mu_;
+    std::condition_variable cv_, done_;
+    uint64_t gen_ = 0;
+    unsigned pending_ = 0;
+    bool stop_ = false;
+    char* dst_ = nullptr;
+    const char* src_ = nullptr;
+    uint64_t len_ = 0;
+};
+
+}  // namespace
+
+struct Ring {
+    cudaStream_t s_copy = nullptr, s_relay = nullptr;
+    char* base = nullptr;  // pinned, slots * chunk bytes
+    uint64_t chunk = 0;
+    uint32_t slots = 0;
+    std::vector<cudaEvent_t> ev_copy, ev_relay;  // one per slot
+    std::unique_ptr<CopyPool> pool;
+};
+
+void ring_destroy(Ring* r)
+{
+    if (!r) return;
+    if (r->s_copy) cudaStreamSynchronize(r->s_copy);
+    if (r->s_relay) cudaStreamSynchronize(r->s_relay);
+    for (auto e : r->ev_copy) cudaEventDestroy(e);
+    for (auto e : r->ev_relay) cudaEventDestroy(e);
+    if (r->base) cudaFreeHost(r->base);
+    if (r->s_copy) cudaStreamDestroy(r->s_copy);
+    if (r->s_relay) cudaStreamDestroy(r->s_relay);
+    delete r;
+}
+
+namespace {
+
+#define DR_CUDA(call)                                                        \
+    do {                                                                     \
+        cudaError_t e_ = (call);                                             \
+        if (e_ != cudaSuccess) {                                             \
+            set_error("%s: %s", #call, cudaGetErrorString(e_));              \
+            return e_ == cudaErrorMemoryAllocation ? DR_ERR_NOMEM : DR_ERR_CUDA; \
+        }                                                                    \
+    } while (0)
+
+struct Geometry {
+    uint64_t total = 0, chunk = 0, n_chunks = 0;
+    uint32_t slots = 0;
+    uint64_t prefix[DR_MAX_STAGE_BUFS + 1] = {0};
+};
+
+int geometry(const dr_stage_desc* d, Geometry* g)
+{
+    if (!d || d->struct_size != sizeof(dr_stage_desc) || d->n_bufs == 0 || d->n_bufs > DR_MAX_STAGE_BUFS) {
+        set_error("bad staging descriptor");
+        return DR_ERR_INVALID;
+    }
+    for (uint32_t i = 0; i < d->n_bufs; ++i) {
+        if (!d->dev_ptr[i] && d->bytes[i]) {
+            set_error("NULL device buffer %u", i);
+            return DR_ERR_INVALID;
+        }
+        g->prefix[i + 1] = g->prefix[i] + d->bytes[i];
+    }
+    g->total = g->prefix[d->n_bufs];
+    g->chunk = d->chunk_bytes ? d->chunk_bytes : d->budget_bytes / 2 / 4096 * 4096;
+    if (g->chunk == 0 || d->budget_bytes / g->chunk < 2) {
+        set_error("budget %llu cannot hold two slots of %llu bytes", (unsigned long long)d->budget_bytes,
+                  (unsigned long long)g->chunk);
+        return DR_ERR_BUDGET;
+    }
+    g->slots = (uint32_t)std::min<uint64_t>(d->budget_bytes / g->chunk, 64);
+    g->n_chunks = (g->total + g->chunk - 1) / g->chunk;
+    return DR_OK;
+}
+
+int ensure_ring(dr_plan* p, const Geometry& g, bool need_memory)
+{
+    if (!p->ring) {
+        Ring* r = new (std::nothrow) Ring();
+        if (!r) return DR_ERR_NOMEM;
+        p->ring = r;
+        DR_CUDA(cudaStreamCreateWithFlags(&r->s_copy, cudaStreamNonBlocking));
+        DR_CUDA(cudaStreamCreateWithFlags(&r->s_relay, cudaStreamNonBlocking));
+        unsigned hw = std::thread::hardware_concurrency();
+        r->pool.reset(new CopyPool(std::max(1u, std::min(16u, hw / 2))));
+    }
+    Ring* r = p->ring;
+    while (r->ev_copy.size() < g.slots) {
+        cudaEvent_t a, b;
+        DR_CUDA(cudaEventCreateWithFlags(&a, cudaEventDisableTiming));
+        r->ev_copy.push_back(a);
+        DR_CUDA(cudaEventCreateWithFlags(&b, cudaEventDisableTiming));
+        r->ev_relay.push_back(b);
+    }
+    if (need_memory && (r->chunk != g.chunk || r->slots != g.slots)) {
+        if (r->base) {
+            DR_CUDA(cudaStreamSynchronize(r->s_copy));
+            DR_CUDA(cudaStreamSynchronize(r->s_relay));
+            cudaFreeHost(r->base);
+            r->base = nullptr;
+            r->chunk = 0;
+            r->slots = 0;
+        }
+        DR_CUDA(cudaHostAlloc((void**)&r->base, g.chunk * g.slots, cudaHostAllocDefault));
+        r->chunk = g.chunk;
+        r->slots = g.slots;
+    }
+    return DR_OK;
+}
+
+// Bounded wait for an event: poll, back off, give up at the deadline.
+int wait_event(cudaEvent_t ev, Clock::time_point deadline)
+{
+    for (unsigned spins = 0;; ++spins) {
+        cudaError_t e = cudaEventQuery(ev);
+        if (e == cudaSuccess) return DR_OK;
+        if (e != cudaErrorNotReady) {
+            set_error("cudaEventQuery: %s", cudaGetErrorString(e));
+            return DR_ERR_CUDA;
+        }
+        if (Clock::now() > deadline) {
+            set_error("staging wait timed out");
+            return DR_ERR_TIMEOUT;
+        }
+        if (spins < 200) std::this_thread::yield();
+        else std::this_thread::sleep_for(std::chrono::microseconds(20));
+    }
+}
+
+// Bounded drain of both streams on an error path, so that no copy still targets the ring on return.
+void drain(Ring* r, Clock::time_point deadline)
+{
+    for (cudaStream_t s : {r->s_copy, r->s_relay})
+        while (cudaStreamQuery(s) == cudaErrorNotReady && Clock::now() < deadline)
+            std::this_thread::sleep_for(std::chrono::microseconds(50));
+}
+
+bool is_pinned_host(const void* p)
+{
+    cudaPointerAttributes a{};
+    if (cudaPointerGetAttributes(&a, p) != cudaSuccess) {
+        cudaGetLastError();
+        return false;
+    }
+    return a.type == cudaMemoryTypeHost;
+}
+
+int check_common(dr_plan* p, const dr_stage_desc* d, const Geometry& g, bool out)
+{
+    if (p->host_only) {
+        set_error("host-only plan cannot stage");
+        return DR_ERR_STATE;
+    }
+    int n_sinks = (d->callback != nullptr) + (d->host_arena != nullptr) + (out && d->relay_dev[0] != nullptr);
+    if (n_sinks != 1) {
+        set_error("exactly one of callback, relay_dev, host_arena must be given");
+        return DR_ERR_INVALID;
+    }
+    if (d->host_arena && d->host_arena_bytes < g.total) {
+        set_error("host arena holds %llu bytes, stream is %llu", (unsigned long long)d->host_arena_bytes,
+                  (unsigned long long)g.total);
+        return DR_ERR_SIZE;
+    }
+    int dev = -1;
+    if (cudaGetDevice(&dev) != cudaSuccess || dev != p->device) {
+        set_error("current device differs from the plan's device");
+        return DR_ERR_STATE;
+    }
+    return DR_OK;
+}
+
+}  // namespace
+}  // namespace dr
+
+using namespace dr;
+
+extern "C" int dr_stage_out(dr_plan* plan, const dr_stage_desc* d, dr_stage_stats* stats)
+{
+    if (!plan) {
+        set_error("NULL plan");
+        return DR_ERR_INVALID;
+    }
+    Geometry g;
+    int rc = geometry(d, &g);
+    if (rc) return rc;
+    if ((rc = check_common(plan, d, g, true))) return rc;
+    std::lock_guard<std::mutex> lock(plan->stage_mu);
+    const bool relay = !d->callback && d->relay_dev[0];
+    const bool direct = !d->callback && !relay && is_pinned_host(d->host_arena);  // DMA straight into the arena
+    if ((rc = ensure_ring(plan, g, !direct))) return rc;
+    Ring* r = plan->ring;
+    const auto t0 = Clock::now();
+    const auto limit = std::chrono::milliseconds(d->timeout_ms ? d->timeout_ms : 60000);
+    dr_stage_stats st{};
+    st.n_chunks = g.n_chunks;
+    st.chunks_done = std::min<uint64_t>(d->first_chunk, g.n_chunks);
+    st.pinned_high_water_bytes = direct ? 0 : g.chunk * g.slots;
+    if (d->wait_event) DR_CUDA(cudaStreamWaitEvent(r->s_copy, (cudaEvent_t)d->wait_event, 0));
+
+    auto slot_ptr = [&](uint64_t k) -> char* {
+        return direct ? (char*)d->host_arena + k * g.chunk : r->base + (k % g.slots) * g.chunk;
+    };
+    // enqueue the copies of chunk k: one per buffer it touches
+    auto issue = [&](uint64_t k) -> int {
+        uint64_t lo = k * g.chunk, hi = std::min(lo + g.chunk, g.total);
+        uint32_t s = (uint32_t)(k % g.slots);
+        char* host = slot_ptr(k);
+        for (uint32_t b = 0; b < d->n_bufs; ++b) {
+            uint64_t a = std::max(lo, g.prefix[b]), e = std::min(hi, g.prefix[b + 1]);
+            if (a >= e) continue;
+            DR_CUDA(cudaMemcpyAsync(host + (a - lo), (const char*)d->dev_ptr[b] + (a - g.prefix[b]), e - a,
+                                    cudaMemcpyDeviceToHost, r->s_copy));
+        }
+        DR_CUDA(cudaEventRecord(r->ev_copy[s], r->s_copy));
+        if (relay) {
+            DR_CUDA(cudaStreamWaitEvent(r->s_relay, r->ev_copy[s], 0));
+            for (uint32_t b = 0; b < d->n_bufs; ++b) {
+                uint64_t a = std::max(lo, g.prefix[b]), e = std::min(hi, g.prefix[b + 1]);
+                if (a >= e) continue;
+                if (!d->relay_dev[b]) {
+                    set_error("relay_dev[%u] is NULL", b);
+                    return DR_ERR_INVALID;
+                }
+                DR_CUDA(cudaMemcpyAsync((char*)d->relay_dev[b] + (a - g.prefix[b]), host + (a - lo), e - a,
+                                        cudaMemcpyHostToDevice, r->s_relay));
+            }
+            DR_CUDA(cudaEventRecord(r->ev_relay[s], r->s_relay));
+        }
+        return DR_OK;
+    };
+    // wait for chunk k and hand it to the sink
+    auto complete = [&](uint64_t k) -> int {
+        uint64_t lo = k * g.chunk, n = std::min(lo + g.chunk, g.total) - lo;
+        uint32_t s = (uint32_t)(k % g.slots);
+        int w = wait_event(relay ? r->ev_relay[s] : r->ev_copy[s], Clock::now() + limit);
+        if (w) return w;
+        if (d->callback) {
+            if (d->callback(d->user, k, lo, slot_ptr(k), n)) {
+                set_error("chunk callback failed at chunk %llu", (unsigned long long)k);
+                return DR_ERR_SINK;
+            }
+        } else if (!relay && !direct) {
+            r->pool->copy((char*)d->host_arena + lo, slot_ptr(k), n);
+        }
+        st.bytes += n;
+        return DR_OK;
+    };
+
+    uint64_t next_issue = st.chunks_done, next_done = st.chunks_done;
+    while (rc == DR_OK && next_done < g.n_chunks) {
+        while (rc == DR_OK && next_issue < g.n_chunks && next_issue - next_done < g.slots) rc = issue(next_issue++);
+        if (rc == DR_OK && (rc = complete(next_done)) == DR_OK) st.chunks_done = ++next_done;
+    }
+    if (rc) drain(r, Clock::now() + limit);
+    st.elapsed_ms = ms_since(t0);
+    st.link_gbs = st.elapsed_ms > 0 ? (double)st.bytes / st.elapsed_ms * 1e-6 : 0;
+    if (stats) *stats = st;
+    return rc;
+}
+
+extern "C" int dr_stage_in(dr_plan* plan, const dr_stage_desc* d, dr_stage_stats* stats)
+{
+    if (!plan) {
+        set_error("NULL plan");
+        return DR_ERR_INVALID;
+    }
+    Geometry g;
+    int rc = geometry(d, &g);
+    if (rc) return rc;
+    if ((rc = check_common(plan, d, g, false))) return rc;
+    {
+        uint32_t seen = 0;
+        for (uint32_t i = 0; i < d->n_bufs; ++i)
+            if (d->order[i] < d->n_bufs) seen |= 1u << d->order[i];
+        if (seen != (1u << d->n_bufs) - 1) {
+            set_error("order[] must be a permutation of 0..n_bufs-1");
+            return DR_ERR_INVALID;
+        }
+    }
+    std::lock_guard<std::mutex> lock(plan->stage_mu);
+    const bool direct = !d->callback && is_pinned_host(d->host_arena);
+    if ((rc = ensure_ring(plan, g, !direct))) return rc;
+    Ring* r = plan->ring;
+    const auto t0 = Clock::now();
+    const auto limit = std::chrono::milliseconds(d->timeout_ms ? d->timeout_ms : 60000);
+
+    struct Piece {
+        uint32_t buf;
+        bool last;
+        uint64_t pos, n;
+    };
+    std::vector<Piece> pieces;
+    for (uint32_t o = 0; o < d->n_bufs; ++o) {
+        uint32_t b = d->order[o];
+        for (uint64_t pos = 0; pos < d->bytes[b]; pos += g.chunk) {
+            uint64_t n = std::min(g.chunk, d->bytes[b] - pos);
+            pieces.push_back(Piece{b, pos + n == d->bytes[b], pos, n});
+        }
+    }
+    dr_stage_stats st{};
+    st.n_chunks = pieces.size();
+    st.chunks_done = std::min<uint64_t>(d->first_chunk, pieces.size());
+    st.pinned_high_water_bytes = direct ? 0 : g.chunk * g.slots;
+    if (d->wait_event) DR_CUDA(cudaStreamWaitEvent(r->s_copy, (cudaEvent_t)d->wait_event, 0));
+
+    auto issue = [&](uint64_t i) -> int {
+        const Piece& pc = pieces[i];
+        uint32_t s = (uint32_t)(i % g.slots);
+        uint64_t off = g.prefix[pc.buf] + pc.pos;
+        const char* host;
+        if (direct) {
+            host = (const char*)d->host_arena + off;
+        } else {
+            char* slot = r->base + (uint64_t)s * g.chunk;
+            if (d->callback) {
+                if (d->callback(d->user, i, off, slot, pc.n)) {
+                    set_error("chunk callback failed at piece %llu", (unsigned long long)i);
+                    return DR_ERR_SINK;
+                }
+            } else {
+                r->pool->copy(slot, (const char*)d->host_arena + off, pc.n);
+            }
+            host = slot;
+        }
+        DR_CUDA(cudaMemcpyAsync((char*)d->dev_ptr[pc.buf] + pc.pos, host, pc.n, cudaMemcpyHostToDevice, r->s_copy));
+        DR_CUDA(cudaEventRecord(r->ev_copy[s], r->s_copy));
+        if (pc.last && d->ready_events[pc.buf]) DR_CUDA(cudaEventRecord((cudaEvent_t)d->ready_events[pc.buf], r->s_copy));
+        return DR_OK;
+    };
+    auto complete = [&](uint64_t i) -> int {
+        int w = wait_event(r->ev_copy[i % g.slots], Clock::now() + limit);
+        if (w) return w;
+        st.bytes += pieces[i].n;
+        if (pieces[i].last) st.ready_ms[pieces[i].buf] = ms_since(t0);
+        return DR_OK;
+    };
+
+    uint64_t next_issue = st.chunks_done, next_done = st.chunks_done;
+    while (rc == DR_OK && next_done < pieces.size()) {
+        if (next_issue < pieces.size() && next_issue - next_done < g.slots) rc = issue(next_issue++);
+        else if ((rc = complete(next_done)) == DR_OK) st.chunks_done = ++next_done;
+    }
+    if (rc) drain(r, Clock::now() + limit);
+    st.elapsed_ms = ms_since(t0);
+    st.link_gbs = st.elapsed_ms > 0 ? (double)st.bytes / st.elapsed_ms * 1e-6 : 0;
+    if (stats) *stats = st;
+    return rc;
+}

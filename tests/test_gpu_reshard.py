@@ -1,0 +1,168 @@
+"""GPU parity: dr_reshard / dr_reshard_inverse through the C ABI against the CPU oracle, bit for bit,
+on seeded inputs that span many tiles, ragged tails, unaligned runs and every special value."""
+import numpy as np
+import pytest
+import torch
+
+import oracle
+import paper_2607_22614_b200 as dr
+import synth
+from gpu_util import SENT8, arena_dev, dev, first_diff, forward_both, make_source, special_values, to_dev_u32
+from synth.configs import BRUTE, CONFIGS, MID
+
+pytestmark = pytest.mark.gpu
+
+
+FWD = []
+for cfg in BRUTE:
+    for T in (1, 2):
+        for (W, g, A) in ((1, True, 1), (3, True, 4), (3, False, 1), (2, False, 16)):
+            for dt in (dr.DR_BF16, dr.DR_F32):
+                FWD.append((cfg, T, W, g, A, dt))
+for cfg in MID + [CONFIGS[0]]:
+    for (T, W, g, A, dt) in ((1, 1, True, 1, dr.DR_BF16), (2, 1, True, 1, dr.DR_BF16), (2, 3, False, 1, dr.DR_BF16),
+                            (4 if cfg["spec"]["n_kv_heads"] % 4 == 0 else 2, 2, False, 4, dr.DR_BF16),
+                            (2, 1, True, 1, dr.DR_F32), (1, 5, False, 3, dr.DR_F32)):
+        FWD.append((cfg, T, W, g, A, dt))
+
+
+@pytest.mark.parametrize("cfg,T,W,gathered,A,dtype", FWD,
+                         ids=[f"{c[0]['name']}-tp{c[1]}-w{c[2]}-g{int(c[3])}-a{c[4]}-d{c[5]}" for c in FWD])
+def test_forward_matches_oracle(cfg, T, W, gathered, A, dtype):
+    for t in range(T):
+        for r in ((W - 1,) if gathered else range(W)):
+            got, want, plan, _, _ = forward_both(cfg["spec"], world=W, rank=r, gathered=gathered, align=A, tp=T,
+                                                 tp_rank=t, dtype=dtype, seed=7 + t)
+            assert first_diff(got, want) is None  # includes sentinel bytes in gaps and uncovered elements
+            plan.close()
+
+
+@pytest.mark.parametrize("misalign", [16, 48])
+@pytest.mark.parametrize("dtype", [dr.DR_BF16, dr.DR_F32])
+def test_sixteen_byte_aligned_bases_take_the_narrow_path(misalign, dtype):
+    got, want, plan, _, _ = forward_both(MID[0]["spec"], tp=2, tp_rank=1, dtype=dtype, misalign=misalign)
+    assert first_diff(got, want) is None
+    plan.close()
+
+
+def test_cast_special_values_in_hardware():
+    """Every hand-picked pattern (ties, carries, overflow, subnormals, NaNs) through the vector path and,
+    via an odd-sized spec, through the scalar path."""
+    sp = special_values()
+    for cfg in (MID[2], BRUTE[0]):
+        om = oracle.Model(cfg["spec"])
+        src = np.resize(sp, om.flat_elems).astype(np.uint32)
+        got, want, plan, _, _ = forward_both(cfg["spec"], src=src)
+        assert first_diff(got, want) is None
+        plan.close()
+    # all 65536 high halves x tie / near-tie low halves, as one big "embedding"
+    spec = dict(MID[2]["spec"], vocab=4096 * 6 // 8, hidden=128, n_layers=0, n_q_heads=1, n_kv_heads=1, head_dim=8,
+                tied=1)
+    highs = np.arange(1 << 16, dtype=np.uint32) << 16
+    pats = np.concatenate([highs | np.uint32(lo) for lo in (0x0000, 0x0001, 0x7FFF, 0x8000, 0x8001, 0xFFFF)])
+    om = oracle.Model(spec)
+    assert om.flat_elems >= pats.size
+    src = np.resize(pats, om.flat_elems).astype(np.uint32)
+    got, want, plan, _, _ = forward_both(spec, src=src)
+    assert first_diff(got, want) is None
+    plan.close()
+
+
+def test_union_of_shards_fills_the_arena_like_a_gathered_call():
+    cfg = CONFIGS[0]  # tiny, world 2: rank 0 alone, then rank 1 into the same arena
+    spec, W = cfg["spec"], cfg["world"]
+    om = oracle.Model(spec, world=W)
+    src = make_source(W * om.shard_elems, 5)
+    full = np.full(om.arena_bytes, SENT8, dtype=np.uint8)
+    om.forward(src, full)
+    arena = arena_dev(om.arena_bytes)
+    for r in range(W):
+        plan = dr.Plan(spec, world=W, rank=r, gathered=False)
+        shard = to_dev_u32(src[r * om.shard_elems:(r + 1) * om.shard_elems].copy())
+        plan.reshard(shard, arena)
+        torch.cuda.synchronize()
+        if r == 0:
+            one = np.full(om.arena_bytes, SENT8, dtype=np.uint8)
+            om.forward(src[:om.shard_elems].copy(), one, gathered=False, rank=0)
+            assert first_diff(arena.cpu().numpy(), one) is None
+            assert plan.info.elems_moved == 987_904
+        plan.close()
+    assert first_diff(arena.cpu().numpy(), full) is None
+
+
+INV = [(BRUTE[0], 2, 3, False, 4, dr.DR_BF16), (BRUTE[2], 2, 1, True, 1, dr.DR_F32), (MID[0], 2, 1, True, 1, dr.DR_BF16),
+       (MID[1], 2, 3, False, 1, dr.DR_BF16), (MID[2], 1, 2, False, 16, dr.DR_F32), (MID[0], 4, 4, False, 1, dr.DR_BF16),
+       (CONFIGS[0], 1, 2, False, 1, dr.DR_BF16)]
+
+
+@pytest.mark.parametrize("cfg,T,W,gathered,A,dtype", INV,
+                         ids=[f"{c[0]['name']}-tp{c[1]}-w{c[2]}-g{int(c[3])}-a{c[4]}-d{c[5]}" for c in INV])
+def test_inverse_matches_oracle(cfg, T, W, gathered, A, dtype):
+    es = 2 if dtype == dr.DR_BF16 else 4
+    spec = cfg["spec"]
+    for t in range(T):
+        om = oracle.Model(spec, align=A, world=W, tp=T, tp_rank=t, elem_size=es)
+        arena = synth.fill_bf16(3, synth.BUF_ROLLOUT, 0, om.arena_bytes // 2).view(np.uint8)
+        if es == 2:  # sprinkle NaN, Inf and subnormal bf16 patterns: widening is a bit copy
+            h = arena.view(np.uint16)
+            h[::97] = np.resize(np.array([0x7FC0, 0xFF81, 0x7F80, 0x0001, 0x8000, 0x7FFF], dtype=np.uint16), h[::97].size)
+        for r in ((0,) if gathered else range(W)):
+            n = W * om.shard_elems if gathered else om.shard_elems
+            want = np.full(n, 0xDEADBEEF, dtype=np.uint32)
+            om.inverse(arena, want, gathered=gathered, rank=r)
+            plan = dr.Plan(spec, world=W, rank=r, gathered=gathered, align_elems=A, tp=T, tp_rank=t, dtype=dtype)
+            flat = torch.full((n,), 0xDEADBEEF - (1 << 32), dtype=torch.int32, device=dev())
+            a_dev = torch.from_numpy(arena).to(dev())
+            plan.reshard_inverse(a_dev, flat)
+            torch.cuda.synchronize()
+            assert first_diff(flat.cpu().numpy().view(np.uint32), want) is None
+            plan.close()
+
+
+def test_round_trip_on_layout_only_plan_is_identity():
+    spec = MID[0]["spec"]
+    T = 2
+    om = oracle.Model(spec, tp=T, elem_size=4)
+    src = make_source(om.flat_elems, 21)
+    s_dev = to_dev_u32(src)
+    back = torch.zeros_like(s_dev)
+    for t in range(T):
+        plan = dr.Plan(spec, tp=T, tp_rank=t, dtype=dr.DR_F32)
+        arena = arena_dev(plan.info.dst_bytes)
+        plan.reshard(s_dev, arena)
+        plan.reshard_inverse(arena, back)
+        torch.cuda.synchronize()
+        plan.close()
+    assert torch.equal(back, s_dev)
+
+
+def test_argument_errors_are_found_before_launch():
+    spec = MID[2]["spec"]
+    plan = dr.Plan(spec)
+    src = torch.zeros(plan.info.src_bytes // 4, dtype=torch.int32, device=dev())
+    arena = arena_dev(plan.info.dst_bytes)
+    B = dr.binding
+    s = torch.cuda.current_stream().cuda_stream
+    assert dr.dr_reshard(plan.handle, src.data_ptr(), plan.info.src_bytes - 4, arena.data_ptr(), plan.info.dst_bytes, s) == B.DR_ERR_SIZE
+    assert dr.dr_reshard(plan.handle, src.data_ptr(), plan.info.src_bytes, arena.data_ptr(), plan.info.dst_bytes - 1, s) == B.DR_ERR_SIZE
+    assert dr.dr_reshard(plan.handle, src.data_ptr() + 4, plan.info.src_bytes, arena.data_ptr(), plan.info.dst_bytes, s) == B.DR_ERR_ALIGN
+    assert dr.dr_reshard(plan.handle, None, plan.info.src_bytes, arena.data_ptr(), plan.info.dst_bytes, s) == B.DR_ERR_INVALID
+    assert dr.dr_reshard_inverse(plan.handle, arena.data_ptr(), 10, src.data_ptr(), plan.info.src_bytes, s) == B.DR_ERR_SIZE
+    assert "small" in dr.dr_last_error()
+    torch.cuda.synchronize()
+    assert (arena.cpu().numpy() == SENT8).all()  # nothing ran
+    plan.close()
+
+
+def test_device_generator_equals_host_generator():
+    n = 3_000_001
+    for buf in (synth.BUF_MASTER, synth.BUF_ADAM_M, synth.BUF_ADAM_V):
+        t = torch.empty(n, dtype=torch.int32, device=dev())
+        synth.cuda_fill_f32(t, 99, buf, start=12345)
+        assert np.array_equal(t.cpu().numpy().view(np.uint32), synth.fill_f32(99, buf, 12345, n))
+        assert synth.cuda_mismatch_f32(t, 99, buf, start=12345) == 0
+        t[77] += 1
+        assert synth.cuda_mismatch_f32(t, 99, buf, start=12345) == 1
+    h = torch.empty(n, dtype=torch.int16, device=dev())
+    synth.cuda_fill_bf16(h, 99, synth.BUF_ROLLOUT, start=5)
+    assert np.array_equal(h.cpu().numpy().view(np.uint16), synth.fill_bf16(99, synth.BUF_ROLLOUT, 5, n))

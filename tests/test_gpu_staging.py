@@ -1,0 +1,178 @@
+"""GPU parity for the chunked staging engine: byte-exact against the oracle's staging model on every
+sink (pageable arena, pinned arena, callback, relay), chunk geometry, resume after an injected
+failure, weights-first ordering, and overlap with the repack."""
+import ctypes as C
+
+import numpy as np
+import pytest
+import torch
+
+import oracle
+import paper_2607_22614_b200 as dr
+import synth
+from gpu_util import dev, to_dev_u32
+from synth.configs import CONFIGS, MID, MiB
+
+pytestmark = pytest.mark.gpu
+B = dr.binding
+
+
+def _state(n_elems, seed, bufs=(synth.BUF_ADAM_M, synth.BUF_ADAM_V)):
+    host = [synth.fill_f32(seed, b, 0, n_elems) for b in bufs]
+    return host, [to_dev_u32(h) for h in host]
+
+
+@pytest.fixture(scope="module")
+def plan():
+    p = dr.Plan(CONFIGS[0]["spec"], world=2, rank=0, gathered=False)
+    yield p
+    p.close()
+
+
+def test_tiny_workload_stage_out_and_in_pageable_arena(plan):
+    """Adam m and v of rank 0's shard, 1 MiB budget: 16 chunks of 512 KiB through a two-slot ring."""
+    S = plan.info.shard_elems
+    host, devs = _state(S, synth.SEED_BASE)
+    want_sink, want_sizes = oracle.stage_out([h.view(np.uint8) for h in host], 1 * MiB)
+    arena = np.zeros(want_sink.size + 64, dtype=np.uint8)
+    arena[-64:] = 0x5A
+    d = dr.stage_desc([t.data_ptr() for t in devs], [4 * S, 4 * S], budget=1 * MiB, host_arena=arena.ctypes.data,
+                      host_arena_bytes=want_sink.size)
+    st = plan.stage_out(d)
+    assert np.array_equal(arena[:-64], want_sink) and (arena[-64:] == 0x5A).all()
+    assert st.n_chunks == st.chunks_done == len(want_sizes) == 16
+    assert st.bytes == want_sink.size == 7_903_232
+    assert 0 < st.pinned_high_water_bytes <= 1 * MiB
+    # stage back in, v first this time
+    back = [torch.zeros_like(t) for t in devs]
+    d = dr.stage_desc([t.data_ptr() for t in back], [4 * S, 4 * S], budget=1 * MiB, order=[1, 0],
+                      host_arena=arena.ctypes.data, host_arena_bytes=want_sink.size)
+    st = plan.stage_in(d)
+    ob = [np.zeros(4 * S, dtype=np.uint8) for _ in host]
+    pieces, done = oracle.stage_in(ob, want_sink, 1 * MiB, order=[1, 0])
+    assert st.chunks_done == st.n_chunks == pieces and done == [1, 0]
+    for t, h, o in zip(back, host, ob):
+        assert np.array_equal(t.cpu().numpy().view(np.uint32), h) and np.array_equal(o.view(np.uint32), h)
+    assert 0 < st.ready_ms[1] <= st.ready_ms[0]  # buffer 1 was asked for first and is resident first
+
+
+def test_pinned_arena_is_copied_to_directly(plan):
+    S = 300_000
+    host, devs = _state(S, 3, bufs=(0, 1, 2))
+    total = 12 * S
+    pinned = torch.zeros(total, dtype=torch.uint8).pin_memory()
+    d = dr.stage_desc([t.data_ptr() for t in devs], [4 * S] * 3, budget=256 * 1024, chunk=64 * 1024,
+                      host_arena=pinned.data_ptr(), host_arena_bytes=total)
+    st = plan.stage_out(d)
+    assert st.pinned_high_water_bytes == 0 and st.n_chunks == -(-total // (64 * 1024))
+    assert np.array_equal(pinned.numpy(), np.concatenate([h.view(np.uint8) for h in host]))
+    back = [torch.zeros_like(t) for t in devs]
+    d = dr.stage_desc([t.data_ptr() for t in back], [4 * S] * 3, budget=256 * 1024, chunk=64 * 1024,
+                      host_arena=pinned.data_ptr(), host_arena_bytes=total)
+    plan.stage_in(d)
+    assert all(torch.equal(a, b) for a, b in zip(back, devs))
+
+
+def test_callback_sink_failure_and_resume(plan):
+    sizes = [100_000, 3, 250_001]  # odd sizes: chunks straddle buffers, ragged tail
+    rng = np.random.default_rng(0)
+    host = [rng.integers(0, 256, size=n, dtype=np.uint64).astype(np.uint8) for n in sizes]
+    devs = [torch.from_numpy(h).to(dev()) for h in host]
+    want, sizes_k = oracle.stage_out(host, 64 * 1024, 16 * 1024)
+    got = np.zeros_like(want)
+    calls = []
+    fail_at = [5]
+
+    @dr.dr_chunk_fn
+    def sink(user, k, off, ptr, n):
+        if k == fail_at[0]:
+            return 1
+        calls.append((k, off, n))
+        C.memmove(got.ctypes.data + off, ptr, n)
+        return 0
+
+    d = dr.stage_desc([t.data_ptr() for t in devs], sizes, budget=64 * 1024, chunk=16 * 1024, callback=sink)
+    rc, st = dr.dr_stage_out(plan.handle, d)
+    assert rc == B.DR_ERR_SINK and st.chunks_done == 5 and "callback" in dr.dr_last_error()
+    assert [c[0] for c in calls] == [0, 1, 2, 3, 4]
+    assert np.array_equal(got[:5 * 16 * 1024], want[:5 * 16 * 1024])
+    fail_at[0] = -1
+    d.first_chunk = st.chunks_done
+    rc, st2 = dr.dr_stage_out(plan.handle, d)
+    assert rc == 0 and st2.chunks_done == st2.n_chunks == len(sizes_k)
+    assert [c[0] for c in calls] == list(range(len(sizes_k)))
+    assert [c[2] for c in calls] == [int(x) for x in sizes_k]
+    assert np.array_equal(got, want)
+
+    # stage-in from a callback source
+    @dr.dr_chunk_fn
+    def source(user, k, off, ptr, n):
+        C.memmove(ptr, want.ctypes.data + off, n)
+        return 0
+
+    back = [torch.zeros_like(t) for t in devs]
+    d = dr.stage_desc([t.data_ptr() for t in back], sizes, budget=64 * 1024, chunk=16 * 1024, callback=source,
+                      order=[2, 0, 1])
+    plan.stage_in(d)
+    assert all(torch.equal(a, b) for a, b in zip(back, devs))
+
+
+def test_relay_sink_moves_state_to_other_device_buffers(plan):
+    S = 1_000_003
+    host, devs = _state(S, 11, bufs=(0, 1))
+    relay = [torch.zeros_like(t) for t in devs]
+    d = dr.stage_desc([t.data_ptr() for t in devs], [4 * S] * 2, budget=1 * MiB, chunk=128 * 1024,
+                      relay_dev=[t.data_ptr() for t in relay])
+    st = plan.stage_out(d)
+    assert st.bytes == 8 * S and st.pinned_high_water_bytes == 1 * MiB
+    assert all(torch.equal(a, b) for a, b in zip(relay, devs))
+
+
+def test_ready_events_and_overlap_with_the_repack():
+    """The repack kernel is enqueued first, then stage-out runs on the side stream while it executes;
+    both only read the master buffer.  Stage-in then records the caller's events per buffer."""
+    spec = MID[0]["spec"]
+    p = dr.Plan(spec)
+    N = p.info.flat_elems
+    master = torch.empty(N, dtype=torch.int32, device=dev())
+    synth.cuda_fill_f32(master, 5, synth.BUF_MASTER)
+    m = torch.empty(N, dtype=torch.int32, device=dev())
+    synth.cuda_fill_f32(m, 5, synth.BUF_ADAM_M)
+    arena = torch.zeros(p.info.dst_bytes, dtype=torch.uint8, device=dev())
+    produced = torch.cuda.Event()
+    produced.record()
+    host = np.zeros(8 * N, dtype=np.uint8)
+    p.reshard(master, arena)
+    d = dr.stage_desc([master.data_ptr(), m.data_ptr()], [4 * N] * 2, budget=8 * MiB, host_arena=host.ctypes.data,
+                      host_arena_bytes=host.size, wait_event=produced.cuda_event)
+    st = p.stage_out(d)
+    torch.cuda.synchronize()
+    assert np.array_equal(host.view(np.uint32)[:N], synth.fill_f32(5, synth.BUF_MASTER, 0, N))
+    assert np.array_equal(host.view(np.uint32)[N:], synth.fill_f32(5, synth.BUF_ADAM_M, 0, N))
+    om = oracle.Model(spec)
+    want = np.zeros(om.arena_bytes, dtype=np.uint8)
+    om.forward(host.view(np.uint32)[:N].copy(), want)
+    assert np.array_equal(arena.cpu().numpy(), want)
+    # stage-in: weights first, one event per buffer
+    back = [torch.zeros_like(master), torch.zeros_like(m)]
+    evs = [torch.cuda.Event(), torch.cuda.Event()]
+    for e in evs:
+        e.record()
+    d = dr.stage_desc([t.data_ptr() for t in back], [4 * N] * 2, budget=8 * MiB, host_arena=host.ctypes.data,
+                      host_arena_bytes=host.size, order=[0, 1], ready_events=[e.cuda_event for e in evs])
+    st = p.stage_in(d)
+    evs[0].synchronize()
+    evs[1].synchronize()
+    assert torch.equal(back[0], master) and torch.equal(back[1], m)
+    assert 0 < st.ready_ms[0] <= st.ready_ms[1]
+    p.close()
+
+
+def test_staging_argument_errors(plan):
+    t = torch.zeros(1024, dtype=torch.int32, device=dev())
+    host = np.zeros(4096, dtype=np.uint8)
+    mk = lambda **kw: dr.stage_desc([t.data_ptr()], [4096], **kw)
+    assert dr.dr_stage_out(plan.handle, mk(budget=4096, chunk=4096, host_arena=host.ctypes.data, host_arena_bytes=4096))[0] == B.DR_ERR_BUDGET
+    assert dr.dr_stage_out(plan.handle, mk(budget=8192, chunk=4096, host_arena=host.ctypes.data, host_arena_bytes=100))[0] == B.DR_ERR_SIZE
+    assert dr.dr_stage_out(plan.handle, mk(budget=8192, chunk=4096))[0] == B.DR_ERR_INVALID
+    assert dr.dr_stage_in(plan.handle, mk(budget=8192, chunk=4096, host_arena=host.ctypes.data, host_arena_bytes=4096, order=[3]))[0] == B.DR_ERR_INVALID

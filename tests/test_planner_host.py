@@ -1,0 +1,158 @@
+"""Host logic of the CUDA library, checked without a GPU: the planner's segment table expanded to a
+per-element map must be the oracle's map; sizes, tensor descriptors and error codes."""
+import ctypes as C
+import re
+import os
+
+import numpy as np
+import pytest
+
+import oracle
+import paper_2607_22614_b200 as dr
+from synth.configs import BRUTE, CONFIGS, MID
+
+ROOT = os.path.dirname(os.path.dirname(os.path.abspath(__file__)))
+
+
+def expand(plan, es):
+    """flat index (relative to the buffer the call receives) of every arena element slot the
+    segment table writes; -1 elsewhere.  Also checks that no slot is written twice."""
+    n_slots = plan.info.dst_bytes // es
+    m = np.full(n_slots, -1, dtype=np.int64)
+    moved = 0
+    for s in plan.segments():
+        assert s.dst_off % es == 0
+        rows = np.arange(s.rows, dtype=np.int64)[:, None]
+        cols = np.arange(s.row_len, dtype=np.int64)[None, :]
+        d = (s.dst_off // es + rows * s.dst_row_stride + cols).ravel()
+        f = (s.src_off + rows * s.src_row_stride + cols).ravel()
+        assert (m[d] == -1).all(), "two segments write the same arena element"
+        m[d] = f
+        moved += s.rows * s.row_len
+        if s.vector_bytes:
+            assert s.row_len % 8 == 0 and s.dst_off % (8 * es) == 0 and (s.src_off * 4) % s.vector_bytes == 0
+            if s.rows > 1:
+                assert (s.src_row_stride * 4) % s.vector_bytes == 0 and s.dst_row_stride % 8 == 0
+    assert moved == plan.info.elems_moved
+    return m
+
+
+def oracle_map(om, es, gathered, rank):
+    n_slots = om.arena_bytes // es
+    m = np.full(n_slots, -1, dtype=np.int64)
+    lo, hi = rank * om.shard_elems, (rank + 1) * om.shard_elems
+    for i, d in enumerate(om.dst_tensors()):
+        if d.alias_of >= 0:
+            continue
+        f = om.map_rows(i, 0, d.rows, d.cols).ravel()
+        if not gathered:
+            f = np.where((f >= lo) & (f < hi), f - lo, -1)
+        m[d.arena_off // es:d.arena_off // es + f.size] = f
+    return m
+
+
+CASES = []
+for cfg in BRUTE:
+    for T in (1, 2):
+        for (W, gathered, A) in ((1, True, 1), (3, True, 4), (3, False, 1), (2, False, 16), (5, False, 3)):
+            for dtype in (dr.DR_BF16, dr.DR_F32):
+                CASES.append((cfg["name"], cfg["spec"], T, W, gathered, A, dtype))
+for cfg in MID + [CONFIGS[0]]:
+    CASES.append((cfg["name"], cfg["spec"], 2, 1, True, 1, dr.DR_BF16))
+    CASES.append((cfg["name"], cfg["spec"], 2, 3, False, 1, dr.DR_BF16))
+    CASES.append((cfg["name"], cfg["spec"], 1, 2, False, 4, dr.DR_F32))
+
+
+@pytest.mark.parametrize("name,spec,T,W,gathered,A,dtype", CASES,
+                         ids=[f"{c[0]}-tp{c[2]}-w{c[3]}-g{int(c[4])}-a{c[5]}-d{c[6]}" for c in CASES])
+def test_segment_table_is_the_oracle_map(name, spec, T, W, gathered, A, dtype):
+    es = 2 if dtype == dr.DR_BF16 else 4
+    for t in range(T):
+        for r in (range(W) if not gathered else (0,)):
+            p = dr.Plan(spec, world=W, rank=r, gathered=gathered, align_elems=A, tp=T, tp_rank=t, dtype=dtype,
+                        arena_align_bytes=64, host_only=True)
+            om = oracle.Model(spec, align=A, world=W, tp=T, tp_rank=t, elem_size=es, arena_align=64)
+            assert p.info.flat_elems == om.flat_elems and p.info.shard_elems == om.shard_elems
+            assert p.info.dst_bytes == om.arena_bytes
+            assert p.info.src_bytes == 4 * (W * om.shard_elems if gathered else om.shard_elems)
+            assert p.info.bytes_moved_fwd == p.info.elems_moved * (4 + es) == p.info.bytes_moved_inv
+            assert np.array_equal(expand(p, es), oracle_map(om, es, gathered, r))
+            for a, b in zip(p.tensors(), om.dst_tensors()):
+                assert (a.name.decode(), a.arena_off, a.rows, a.cols, a.alias_of) == \
+                       (b.name, b.arena_off, b.rows, b.cols, b.alias_of)
+            p.close()
+
+
+def test_full_size_plans_match_quoted_sizes():
+    quoted_moved = {"tiny": 987_904, "qwen3-1.7b": 860_349_440, "qwen3-8b": 8_190_735_360,
+                    "qwen3-30b-a3b": 29_767_972_864}
+    for cfg in CONFIGS:
+        p = dr.Plan(cfg["spec"], world=cfg["world"], rank=cfg["rank"], gathered=cfg["gathered"], tp=cfg["tp"],
+                    tp_rank=cfg["tp_rank"], host_only=True)
+        om = oracle.Model(cfg["spec"], world=cfg["world"], tp=cfg["tp"], tp_rank=cfg["tp_rank"])
+        assert p.info.flat_elems == cfg["flat_elems"] and p.info.dst_bytes == om.arena_bytes
+        if cfg["name"] in quoted_moved:
+            assert p.info.elems_moved == quoted_moved[cfg["name"]]
+        segs = p.segments()
+        assert all(s.vector_bytes == 32 for s in segs)  # the benchmark shapes never need the scalar path
+        # sampled elements of sampled segments agree with the oracle's single-element map
+        rng = np.random.default_rng(1)
+        dst = om.dst_tensors()
+        lo = 0 if cfg["gathered"] else cfg["rank"] * om.shard_elems
+        starts = np.array([d.arena_off if d.alias_of < 0 else -1 for d in dst])
+        own = np.flatnonzero(starts >= 0)
+        for s in [segs[i] for i in rng.integers(0, len(segs), size=min(60, len(segs)))]:
+            for _ in range(20):
+                i, j = int(rng.integers(0, s.rows)), int(rng.integers(0, s.row_len))
+                byte = s.dst_off + (i * s.dst_row_stride + j) * 2
+                ti = int(own[np.searchsorted(starts[own], byte, side="right") - 1])  # merged runs span tensors
+                d = dst[ti]
+                slot = (byte - d.arena_off) // 2
+                assert slot < d.rows * d.cols
+                assert om.map(ti, slot // d.cols, slot % d.cols) == lo + s.src_off + i * s.src_row_stride + j
+        p.close()
+
+
+def test_library_exports_every_declared_symbol():
+    header = open(os.path.join(ROOT, "include", "dynaresize.h")).read()
+    declared = set(re.findall(r"\b(dr_[a-z_]+)\s*\(", header)) - {"dr_chunk_fn"}
+    assert declared == set(dr.EXPORTS)
+    L = C.CDLL(dr.lib_path)
+    for name in declared:
+        assert getattr(L, name) is not None
+
+
+def test_struct_sizes_match_the_header_layout():
+    assert C.sizeof(dr.dr_model_spec) == 48 and C.sizeof(dr.dr_src_layout) == 28 and C.sizeof(dr.dr_dst_layout) == 20
+    assert C.sizeof(dr.dr_plan_info) == 80 and C.sizeof(dr.dr_tensor_desc) == 96 and C.sizeof(dr.dr_segment_desc) == 56
+
+
+def test_error_codes():
+    spec = BRUTE[0]["spec"]
+    with pytest.raises(dr.DrError) as e:
+        dr.Plan(spec, tp=4, host_only=True)
+    assert e.value.status == dr.binding.DR_ERR_UNSUPPORTED
+    with pytest.raises(dr.DrError) as e:
+        dr.Plan(spec, tp=2, tp_rank=2, host_only=True)
+    assert e.value.status == dr.binding.DR_ERR_INVALID
+    with pytest.raises(dr.DrError) as e:
+        dr.Plan(spec, arena_align_bytes=24, host_only=True)
+    assert e.value.status == dr.binding.DR_ERR_INVALID
+    s = dr.model_spec(spec)
+    s.version = 99
+    rc, h = dr.dr_plan_create_host(s, dr.src_layout(), dr.dst_layout(), 1, 0)
+    assert rc == dr.binding.DR_ERR_INVALID and not h
+    rc, h = dr.dr_plan_create_host(dr.model_spec(spec), dr.src_layout(), dr.dst_layout(moe_tp=2), 1, 0)
+    assert rc == dr.binding.DR_ERR_UNSUPPORTED
+    # a host-only plan answers queries but refuses to launch or stage
+    p = dr.Plan(spec, host_only=True)
+    assert dr.dr_reshard(p.handle, 16, 1 << 30, 32, 1 << 30, None) == dr.binding.DR_ERR_STATE
+    d = dr.stage_desc([16], [4096], budget=1 << 20, host_arena=4096, host_arena_bytes=4096)
+    rc, _ = dr.dr_stage_out(p.handle, d)
+    assert rc == dr.binding.DR_ERR_STATE
+    d = dr.stage_desc([16], [4096], budget=4096, chunk=4096, host_arena=4096, host_arena_bytes=4096)
+    rc, _ = dr.dr_stage_out(p.handle, d)
+    assert rc == dr.binding.DR_ERR_BUDGET
+    assert dr.dr_plan_tensor(p.handle, 10_000)[0] == dr.binding.DR_ERR_INVALID
+    assert "budget" in dr.dr_strerror(dr.binding.DR_ERR_BUDGET)
+    assert dr.dr_plan_destroy(None) == 0
