@@ -1,0 +1,543 @@
+#!/usr/bin/env python
+"""Benchmark of the role-switch state transform on B200.
+
+One step = the device-resident transform of one whole model in both switch directions through the
+C ABI: ``dr_reshard`` (Training -> Rollout: un-flatten, fuse, TP-slice, cast to bf16) followed by
+``dr_reshard_inverse`` (Rollout -> Training).  ``value`` is the algorithmic bytes of those two calls
+over the device time of K steps.  The same run also measures, outside the K-step loop because they
+are bound by the host link and take seconds: chunked stage-out / stage-in of the fp32 master and Adam
+state, the switch latencies, the end-to-end number with host buffers, and the CPU oracle on a bounded
+sample.  Prints one JSON line on rank 0.
+
+    python bench.py [--gpus N] [--steps K] [--warmup W] [--cfg I] [--impl reference]
+"""
+from __future__ import annotations
+
+import argparse
+import json
+import os
+import subprocess
+import sys
+import tempfile
+import threading
+import time
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+if ROOT not in sys.path:
+    sys.path.insert(0, ROOT)
+
+METRIC = "role-switch transform GB/s (% of HBM peak); stage-out/in GB/s; switch ms"
+GiB = 1 << 30
+# DRAM bytes per element (dram__bytes_read.sum + dram__bytes_write.sum over elements moved) of the forward
+# kernel, from the ncu capture summarised in profiles/reshard_kernel_qwen3-8b.md (a 654 M-element case of the
+# same kernel; traffic grows in proportion to the elements, so it is scaled to the launch timed here).
+NCU_DRAM_BYTES_PER_ELEMENT_FWD = 5.948
+
+
+def load_peaks():
+    """Measured HBM copy bandwidth of this machine's B200s (generated file), else the stated fallback."""
+    path = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    try:
+        with open(path) as f:
+            return float(json.load(f)["hbm_gbs"]), "measured"
+    except Exception:
+        return 6650.0, "fallback"
+
+
+def mem_available_bytes() -> int:
+    with open("/proc/meminfo") as f:
+        for line in f:
+            if line.startswith("MemAvailable:"):
+                return int(line.split()[1]) * 1024
+    return 0
+
+
+class ClockSampler:
+    """Samples SM clocks and throttle reasons with nvidia-smi while a timed region runs."""
+
+    FIELDS = ("clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.hw_slowdown,"
+              "clocks_event_reasons.hw_thermal_slowdown,clocks_event_reasons.sw_thermal_slowdown,"
+              "clocks_event_reasons.sw_power_cap")
+
+    def __init__(self, index: int):
+        self.index = index
+        self.proc = None
+        self.path = None
+
+    def start(self):
+        fd, self.path = tempfile.mkstemp(suffix=".csv")
+        os.close(fd)
+        try:
+            self.proc = subprocess.Popen(
+                ["nvidia-smi", "-i", str(self.index), f"--query-gpu={self.FIELDS}", "--format=csv,noheader,nounits",
+                 "-lms", "100"], stdout=open(self.path, "w"), stderr=subprocess.DEVNULL)
+        except OSError:
+            self.proc = None
+
+    def stop(self) -> dict:
+        if self.proc is None:
+            return {"sm_mhz": None, "sm_max_mhz": None, "reasons": ["nvidia-smi unavailable"]}
+        time.sleep(0.15)
+        self.proc.terminate()
+        try:
+            self.proc.wait(timeout=5)
+        except subprocess.TimeoutExpired:
+            self.proc.kill()
+        sm, mx, reasons = [], [], set()
+        names = ["hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"]
+        with open(self.path) as f:
+            for line in f:
+                p = [x.strip() for x in line.split(",")]
+                if len(p) < 7:
+                    continue
+                try:
+                    sm.append(float(p[0]))
+                    mx.append(float(p[1]))
+                except ValueError:
+                    continue
+                for n, v in zip(names, p[3:7]):
+                    if v.lower().startswith("active"):
+                        reasons.add(n)
+        os.unlink(self.path)
+        sm.sort()
+        # the load is bursty: the median of the upper half is the clock while kernels ran
+        busy = sm[len(sm) // 2:] if sm else []
+        return {"sm_mhz": busy[len(busy) // 2] if busy else None, "sm_max_mhz": max(mx) if mx else None,
+                "samples": len(sm), "reasons": sorted(reasons)}
+
+
+def workload_name(cfg) -> str:
+    return (f"cfg{cfg['index']} {cfg['name']}: fp32 flat master -> bf16 rollout arena at TP={cfg['tp']} "
+            f"rank {cfg['tp_rank']}, and back")
+
+
+def median(xs):
+    s = sorted(xs)
+    return s[len(s) // 2]
+
+
+# ------------------------------------------------------------------------------------------------
+# CPU oracle legs (the only places this file touches oracle/)
+# ------------------------------------------------------------------------------------------------
+def oracle_sample(cfg, seconds: float, max_layers: int = 1 << 30):
+    """Times the oracle's forward transform, as it stands, on whole rollout tensors of the workload:
+    embed is skipped (4.7 GB of source), layers are taken in order until `seconds` have elapsed.
+    The source values come from the seeded generator (its time is not counted).  Returns
+    (GB/s on the same 6 B/element accounting, elements, seconds, description)."""
+    import numpy as np
+
+    import oracle
+    import synth
+
+    om = oracle.Model(cfg["spec"], world=cfg["world"], tp=cfg["tp"], tp_rank=cfg["tp_rank"])
+    srcs = {s.name: s for s in om.src_tensors()}
+    dst = om.dst_tensors()
+    # a lazily committed view of the whole flat buffer: only the sampled layers are ever touched
+    flat = np.empty(om.world * om.shard_elems, dtype=np.uint32)
+    arena = np.empty(om.arena_bytes, dtype=np.uint8)
+    seed = synth.SEED_BASE + cfg["index"]
+    elems, spent, layers = 0, 0.0, 0
+    for layer in range(min(max_layers, cfg["spec"]["n_layers"])):
+        names = [n for n in srcs if n.startswith(f"layers.{layer}.")]
+        lo = min(srcs[n].flat_off for n in names)
+        hi = max(srcs[n].flat_off + srcs[n].rows * srcs[n].cols for n in names)
+        flat[lo:hi] = synth.fill_f32(seed, synth.BUF_MASTER, lo, hi - lo)
+        for i, d in enumerate(dst):
+            if d.name.startswith(f"layers.{layer}.") and d.alias_of < 0:
+                t0 = time.perf_counter()
+                om.forward(flat, arena, gathered=True, only=i)
+                spent += time.perf_counter() - t0
+                elems += d.rows * d.cols
+        layers += 1
+        if spent >= seconds:
+            break
+    gbs = elems * 6 / spent / 1e9
+    return gbs, elems, spent, f"forward transform of rollout layers 0..{layers - 1} of {cfg['name']} ({elems} elements)"
+
+
+def run_reference(args, cfg):
+    """--impl reference: the oracle on this machine's host cores, each step a bounded sample."""
+    rank = int(os.environ.get("RANK", "0"))
+    if rank != 0:
+        return
+    per_step = max(1.0, min(10.0, 120.0 / max(1, args.steps + args.warmup)))
+    for _ in range(args.warmup):
+        oracle_sample(cfg, per_step, max_layers=1)
+    t_total, e_total, desc = 0.0, 0, ""
+    for _ in range(args.steps):
+        _, elems, spent, desc = oracle_sample(cfg, per_step, max_layers=1)
+        t_total += spent
+        e_total += elems
+    gbs = e_total * 6 / t_total / 1e9
+    line = {"impl": "reference", "metric": METRIC, "value": gbs, "unit": "GB/s", "n_gpus": args.gpus,
+            "steps": args.steps, "warmup": args.warmup, "ms_per_step": t_total / args.steps * 1e3,
+            "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "f32->bf16", "data": "synthetic",
+            "config": {"workload": workload_name(cfg), "step": "oracle forward transform of one layer's rollout tensors "
+                       "(bounded sample of the workload)"},
+            "cpu_baseline": {"value": gbs, "unit": "GB/s", "cores": 1, "kind": "oracle", "sample": desc},
+            "e2e": {"value": gbs, "unit": "GB/s", "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
+            "gpu_launches": 0}
+    print(json.dumps(line))
+
+
+# ------------------------------------------------------------------------------------------------
+# CUDA path
+# ------------------------------------------------------------------------------------------------
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=20)
+    ap.add_argument("--warmup", type=int, default=3)
+    ap.add_argument("--cfg", type=int, default=2, help="workload index 0..4 (default: Qwen3-8B-shaped, the paper's model)")
+    ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
+    ap.add_argument("--no-staging", action="store_true", help="skip the host-link sections")
+    ap.add_argument("--no-cpu", action="store_true", help="skip the CPU oracle baseline")
+    ap.add_argument("--cpu-seconds", type=float, default=12.0)
+    ap.add_argument("--layers", type=int, default=0, help="profiling aid: override the layer count (smaller case)")
+    ap.add_argument("--vocab", type=int, default=0, help="profiling aid: override the vocabulary size")
+    ap.add_argument("--profile", action="store_true", help="profiling aid: allow fewer than 3 warm-up steps")
+    args = ap.parse_args()
+    if args.impl == "ours" and not args.profile:
+        args.warmup = max(args.warmup, 3)
+
+    from synth.configs import CONFIGS
+    cfg = dict(CONFIGS[args.cfg], index=args.cfg)
+    if args.layers or args.vocab:
+        cfg["spec"] = dict(cfg["spec"], n_layers=args.layers or cfg["spec"]["n_layers"],
+                           vocab=args.vocab or cfg["spec"]["vocab"])
+        cfg["name"] += f" (reduced: {cfg['spec']['n_layers']} layers, vocab {cfg['spec']['vocab']})"
+    if args.impl == "reference":
+        run_reference(args, cfg)
+        return
+
+    import numpy as np
+    import torch
+
+    import paper_2607_22614_b200 as dr
+    import synth
+
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    rank = int(os.environ.get("RANK", "0"))
+    local = int(os.environ.get("LOCAL_RANK", "0"))
+    torch.cuda.set_device(local)
+    dev = torch.device("cuda", local)
+    if world > 1:
+        import torch.distributed as dist
+        dist.init_process_group("nccl", device_id=dev)
+
+    def barrier():
+        if world > 1:
+            dist.barrier()
+        torch.cuda.synchronize()
+
+    def max_over_ranks(x: float) -> float:
+        if world == 1:
+            return x
+        t = torch.tensor([x], dtype=torch.float64, device=dev)
+        dist.all_reduce(t, op=dist.ReduceOp.MAX)
+        return float(t.item())
+
+    peak, peak_kind = load_peaks()
+    seed = synth.SEED_BASE + args.cfg
+    inverse_dir = cfg["direction"] == "inv"
+
+    # cfg 4 does not fit beside its arena as one buffer: two shard-local halves, back to back
+    free_b, _ = torch.cuda.mem_get_info()
+    probe = dr.Plan(cfg["spec"], world=cfg["world"], rank=cfg["rank"], gathered=cfg["gathered"], tp=cfg["tp"],
+                    tp_rank=cfg["tp_rank"], host_only=True)
+    halves = 1
+    if probe.info.src_bytes * (1 if args.cfg == 4 else 2) + probe.info.dst_bytes > free_b * 0.92 and cfg["gathered"]:
+        halves = 2
+    probe.close()
+    if halves == 2:
+        plans = [dr.Plan(cfg["spec"], world=2, rank=r, gathered=False, tp=cfg["tp"], tp_rank=cfg["tp_rank"]) for r in (0, 1)]
+    else:
+        plans = [dr.Plan(cfg["spec"], world=cfg["world"], rank=cfg["rank"], gathered=cfg["gathered"], tp=cfg["tp"],
+                         tp_rank=cfg["tp_rank"])]
+    info = plans[0].info
+    n_src = info.src_bytes // 4
+    bytes_fwd = sum(p.info.bytes_moved_fwd for p in plans)
+    bytes_inv = sum(p.info.bytes_moved_inv for p in plans)
+
+    master = torch.empty(n_src, dtype=torch.int32, device=dev)
+    base = cfg["rank"] * info.shard_elems if not cfg["gathered"] else 0
+    synth.cuda_fill_f32(master, seed, synth.BUF_MASTER, start=base)
+    arena = torch.empty(info.dst_bytes, dtype=torch.uint8, device=dev)
+    if inverse_dir:
+        synth.cuda_fill_bf16(arena.view(torch.int16), seed, synth.BUF_ROLLOUT)
+    do_inverse = halves == 1 and free_b > (2 * info.src_bytes + info.dst_bytes) * 1.05
+    flat_back = torch.empty(n_src, dtype=torch.int32, device=dev) if do_inverse else None
+    torch.cuda.synchronize()
+
+    def step(events=None):
+        for hi, p in enumerate(plans):
+            if halves == 2:
+                synth.cuda_fill_f32(master, seed, synth.BUF_MASTER, start=hi * info.shard_elems)
+            if events is not None:
+                events.append(torch.cuda.Event(enable_timing=True))
+                events[-1].record()
+            p.reshard(master, arena)
+            if events is not None:
+                events.append(torch.cuda.Event(enable_timing=True))
+                events[-1].record()
+        if do_inverse:
+            plans[0].reshard_inverse(arena, flat_back)
+            if events is not None:
+                events.append(torch.cuda.Event(enable_timing=True))
+                events[-1].record()
+
+    for _ in range(args.warmup):
+        step()
+    barrier()
+    sampler = ClockSampler(local)
+    sampler.start()
+    evs = []
+    wall0 = torch.cuda.Event(enable_timing=True)
+    wall1 = torch.cuda.Event(enable_timing=True)
+    barrier()
+    wall0.record()
+    for _ in range(args.steps):
+        step(evs)
+    wall1.record()
+    barrier()
+    clocks = sampler.stop()
+    per = len(evs) // args.steps
+    fwd_ms, inv_ms = [], []
+    for s in range(args.steps):
+        e = evs[s * per:(s + 1) * per]
+        if halves == 2:
+            fwd_ms.append(e[0].elapsed_time(e[1]) + e[2].elapsed_time(e[3]))
+        else:
+            fwd_ms.append(e[0].elapsed_time(e[1]))
+            if do_inverse:
+                inv_ms.append(e[1].elapsed_time(e[2]))
+    if halves == 2:
+        total_ms = sum(fwd_ms)  # the generator refills between halves are not part of the transform
+    else:
+        total_ms = wall0.elapsed_time(wall1)
+    total_ms = max_over_ranks(total_ms)
+    step_bytes = bytes_fwd + (bytes_inv if do_inverse else 0)
+    value = world * step_bytes * args.steps / total_ms / 1e6
+    fwd_avg = sum(fwd_ms) / len(fwd_ms)
+    ach = bytes_fwd / fwd_avg / 1e6
+
+    line = {
+        "metric": METRIC, "value": value, "unit": "GB/s", "n_gpus": world, "steps": args.steps, "warmup": args.warmup,
+        "ms_per_step": total_ms / args.steps, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
+        "dtype": "f32->bf16", "data": "synthetic",
+        "config": {"workload": workload_name(cfg),
+                   "step": "dr_reshard + dr_reshard_inverse" if do_inverse else "dr_reshard",
+                   "elements": int(info.elems_moved if halves == 1 else sum(p.info.elems_moved for p in plans)),
+                   "bytes_per_step": int(step_bytes), "l2": "inputs larger than L2 (no flush needed)",
+                   "passes": halves, "parallelism": "replicas only" if world > 1 else "1 GPU",
+                   "segments": int(info.n_segments), "tiles": int(info.n_tiles)},
+        "clocks": clocks,
+        "gpu_launches": args.steps * (len(plans) + (1 if do_inverse else 0)),
+        "forward": {"gbs_avg": ach, "gbs_best": bytes_fwd / min(fwd_ms) / 1e6, "ms_avg": fwd_avg, "ms_best": min(fwd_ms),
+                    "ms_median": median(fwd_ms), "frac_of_measured_peak": ach / peak, "frac_of_nominal_8000": ach / 8000.0},
+        "roofline": {"bound": "hbm", "kernel": "reshard_kernel<2,false> (dr_reshard)", "achieved": ach, "peak": peak,
+                     "peak_kind": f"{peak_kind} copy bandwidth (burst)", "unit": "GB/s", "frac": ach / peak,
+                     "traffic": None, "algorithmic_bytes": int(bytes_fwd // len(plans))},
+    }
+    if inv_ms:
+        ia = sum(inv_ms) / len(inv_ms)
+        line["inverse"] = {"gbs_avg": bytes_inv / ia / 1e6, "gbs_best": bytes_inv / min(inv_ms) / 1e6, "ms_avg": ia,
+                           "ms_best": min(inv_ms), "frac_of_measured_peak": bytes_inv / ia / 1e6 / peak}
+    line["roofline"]["traffic"] = NCU_DRAM_BYTES_PER_ELEMENT_FWD * (bytes_fwd // 6 // len(plans)) if cfg["spec"] else None
+    line["roofline"]["traffic_source"] = "ncu capture of a 654 M-element case, scaled by elements (profiles/reshard_kernel_qwen3-8b.md)"
+
+    del flat_back
+    torch.cuda.empty_cache()
+
+    # ---- host-link sections ---------------------------------------------------------------------
+    if not args.no_staging:
+        line.update(staging_sections(args, cfg, plans[0], master, arena, seed, base, dev, world, line, max_over_ranks))
+
+    if rank == 0 and not args.no_cpu and world == 1:
+        gbs, elems, spent, desc = oracle_sample(cfg, args.cpu_seconds)
+        line["cpu_baseline"] = {"value": gbs, "unit": "GB/s", "cores": 1, "kind": "oracle", "sample": desc,
+                                "seconds": spent}
+    for p in plans:
+        p.close()
+    if world > 1:
+        dist.barrier()
+        dist.destroy_process_group()
+    if rank == 0:
+        print(json.dumps(line))
+
+
+def staging_sections(args, cfg, plan, master, arena, seed, base, dev, world, line, max_over_ranks):
+    """Chunked stage-out / stage-in of (master, Adam m, Adam v) to pinned host memory under the workload's
+    budget, the switch latencies, the measured host link, the same engine through its pinned ring into
+    pageable memory, and the end-to-end transform with host buffers."""
+    import numpy as np
+    import torch
+
+    import paper_2607_22614_b200 as dr
+    import synth
+
+    out = {}
+    info = plan.info
+    n = master.numel()
+    budget = cfg["budget"] or 2 * GiB
+    chunk = budget // 2
+
+    # measured pinned-copy bandwidth of the link, at 1 GiB and at this workload's chunk size
+    pin = torch.empty(max(chunk, GiB), dtype=torch.uint8, pin_memory=True)
+    scratch = torch.empty(max(chunk, GiB), dtype=torch.uint8, device=dev)
+
+    def link(nbytes, d2h):
+        best = 1e30
+        for _ in range(8):
+            a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            a.record()
+            if d2h:
+                pin[:nbytes].copy_(scratch[:nbytes], non_blocking=True)
+            else:
+                scratch[:nbytes].copy_(pin[:nbytes], non_blocking=True)
+            b.record()
+            torch.cuda.synchronize()
+            best = min(best, a.elapsed_time(b))
+        return nbytes / best / 1e6
+
+    link_d2h, link_h2d = link(GiB, True), link(GiB, False)
+    link_d2h_c, link_h2d_c = link(chunk, True), link(chunk, False)
+    del pin, scratch
+    torch.cuda.empty_cache()
+
+    # which state buffers fit: device memory for m and v, host memory for the image
+    names = list(cfg["stage"]) or ["master"]
+    free_b, _ = torch.cuda.mem_get_info()
+    host_room = int(mem_available_bytes() * 0.62 / world)
+    bufs, ids = [master], [synth.BUF_MASTER]
+    for nm, bid in (("m", synth.BUF_ADAM_M), ("v", synth.BUF_ADAM_V)):
+        if nm in names and free_b > 4 * n * 1.1 and (len(bufs) + 1) * 4 * n <= host_room:
+            t = torch.empty(n, dtype=torch.int32, device=dev)
+            synth.cuda_fill_f32(t, seed, bid, start=base)
+            bufs.append(t)
+            ids.append(bid)
+            free_b -= 4 * n
+    if "master" not in names and len(bufs) > 1:
+        bufs, ids = bufs[1:], ids[1:]
+    total = 4 * n * len(bufs)
+    if total > host_room:
+        return {"staging": {"skipped": f"host memory: need {total} bytes, room {host_room}"}}
+    sizes = [4 * n] * len(bufs)
+    torch.cuda.synchronize()
+
+    t0 = time.perf_counter()
+    image = torch.empty(total, dtype=torch.uint8, pin_memory=True)  # the pinned host resting place
+    pin_s = time.perf_counter() - t0
+
+    def desc(ptrs, host, **kw):
+        return dr.stage_desc(ptrs, sizes[:len(ptrs)], budget=budget, host_arena=host.data_ptr(),
+                             host_arena_bytes=host.numel(), **kw)
+
+    ptrs = [b.data_ptr() for b in bufs]
+    # T -> R switch: repack enqueued first, stage-out pumps while it runs
+    ev = [torch.cuda.Event(enable_timing=True) for _ in range(2)]
+    torch.cuda.synchronize()
+    t0 = time.perf_counter()
+    ev[0].record()
+    plan.reshard(master, arena)
+    ev[1].record()
+    st_out = plan.stage_out(desc(ptrs, image))
+    torch.cuda.synchronize()
+    t_switch = (time.perf_counter() - t0) * 1e3
+    repack_overlapped_ms = ev[0].elapsed_time(ev[1])
+    outs = [st_out.link_gbs] + [plan.stage_out(desc(ptrs, image)).link_gbs for _ in range(2)]
+    # spot-check the host image against the generator (a few windows per buffer)
+    img = image.numpy().view(np.uint32)
+    rng = np.random.default_rng(0)
+    image_ok = True
+    for k, bid in enumerate(ids):
+        for off in [0, n - 4096] + [int(x) for x in rng.integers(0, n - 4096, size=6)]:
+            image_ok &= bool(np.array_equal(img[k * n + off:k * n + off + 4096], synth.fill_f32(seed, bid, base + off, 4096)))
+
+    # R -> T switch: stage-in with the weights first; the inverse map can run as soon as they are resident
+    for b in bufs:
+        b.zero_()
+    torch.cuda.synchronize()
+    order = list(range(len(bufs)))
+    st_in = plan.stage_in(desc(ptrs, image, order=order))
+    torch.cuda.synchronize()
+    restored_ok = all(synth.cuda_mismatch_f32(b, seed, bid, start=base) == 0 for b, bid in zip(bufs, ids))
+    ins = [st_in.link_gbs] + [plan.stage_in(desc(ptrs, image, order=order)).link_gbs for _ in range(2)]
+
+    out["staging"] = {
+        "bytes": int(total), "buffers": [("master", "m", "v")[i] for i in ids], "budget_bytes": int(budget),
+        "chunk_bytes": int(chunk), "chunks": int(st_out.n_chunks), "sink": "pinned host image, chunked direct copies, "
+        "at most `budget` bytes in flight", "pin_seconds": pin_s,
+        "stage_out_gbs": max(outs), "stage_in_gbs": max(ins), "stage_out_gbs_runs": outs, "stage_in_gbs_runs": ins,
+        "link_d2h_gbs_1GiB": link_d2h, "link_h2d_gbs_1GiB": link_h2d, "link_d2h_gbs_chunk": link_d2h_c,
+        "link_h2d_gbs_chunk": link_h2d_c, "stage_out_frac_of_link": max(outs) / link_d2h,
+        "stage_in_frac_of_link": max(ins) / link_h2d, "host_image_matches_generator": image_ok,
+        "restored_state_matches_generator": bool(restored_ok),
+    }
+    out["switch_ms"] = {
+        "train_to_rollout": {"repack_alone": line["forward"]["ms_avg"], "repack_while_staging_out": repack_overlapped_ms,
+                             "until_state_staged_out": t_switch},
+        "rollout_to_train": {"weights_resident": st_in.ready_ms[0] if ids[0] == synth.BUF_MASTER else None,
+                             "inverse_map": line.get("inverse", {}).get("ms_avg"),
+                             "all_state_resident_deferred": st_in.elapsed_ms},
+    }
+
+    # the same engine with a pageable resting place: chunks go through the pinned ring and worker threads
+    if mem_available_bytes() > 4 * n * 1.5:
+        pageable = torch.empty(4 * n, dtype=torch.uint8)
+        pageable.fill_(0)  # commit the pages before timing
+        r_out = [plan.stage_out(desc(ptrs[:1], pageable)) for _ in range(2)]
+        ok = bool(np.array_equal(pageable.numpy().view(np.uint32)[:1 << 20], img[:1 << 20]))
+        bufs[0].zero_()
+        r_in = [plan.stage_in(desc(ptrs[:1], pageable, order=[0])) for _ in range(2)]
+        ok &= synth.cuda_mismatch_f32(bufs[0], seed, ids[0], start=base) == 0
+        out["staging"]["through_ring_to_pageable"] = {
+            "bytes": int(4 * n), "pinned_high_water_bytes": int(r_out[0].pinned_high_water_bytes),
+            "stage_out_gbs": max(x.link_gbs for x in r_out), "stage_in_gbs": max(x.link_gbs for x in r_in),
+            "stage_out_frac_of_link": max(x.link_gbs for x in r_out) / link_d2h,
+            "stage_in_frac_of_link": max(x.link_gbs for x in r_in) / link_h2d, "bytes_match": ok}
+        del pageable
+    for b in bufs[1:]:
+        del b
+    bufs = None
+    torch.cuda.empty_cache()
+
+    # ---- end to end with host buffers: H2D of the master, repack, D2H of the rollout arena, all through the C ABI
+    e2e_steps = 3
+    if image.numel() >= info.src_bytes + info.dst_bytes:
+        h_src, h_dst = image[:info.src_bytes], image[info.src_bytes:info.src_bytes + info.dst_bytes]
+    else:
+        del img, image
+        image = torch.empty(info.src_bytes + info.dst_bytes, dtype=torch.uint8, pin_memory=True)
+        h_src, h_dst = image[:info.src_bytes], image[info.src_bytes:]
+        plan.stage_out(dr.stage_desc([master.data_ptr()], [info.src_bytes], budget=budget, host_arena=h_src.data_ptr(),
+                                     host_arena_bytes=info.src_bytes))  # untimed: put the inputs on the host
+    if ids[0] != synth.BUF_MASTER:
+        plan.stage_out(dr.stage_desc([master.data_ptr()], [info.src_bytes], budget=budget, host_arena=h_src.data_ptr(),
+                                     host_arena_bytes=info.src_bytes))
+    master.zero_()
+    done = torch.cuda.Event()
+    done.record()
+    times = []
+    for i in range(e2e_steps + 1):
+        torch.cuda.synchronize()
+        t0 = time.perf_counter()
+        plan.stage_in(dr.stage_desc([master.data_ptr()], [info.src_bytes], budget=budget, host_arena=h_src.data_ptr(),
+                                    host_arena_bytes=info.src_bytes))
+        plan.reshard(master, arena)
+        done.record()
+        plan.stage_out(dr.stage_desc([arena.data_ptr()], [info.dst_bytes], budget=budget, host_arena=h_dst.data_ptr(),
+                                     host_arena_bytes=info.dst_bytes, wait_event=done.cuda_event))
+        torch.cuda.synchronize()
+        if i:
+            times.append(time.perf_counter() - t0)
+    t = max_over_ranks(sum(times) / len(times))
+    out["e2e"] = {"value": world * info.bytes_moved_fwd / t / 1e9, "unit": "GB/s", "ms_per_step": t * 1e3,
+                  "steps": e2e_steps, "h2d_bytes_per_step": int(info.src_bytes), "d2h_bytes_per_step": int(info.dst_bytes),
+                  "path": "dr_stage_in(pinned host master) -> dr_reshard -> dr_stage_out(rollout arena to pinned host)",
+                  "link_bound_ideal_ms": (info.src_bytes / link_h2d + info.dst_bytes / link_d2h) / 1e6}
+    return out
+
+
+if __name__ == "__main__":
+    main()

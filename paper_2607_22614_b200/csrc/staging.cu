@@ -171,7 +171,7 @@ int ensure_ring(dr_plan* p, const Geometry& g, bool need_memory)
         DR_CUDA(cudaStreamCreateWithFlags(&r->s_copy, cudaStreamNonBlocking));
         DR_CUDA(cudaStreamCreateWithFlags(&r->s_relay, cudaStreamNonBlocking));
         unsigned hw = std::thread::hardware_concurrency();
-        r->pool.reset(new CopyPool(std::max(1u, std::min(16u, hw / 2))));
+        r->pool.reset(new CopyPool(std::max(1u, std::min(16u, hw))));
     }
     Ring* r = p->ring;
     while (r->ev_copy.size() < g.slots) {
