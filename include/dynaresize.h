@@ -166,6 +166,30 @@ int dr_reshard(const dr_plan* plan, const void* src_dev, uint64_t src_bytes, voi
 int dr_reshard_inverse(const dr_plan* plan, const void* rollout_dev, uint64_t rollout_bytes, void* flat_dev,
                        uint64_t flat_bytes, void* cuda_stream);
 
+/*
+ * dr_reshard_static -- dr_reshard for callers that must not allocate device memory.  (The paper has
+ * no counterpart; this is a deployment aid.)
+ *
+ * Who needs it: a worker whose framework has already given the whole GPU to its own memory pool, so
+ * that a cudaMalloc at switch time would fail or take the head-room the incoming state needs; and a
+ * switch that overlaps staging copies with the repack, which a cudaMalloc or cudaFree would stall
+ * because both synchronise the device.  `plan` may come from dr_plan_create_host (no device memory at
+ * all) or from dr_plan_create.  The segment table, which dr_plan_create keeps in cudaMalloc'ed
+ * memory, is instead copied on `cuda_stream` into a fixed table inside the library (768 KiB, 16 384
+ * segments; every GPU that loads the library holds it until the process exits), and the same kernel
+ * runs from there.  The call itself allocates nothing, on host or device.
+ *
+ * Same arguments, result and errors as dr_reshard, plus DR_ERR_SIZE when the plan has more than
+ * 16 384 segments (dr_plan_query: n_segments).  The first call on each device looks up the table's
+ * device address; make that first call outside any stream capture.  All calls share the one table and
+ * it keeps the previous call's entries: each call rewrites the entries it uses, in stream order,
+ * before its kernel reads them, so calls on one stream are safe back to back, while calls that can
+ * overlap on the GPU (different streams, or different threads on different streams) race on the table
+ * and must be ordered by the caller.
+ */
+int dr_reshard_static(const dr_plan* plan, const void* src_dev, uint64_t src_bytes, void* dst_dev, uint64_t dst_bytes,
+                      void* cuda_stream);
+
 /* Chunk callback: stage-out hands chunk `chunk_idx` (bytes [stream_off, stream_off + n) of the
  * stream) in `pinned`; stage-in asks the callback to fill `pinned` with those bytes.  The pointer is
  * valid only during the call.  A non-zero return stops the transfer with DR_ERR_SINK. */

@@ -17,7 +17,7 @@ DR_F32, DR_BF16 = 1, 2
 DR_MAX_STAGE_BUFS = 8
 
 EXPORTS = ["dr_plan_create", "dr_plan_create_host", "dr_plan_query", "dr_plan_tensor", "dr_plan_segment",
-           "dr_reshard", "dr_reshard_inverse", "dr_stage_out", "dr_stage_in", "dr_plan_destroy", "dr_strerror",
+           "dr_reshard", "dr_reshard_inverse", "dr_reshard_static", "dr_stage_out", "dr_stage_in", "dr_plan_destroy", "dr_strerror",
            "dr_last_error"]
 
 u8, u32, u64, i64, vp = C.c_uint8, C.c_uint32, C.c_uint64, C.c_int64, C.c_void_p
@@ -92,6 +92,7 @@ def lib() -> C.CDLL:
         L.dr_plan_segment.argtypes = [vp, u64, P(dr_segment_desc)]
         L.dr_reshard.argtypes = [vp, vp, u64, vp, u64, vp]
         L.dr_reshard_inverse.argtypes = [vp, vp, u64, vp, u64, vp]
+        L.dr_reshard_static.argtypes = [vp, vp, u64, vp, u64, vp]
         L.dr_stage_out.argtypes = [vp, P(dr_stage_desc), P(dr_stage_stats)]
         L.dr_stage_in.argtypes = [vp, P(dr_stage_desc), P(dr_stage_stats)]
         L.dr_plan_destroy.argtypes = [vp]
@@ -180,6 +181,13 @@ def dr_reshard(plan, src_dev, src_bytes, dst_dev, dst_bytes, cuda_stream):
 
 def dr_reshard_inverse(plan, rollout_dev, rollout_bytes, flat_dev, flat_bytes, cuda_stream):
     return lib().dr_reshard_inverse(plan, rollout_dev, rollout_bytes, flat_dev, flat_bytes, cuda_stream)
+
+
+def dr_reshard_static(plan, src_dev, src_bytes, dst_dev, dst_bytes, cuda_stream):
+    """dr_reshard without any device allocation: the segment table goes into the library's fixed
+    768 KiB table (at most 16 384 segments).  For workers whose memory pool owns the whole GPU, or whose
+    switch must not be stalled by the device synchronisation that cudaMalloc / cudaFree imply."""
+    return lib().dr_reshard_static(plan, src_dev, src_bytes, dst_dev, dst_bytes, cuda_stream)
 
 
 def dr_stage_out(plan, desc):

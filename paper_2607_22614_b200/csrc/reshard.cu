@@ -299,3 +299,114 @@ int launch_reshard(const dr_plan* p, bool inverse, const void* flat, void* arena
 }
 
 }  // namespace dr
+
+// ------------------------------------------------------------------------------------------------
+// Allocation-free forward repack.
+//
+// The ordinary path keeps the segment table in memory that dr_plan_create obtains with cudaMalloc.
+// Some callers must not allocate on the device at the moment of a role switch: a worker whose
+// framework has handed the whole GPU to its own caching pool (a fresh cudaMalloc then fails or eats
+// the head-room the incoming state needs), and a switch that is overlapping staging copies with the
+// repack (cudaMalloc and cudaFree synchronise the device and would stall those copies).  For them the
+// table lives in the fixed array below, which every GPU that loads this library holds until exit.
+// ------------------------------------------------------------------------------------------------
+namespace dr {
+namespace {
+
+constexpr uint32_t kStaticMaxSegs = 16384;  // 768 KiB; the largest benchmark plan (30B-A3B MoE) needs 12 482
+static __device__ __align__(256) unsigned char g_static_segs[kStaticMaxSegs * sizeof(DevSeg)];
+
+constexpr int kMaxDevices = 64;
+struct StaticSlot {
+    DevSeg* table = nullptr;  // device address of g_static_segs on that device
+    int grid[2] = {0, 0};     // persistent grid for bf16 / fp32 rollout plans
+};
+StaticSlot g_slots[kMaxDevices];
+std::mutex g_slots_mu;
+
+// Once per device, with that device current: the array's name is only a host-side handle, the address
+// the kernel needs comes from the runtime.
+int static_setup(int device, StaticSlot* out)
+{
+    std::lock_guard<std::mutex> lock(g_slots_mu);
+    StaticSlot& s = g_slots[device];
+    if (!s.table) {
+        void* ptr = nullptr;
+        cudaError_t e = cudaGetSymbolAddress(&ptr, g_static_segs);
+        if (e != cudaSuccess || !ptr) {
+            set_error("cudaGetSymbolAddress(static segment table): %s", cudaGetErrorString(e));
+            return DR_ERR_CUDA;
+        }
+        int g2 = choose_grid(device, 2), g4 = choose_grid(device, 4);
+        if (g2 <= 0 || g4 <= 0) {
+            set_error("occupancy query failed");
+            return DR_ERR_CUDA;
+        }
+        s.grid[0] = g2;
+        s.grid[1] = g4;
+        s.table = (DevSeg*)ptr;
+    }
+    *out = s;
+    return DR_OK;
+}
+
+}  // namespace
+}  // namespace dr
+
+extern "C" int dr_reshard_static(const dr_plan* plan, const void* src_dev, uint64_t src_bytes, void* dst_dev,
+                                 uint64_t dst_bytes, void* cuda_stream)
+{
+    using namespace dr;
+    if (!plan || !src_dev || !dst_dev) {
+        set_error("NULL plan or buffer");
+        return DR_ERR_INVALID;
+    }
+    const uint64_t n_segs = plan->dev_segs.size();
+    if (n_segs > kStaticMaxSegs) {
+        set_error("plan has %llu segments; the static table holds at most %u (use dr_plan_create + dr_reshard)",
+                  (unsigned long long)n_segs, kStaticMaxSegs);
+        return DR_ERR_SIZE;
+    }
+    if (src_bytes < plan->info.src_bytes || dst_bytes < plan->info.dst_bytes) {
+        set_error("buffer too small: have %llu / %llu bytes, need %llu / %llu", (unsigned long long)src_bytes,
+                  (unsigned long long)dst_bytes, (unsigned long long)plan->info.src_bytes,
+                  (unsigned long long)plan->info.dst_bytes);
+        return DR_ERR_SIZE;
+    }
+    if (((uintptr_t)src_dev | (uintptr_t)dst_dev) & 15) {
+        set_error("base pointers must be 16-byte aligned");
+        return DR_ERR_ALIGN;
+    }
+    int device = -1;
+    if (cudaGetDevice(&device) != cudaSuccess || device < 0 || device >= kMaxDevices) {
+        set_error("no current CUDA device");
+        return DR_ERR_CUDA;
+    }
+    StaticSlot slot;
+    int rc = static_setup(device, &slot);
+    if (rc) return rc;
+    const uint64_t n_tiles = plan->info.n_tiles;
+    if (n_tiles == 0) return DR_OK;
+    cudaStream_t s = (cudaStream_t)cuda_stream;
+    // The table is rewritten for every call, in stream order before the kernel that reads it.
+    cudaError_t e = cudaMemcpyAsync(slot.table, plan->dev_segs.data(), n_segs * sizeof(DevSeg), cudaMemcpyHostToDevice, s);
+    if (e != cudaSuccess) {
+        set_error("static table upload: %s", cudaGetErrorString(e));
+        return DR_ERR_CUDA;
+    }
+    char* f = (char*)src_dev;
+    char* a = (char*)dst_dev;
+    const int allow256 = (((uintptr_t)f | (uintptr_t)a) & 31) == 0;
+    const int g = slot.grid[plan->elem_size == 2 ? 0 : 1];
+    dim3 grid((unsigned)(n_tiles < (uint64_t)g ? n_tiles : (uint64_t)g)), block(kThreads);
+    if (plan->elem_size == 2)
+        reshard_kernel<2, false, false><<<grid, block, 0, s>>>(slot.table, (uint32_t)n_segs, n_tiles, f, a, allow256);
+    else
+        reshard_kernel<4, false, false><<<grid, block, 0, s>>>(slot.table, (uint32_t)n_segs, n_tiles, f, a, allow256);
+    e = cudaGetLastError();
+    if (e != cudaSuccess) {
+        set_error("reshard kernel launch: %s", cudaGetErrorString(e));
+        return DR_ERR_CUDA;
+    }
+    return DR_OK;
+}
