@@ -175,7 +175,7 @@ int dr_reshard_inverse(const dr_plan* plan, const void* rollout_dev, uint64_t ro
  * switch that overlaps staging copies with the repack, which a cudaMalloc or cudaFree would stall
  * because both synchronise the device.  `plan` may come from dr_plan_create_host (no device memory at
  * all) or from dr_plan_create.  The segment table, which dr_plan_create keeps in cudaMalloc'ed
- * memory, is instead copied on `cuda_stream` into a fixed table inside the library (768 KiB, 16 384
+ * memory, is instead copied on `cuda_stream` into a fixed table inside the library (1 MiB, 16 384
  * segments; every GPU that loads the library holds it until the process exits), and the same kernel
  * runs from there.  The call itself allocates nothing, on host or device.
  *

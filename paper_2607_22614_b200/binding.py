@@ -185,7 +185,7 @@ def dr_reshard_inverse(plan, rollout_dev, rollout_bytes, flat_dev, flat_bytes, c
 
 def dr_reshard_static(plan, src_dev, src_bytes, dst_dev, dst_bytes, cuda_stream):
     """dr_reshard without any device allocation: the segment table goes into the library's fixed
-    768 KiB table (at most 16 384 segments).  For workers whose memory pool owns the whole GPU, or whose
+    1 MiB table (at most 16 384 segments).  For workers whose memory pool owns the whole GPU, or whose
     switch must not be stalled by the device synchronisation that cudaMalloc / cudaFree imply."""
     return lib().dr_reshard_static(plan, src_dev, src_bytes, dst_dev, dst_bytes, cuda_stream)
 

@@ -91,6 +91,9 @@ int create(const dr_model_spec* s, const dr_src_layout* a, const dr_dst_layout* 
         size_t bytes = p->dev_segs.size() * sizeof(DevSeg);
         if (e == cudaSuccess && bytes) e = cudaMalloc((void**)&p->d_segs, bytes);
         if (e == cudaSuccess && bytes) e = cudaMemcpy(p->d_segs, p->dev_segs.data(), bytes, cudaMemcpyHostToDevice);
+        size_t hbytes = p->hints.size() * sizeof(uint32_t);
+        if (e == cudaSuccess) e = cudaMalloc((void**)&p->d_hints, hbytes);
+        if (e == cudaSuccess) e = cudaMemcpy(p->d_hints, p->hints.data(), hbytes, cudaMemcpyHostToDevice);
         if (e == cudaSuccess) p->grid = choose_grid(p->device, p->elem_size);
         if (e != cudaSuccess || p->grid <= 0) {
             set_error("plan upload: %s", cudaGetErrorString(e));
@@ -219,6 +222,7 @@ int dr_plan_destroy(dr_plan* plan)
     if (!plan) return DR_OK;
     if (plan->ring) ring_destroy(plan->ring);
     if (plan->d_segs) cudaFree(plan->d_segs);
+    if (plan->d_hints) cudaFree(plan->d_hints);
     delete plan;
     return DR_OK;
 }

@@ -13,10 +13,15 @@ namespace dr {
 
 // A work unit is 8 consecutive elements of one row (32 B of fp32, 16 B of bf16); a tile is
 // kTileUnits consecutive units of one segment.  One CTA iteration processes one tile.
+#ifndef DR_TILE_UNITS
+#define DR_TILE_UNITS 512
+#endif
 constexpr uint32_t kUnitElems = 8;
-constexpr uint32_t kTileUnits = 1024;
+constexpr uint32_t kTileUnits = DR_TILE_UNITS;
 // Contiguous runs are cut so that a segment's unit count fits 32 bits with room to spare.
 constexpr uint64_t kMaxSegElems = 1ull << 31;
+// The tile -> segment hint table has at most this many entries (256 KiB).
+constexpr uint64_t kMaxHints = 65536;
 
 enum SegFlags : uint32_t {
     kSegVec32 = 1u,      // flat-side addresses 32-byte aligned: 256-bit accesses allowed
@@ -63,10 +68,14 @@ struct dr_plan {
     std::vector<dr::Tensor> tensors;
     std::vector<dr::HostSeg> segs;
     std::vector<dr::DevSeg> dev_segs;  // host copy of the device table
+    // hints[i] = segment holding tile i << hint_shift: a tile finds its segment with one load plus a short walk
+    std::vector<uint32_t> hints;
+    uint32_t hint_shift = 0;
     // device side (absent on a host-only plan)
     bool host_only = true;
     int device = -1;
     dr::DevSeg* d_segs = nullptr;
+    uint32_t* d_hints = nullptr;
     int grid = 0;
     // staging
     std::mutex stage_mu;

@@ -308,6 +308,20 @@ int compile_plan(dr_plan* p)
         moved += g.rows * g.row_len;
     }
 
+    // hint table: segment of every (1 << hint_shift)-th tile
+    p->hint_shift = 0;
+    while (((tiles + (1ull << p->hint_shift) - 1) >> p->hint_shift) > kMaxHints) ++p->hint_shift;
+    {
+        const uint64_t n_hints = (tiles + (1ull << p->hint_shift) - 1) >> p->hint_shift;
+        p->hints.resize(n_hints ? n_hints : 1, 0);
+        uint32_t si = 0;
+        for (uint64_t h = 0; h < n_hints; ++h) {
+            const uint64_t tile = h << p->hint_shift;
+            while (si + 1 < p->dev_segs.size() && p->dev_segs[si + 1].tile0 <= tile) ++si;
+            p->hints[h] = si;
+        }
+    }
+
     dr_plan_info& I = p->info;
     I.flat_elems = N;
     I.shard_elems = S;

@@ -1,0 +1,171 @@
+"""GPU parity at the full sizes of the five workloads, in the launch configuration bench.py times.
+
+cfg 1 is compared whole against the oracle (the oracle finishes it in seconds).  cfg 2-4 are too big
+for that: they are checked on sampled outputs that the oracle computes one by one, on whole small
+tensors, on row blocks at the edges of the big tensors, and by counting what the call touched."""
+import numpy as np
+import pytest
+import torch
+
+import oracle
+import paper_2607_22614_b200 as dr
+import synth
+from synth.configs import CONFIGS, seed_of
+
+pytestmark = pytest.mark.gpu
+DEV = "cuda:0"
+
+
+def _need(gb):
+    import gc
+    gc.collect()
+    torch.cuda.empty_cache()  # memory cached by earlier tests counts as free
+    free, _ = torch.cuda.mem_get_info()
+    if free < gb * 1e9:
+        pytest.skip(f"needs {gb} GB of free device memory, {free / 1e9:.0f} GB free")
+
+
+def _models(cfg, world=None, rank=None, gathered=None):
+    world = cfg["world"] if world is None else world
+    rank = cfg["rank"] if rank is None else rank
+    gathered = cfg["gathered"] if gathered is None else gathered
+    plan = dr.Plan(cfg["spec"], world=world, rank=rank, gathered=gathered, tp=cfg["tp"], tp_rank=cfg["tp_rank"])
+    om = oracle.Model(cfg["spec"], world=world, tp=cfg["tp"], tp_rank=cfg["tp_rank"])
+    assert plan.info.dst_bytes == om.arena_bytes and plan.info.flat_elems == cfg["flat_elems"]
+    return plan, om
+
+
+def _sample_positions(om, n, rng):
+    """Random (tensor, row, col) weighted by tensor size, plus every element of the small tensors of three
+    layers and 2-row blocks at the top and bottom of every big tensor of the first and last layer."""
+    dst = [(i, d) for i, d in enumerate(om.dst_tensors()) if d.alias_of < 0]
+    sizes = np.array([d.rows * d.cols for _, d in dst], dtype=np.float64)
+    pick = rng.choice(len(dst), size=n, p=sizes / sizes.sum())
+    ti = np.array([dst[k][0] for k in pick])
+    rows = np.array([rng.integers(0, dst[k][1].rows) for k in pick])
+    cols = np.array([rng.integers(0, dst[k][1].cols) for k in pick])
+    extra = []
+    L = max(1, sum(1 for _, d in dst if d.name.endswith(".in_norm")))
+    for i, d in dst:
+        layer = int(d.name.split(".")[1]) if d.name.startswith("layers.") else -1
+        if d.rows * d.cols <= 8192 and layer in (-1, 0, L // 2, L - 1):
+            r, c = np.divmod(np.arange(d.rows * d.cols), d.cols)
+            extra.append((np.full(r.size, i), r, c))
+        elif layer in (-1, 0, L - 1):
+            for r0 in (0, d.rows - 2):
+                r = np.repeat(np.arange(r0, r0 + 2), d.cols)
+                c = np.tile(np.arange(d.cols), 2)
+                extra.append((np.full(r.size, i), r, c))
+    ti = np.concatenate([ti] + [e[0] for e in extra])
+    rows = np.concatenate([rows] + [e[1] for e in extra])
+    cols = np.concatenate([cols] + [e[2] for e in extra])
+    return ti, rows, cols
+
+
+def _oracle_flat_index(om, ti, rows, cols):
+    return np.array([om.map(int(i), int(r), int(c)) for i, r, c in zip(ti, rows, cols)], dtype=np.int64)
+
+
+def _arena_slots(om, ti, rows, cols):
+    dst = om.dst_tensors()
+    off = np.array([dst[i].arena_off for i in ti], dtype=np.int64) // 2
+    ncol = np.array([dst[i].cols for i in ti], dtype=np.int64)
+    return off + rows * ncol + cols
+
+
+def test_cfg1_whole_arena_equals_oracle():
+    """Qwen3-1.7B-shaped, gathered flat buffer, TP=2 rank 0: every byte of the 1.72 GB arena."""
+    _need(12)
+    cfg = CONFIGS[1]
+    plan, om = _models(cfg)
+    seed = seed_of(1)
+    src = torch.empty(plan.info.src_bytes // 4, dtype=torch.int32, device=DEV)
+    synth.cuda_fill_f32(src, seed, synth.BUF_MASTER)
+    arena = torch.full((plan.info.dst_bytes,), 0xA5, dtype=torch.uint8, device=DEV)
+    plan.reshard(src, arena)
+    torch.cuda.synchronize()
+    got = arena.cpu().numpy()
+    del src, arena
+    flat = synth.fill_f32(seed, synth.BUF_MASTER, 0, om.world * om.shard_elems)
+    want = np.full(om.arena_bytes, 0xA5, dtype=np.uint8)
+    om.forward(flat, want)
+    assert np.array_equal(got, want)
+    assert plan.info.elems_moved == 860_349_440
+    plan.close()
+
+
+def test_cfg2_sampled_outputs():
+    """Qwen3-8B-shaped, TP=1: 8.19 G elements, 49 GB moved per launch."""
+    _need(55)
+    cfg = CONFIGS[2]
+    plan, om = _models(cfg)
+    seed = seed_of(2)
+    src = torch.empty(plan.info.src_bytes // 4, dtype=torch.int32, device=DEV)
+    synth.cuda_fill_f32(src, seed, synth.BUF_MASTER)
+    arena = torch.full((plan.info.dst_bytes,), 0xA5, dtype=torch.uint8, device=DEV)
+    plan.reshard(src, arena)
+    torch.cuda.synchronize()
+    rng = np.random.default_rng(2)
+    ti, rows, cols = _sample_positions(om, 200_000, rng)
+    f = _oracle_flat_index(om, ti, rows, cols)
+    want = oracle.cast_bf16_array(synth.at_f32(seed, synth.BUF_MASTER, f))
+    slots = torch.from_numpy(_arena_slots(om, ti, rows, cols)).to(DEV)
+    got = arena.view(torch.int16)[slots].cpu().numpy().view(np.uint16)
+    assert np.array_equal(got, want)
+    # at TP=1 every arena byte is written: the sentinel pattern (not a value the generator can produce) is gone
+    assert int((arena.view(torch.int16) == (0xA5A5 - 65536)).sum()) == 0
+    plan.close()
+
+
+def test_cfg3_inverse_shard_local_sampled_and_counted():
+    """Qwen3-14B-shaped, Rollout -> Training: TP=4 rank 1 arena scattered into FSDP shard 1 of 4."""
+    _need(26)
+    cfg = CONFIGS[3]
+    plan, om = _models(cfg)
+    seed = seed_of(3)
+    S, r = plan.info.shard_elems, cfg["rank"]
+    arena = torch.empty(plan.info.dst_bytes // 2, dtype=torch.int16, device=DEV)
+    synth.cuda_fill_bf16(arena, seed, synth.BUF_ROLLOUT)
+    sent = 0xDEADBEEF - (1 << 32)
+    flat = torch.full((S,), sent, dtype=torch.int32, device=DEV)
+    plan.reshard_inverse(arena, flat)
+    torch.cuda.synchronize()
+    # every word the call wrote is a widened bf16 (low half zero), so counting non-sentinel words counts writes
+    assert int((flat != sent).sum()) == plan.info.elems_moved
+    rng = np.random.default_rng(3)
+    ti, rows, cols = _sample_positions(om, 300_000, rng)
+    f = _oracle_flat_index(om, ti, rows, cols)
+    inside = (f >= r * S) & (f < (r + 1) * S)
+    assert 0.15 < inside.mean() < 0.5
+    slots = _arena_slots(om, ti, rows, cols)
+    want = synth.at_bf16(seed, synth.BUF_ROLLOUT, slots[inside]).astype(np.uint32) << 16
+    got = flat[torch.from_numpy(f[inside] - r * S).to(DEV)].cpu().numpy().view(np.uint32)
+    assert np.array_equal(got, want)
+    plan.close()
+
+
+def test_cfg4_moe_two_half_shards_sampled():
+    """Qwen3-30B-A3B-shaped MoE: run as two shard-local halves into one arena (it does not fit whole)."""
+    _need(125)
+    cfg = CONFIGS[4]
+    seed = seed_of(4)
+    om = oracle.Model(cfg["spec"], world=2, tp=cfg["tp"], tp_rank=cfg["tp_rank"])
+    S = om.shard_elems
+    arena = torch.full((om.arena_bytes,), 0xA5, dtype=torch.uint8, device=DEV)
+    shard = torch.empty(S, dtype=torch.int32, device=DEV)
+    moved = 0
+    for half in (0, 1):
+        plan, _ = _models(cfg, world=2, rank=half, gathered=False)
+        synth.cuda_fill_f32(shard, seed, synth.BUF_MASTER, start=half * S)
+        plan.reshard(shard, arena)
+        torch.cuda.synchronize()
+        moved += plan.info.elems_moved
+        plan.close()
+    assert moved == 29_767_972_864
+    rng = np.random.default_rng(4)
+    ti, rows, cols = _sample_positions(om, 200_000, rng)
+    f = _oracle_flat_index(om, ti, rows, cols)
+    want = oracle.cast_bf16_array(synth.at_f32(seed, synth.BUF_MASTER, f))
+    slots = torch.from_numpy(_arena_slots(om, ti, rows, cols)).to(DEV)
+    got = arena.view(torch.int16)[slots].cpu().numpy().view(np.uint16)
+    assert np.array_equal(got, want)
