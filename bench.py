@@ -106,6 +106,51 @@ class ClockSampler:
                 "samples": len(sm), "reasons": sorted(reasons)}
 
 
+class Dist:
+    """One process per GPU under torchrun (RANK / LOCAL_RANK / WORLD_SIZE / MASTER_* from the environment).
+    The path has no exchange step, so the process group only carries the barrier and the max-over-ranks of
+    the timings; `backend="gloo"` runs the same plumbing on CPU for the tests."""
+
+    def __init__(self, backend: str = "nccl", device=None):
+        self.world = int(os.environ.get("WORLD_SIZE", "1"))
+        self.rank = int(os.environ.get("RANK", "0"))
+        self.local = int(os.environ.get("LOCAL_RANK", "0"))
+        self.device = device
+        self.backend = backend
+        if self.world > 1:
+            import torch.distributed as dist
+            kw = {"device_id": device} if backend == "nccl" and device is not None else {}
+            dist.init_process_group(backend, **kw)
+
+    def barrier(self):
+        import torch
+        if self.world > 1:
+            import torch.distributed as dist
+            dist.barrier()
+        if self.backend == "nccl":
+            torch.cuda.synchronize()
+
+    def max(self, x: float) -> float:
+        if self.world == 1:
+            return x
+        import torch
+        import torch.distributed as dist
+        t = torch.tensor([x], dtype=torch.float64, device=self.device if self.backend == "nccl" else "cpu")
+        dist.all_reduce(t, op=dist.ReduceOp.MAX)
+        return float(t.item())
+
+    def close(self):
+        if self.world > 1:
+            import torch.distributed as dist
+            dist.barrier()
+            dist.destroy_process_group()
+
+
+def whole_job_gbs(world: int, bytes_per_rank_step: int, steps: int, max_ms_over_ranks: float) -> float:
+    """Replicas only: every rank moves the same bytes; the job's rate is all ranks' bytes over the slowest rank's time."""
+    return world * bytes_per_rank_step * steps / max_ms_over_ranks / 1e6
+
+
 def workload_name(cfg) -> str:
     return (f"cfg{cfg['index']} {cfg['name']}: fp32 flat master -> bf16 rollout arena at TP={cfg['tp']} "
             f"rank {cfg['tp_rank']}, and back")
@@ -216,26 +261,12 @@ def main():
     import paper_2607_22614_b200 as dr
     import synth
 
-    world = int(os.environ.get("WORLD_SIZE", "1"))
-    rank = int(os.environ.get("RANK", "0"))
     local = int(os.environ.get("LOCAL_RANK", "0"))
     torch.cuda.set_device(local)
     dev = torch.device("cuda", local)
-    if world > 1:
-        import torch.distributed as dist
-        dist.init_process_group("nccl", device_id=dev)
-
-    def barrier():
-        if world > 1:
-            dist.barrier()
-        torch.cuda.synchronize()
-
-    def max_over_ranks(x: float) -> float:
-        if world == 1:
-            return x
-        t = torch.tensor([x], dtype=torch.float64, device=dev)
-        dist.all_reduce(t, op=dist.ReduceOp.MAX)
-        return float(t.item())
+    ctx = Dist("nccl", dev)
+    world, rank = ctx.world, ctx.rank
+    barrier, max_over_ranks = ctx.barrier, ctx.max
 
     peak, peak_kind = load_peaks()
     seed = synth.SEED_BASE + args.cfg
@@ -317,7 +348,7 @@ def main():
         total_ms = wall0.elapsed_time(wall1)
     total_ms = max_over_ranks(total_ms)
     step_bytes = bytes_fwd + (bytes_inv if do_inverse else 0)
-    value = world * step_bytes * args.steps / total_ms / 1e6
+    value = whole_job_gbs(world, step_bytes, args.steps, total_ms)
     fwd_avg = sum(fwd_ms) / len(fwd_ms)
     ach = bytes_fwd / fwd_avg / 1e6
 
@@ -359,9 +390,7 @@ def main():
                                 "seconds": spent}
     for p in plans:
         p.close()
-    if world > 1:
-        dist.barrier()
-        dist.destroy_process_group()
+    ctx.close()
     if rank == 0:
         print(json.dumps(line))
 
@@ -487,11 +516,20 @@ def staging_sections(args, cfg, plan, master, arena, seed, base, dev, world, lin
         pageable = torch.empty(4 * n, dtype=torch.uint8)
         pageable.fill_(0)  # commit the pages before timing
         r_out = [plan.stage_out(desc(ptrs[:1], pageable)) for _ in range(2)]
-        ok = bool(np.array_equal(pageable.numpy().view(np.uint32)[:1 << 20], img[:1 << 20]))
+        w = min(n, 1 << 20)
+        ok = bool(np.array_equal(pageable.numpy().view(np.uint32)[:w], img[:w]))
         bufs[0].zero_()
         r_in = [plan.stage_in(desc(ptrs[:1], pageable, order=[0])) for _ in range(2)]
         ok &= synth.cuda_mismatch_f32(bufs[0], seed, ids[0], start=base) == 0
+        small = dr.stage_desc(ptrs[:1], sizes[:1], budget=256 << 20, chunk=64 << 20, host_arena=pageable.data_ptr(),
+                              host_arena_bytes=pageable.numel())
+        s_out = max(plan.stage_out(small).link_gbs for _ in range(2))
+        s_in = max(plan.stage_in(small).link_gbs for _ in range(2))
+        ok &= synth.cuda_mismatch_f32(bufs[0], seed, ids[0], start=base) == 0
         out["staging"]["through_ring_to_pageable"] = {
+            "with_256MiB_budget_64MiB_chunks": {"stage_out_gbs": s_out, "stage_in_gbs": s_in,
+                                                "stage_out_frac_of_link": s_out / link_d2h,
+                                                "stage_in_frac_of_link": s_in / link_h2d},
             "bytes": int(4 * n), "pinned_high_water_bytes": int(r_out[0].pinned_high_water_bytes),
             "stage_out_gbs": max(x.link_gbs for x in r_out), "stage_in_gbs": max(x.link_gbs for x in r_in),
             "stage_out_frac_of_link": max(x.link_gbs for x in r_out) / link_d2h,

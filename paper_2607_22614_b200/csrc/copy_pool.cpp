@@ -1,0 +1,122 @@
+#include "copy_pool.h"
+
+#include <algorithm>
+#include <cstring>
+
+#if defined(__x86_64__)
+#include <immintrin.h>
+#endif
+
+namespace dr {
+namespace {
+
+#if defined(__x86_64__)
+// Streaming copy: ordinary loads, non-temporal 32-byte stores (no read-for-ownership of the destination).
+__attribute__((target("avx2"))) void stream_copy_avx2(char* dst, const char* src, uint64_t n)
+{
+    uint64_t head = (32 - ((uintptr_t)dst & 31)) & 31;
+    if (head > n) head = n;
+    memcpy(dst, src, head);
+    dst += head;
+    src += head;
+    n -= head;
+    uint64_t blocks = n / 128;
+    for (uint64_t i = 0; i < blocks; ++i) {
+        __m256i a = _mm256_loadu_si256((const __m256i*)(src));
+        __m256i b = _mm256_loadu_si256((const __m256i*)(src + 32));
+        __m256i c = _mm256_loadu_si256((const __m256i*)(src + 64));
+        __m256i d = _mm256_loadu_si256((const __m256i*)(src + 96));
+        _mm256_stream_si256((__m256i*)(dst), a);
+        _mm256_stream_si256((__m256i*)(dst + 32), b);
+        _mm256_stream_si256((__m256i*)(dst + 64), c);
+        _mm256_stream_si256((__m256i*)(dst + 96), d);
+        src += 128;
+        dst += 128;
+    }
+    _mm_sfence();
+    memcpy(dst, src, n - blocks * 128);
+}
+bool have_avx2()
+{
+    static const bool v = __builtin_cpu_supports("avx2");
+    return v;
+}
+#endif
+
+void copy_bytes(char* dst, const char* src, uint64_t n)
+{
+#if defined(__x86_64__)
+    if (n >= (1u << 16) && have_avx2()) {
+        stream_copy_avx2(dst, src, n);
+        return;
+    }
+#endif
+    memcpy(dst, src, n);
+}
+
+}  // namespace
+
+CopyPool::CopyPool(unsigned n) : n_(n ? n : 1)
+{
+    for (unsigned i = 1; i < n_; ++i) th_.emplace_back([this, i] { loop(i); });
+}
+
+CopyPool::~CopyPool()
+{
+    {
+        std::lock_guard<std::mutex> l(mu_);
+        stop_ = true;
+        ++gen_;
+    }
+    cv_.notify_all();
+    for (auto& t : th_) t.join();
+}
+
+void CopyPool::copy(void* dst, const void* src, uint64_t n)
+{
+    if (n_ == 1 || n < (1u << 20)) {
+        copy_bytes((char*)dst, (const char*)src, n);
+        return;
+    }
+    {
+        std::lock_guard<std::mutex> l(mu_);
+        dst_ = (char*)dst;
+        src_ = (const char*)src;
+        len_ = n;
+        pending_ = n_ - 1;
+        ++gen_;
+    }
+    cv_.notify_all();
+    part(0);
+    std::unique_lock<std::mutex> l(mu_);
+    done_.wait(l, [this] { return pending_ == 0; });
+}
+
+void CopyPool::part(unsigned i)
+{
+    uint64_t per = (len_ / n_ + 4095) / 4096 * 4096;
+    uint64_t a = std::min<uint64_t>(len_, per * i), b = std::min<uint64_t>(len_, a + per);
+    if (i == n_ - 1) b = len_;
+    if (b > a) copy_bytes(dst_ + a, src_ + a, b - a);
+}
+
+void CopyPool::loop(unsigned i)
+{
+    uint64_t seen = 0;
+    for (;;) {
+        {
+            std::unique_lock<std::mutex> l(mu_);
+            cv_.wait(l, [&] { return gen_ != seen; });
+            seen = gen_;
+            if (stop_) return;
+        }
+        part(i);
+        {
+            std::lock_guard<std::mutex> l(mu_);
+            --pending_;
+        }
+        done_.notify_one();
+    }
+}
+
+}  // namespace dr

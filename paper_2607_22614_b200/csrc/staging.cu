@@ -11,6 +11,7 @@
 #include <functional>
 #include <thread>
 
+#include "copy_pool.h"
 #include "dr_internal.h"
 
 namespace dr {
@@ -20,81 +21,6 @@ namespace {
 using Clock = std::chrono::steady_clock;
 
 double ms_since(Clock::time_point t0) { return std::chrono::duration<double, std::milli>(Clock::now() - t0).count(); }
-
-// Splits one memcpy over a few threads: a single core cannot keep up with the host link.
-class CopyPool {
-public:
-    explicit CopyPool(unsigned n) : n_(n ? n : 1)
-    {
-        for (unsigned i = 1; i < n_; ++i) th_.emplace_back([this, i] { loop(i); });
-    }
-    ~CopyPool()
-    {
-        {
-            std::lock_guard<std::mutex> l(mu_);
-            stop_ = true;
-            ++gen_;
-        }
-        cv_.notify_all();
-        for (auto& t : th_) t.join();
-    }
-    void copy(void* dst, const void* src, uint64_t n)
-    {
-        if (n_ == 1 || n < (1u << 20)) {
-            memcpy(dst, src, n);
-            return;
-        }
-        {
-            std::lock_guard<std::mutex> l(mu_);
-            dst_ = (char*)dst;
-            src_ = (const char*)src;
-            len_ = n;
-            pending_ = n_ - 1;
-            ++gen_;
-        }
-        cv_.notify_all();
-        part(0);
-        std::unique_lock<std::mutex> l(mu_);
-        done_.wait(l, [this] { return pending_ == 0; });
-    }
-
-private:
-    void part(unsigned i)
-    {
-        uint64_t per = (len_ / n_ + 63) / 64 * 64;
-        uint64_t a = std::min<uint64_t>(len_, per * i), b = std::min<uint64_t>(len_, a + per);
-        if (i == n_ - 1) b = len_;
-        if (b > a) memcpy(dst_ + a, src_ + a, b - a);
-    }
-    void loop(unsigned i)
-    {
-        uint64_t seen = 0;
-        for (;;) {
-            {
-                std::unique_lock<std::mutex> l(mu_);
-                cv_.wait(l, [&] { return gen_ != seen; });
-                seen = gen_;
-                if (stop_) return;
-            }
-            part(i);
-            {
-                std::lock_guard<std::mutex> l(mu_);
-                --pending_;
-            }
-            done_.notify_one();
-        }
-    }
-    unsigned n_;
-    std::vector<std::thread> th_;
-    std::mutex mu_;
-    std::condition_variable cv_, done_;
-    uint64_t gen_ = 0;
-    unsigned pending_ = 0;
-    bool stop_ = false;
-    char* dst_ = nullptr;
-    const char* src_ = nullptr;
-    uint64_t len_ = 0;
-};
 
 }  // namespace
 
@@ -216,9 +142,12 @@ int wait_event(cudaEvent_t ev, Clock::time_point deadline)
     }
 }
 
-// Bounded drain of both streams on an error path, so that no copy still targets the ring on return.
-void drain(Ring* r, Clock::time_point deadline)
+// Bounded drain of both streams on an error path, so that no copy still targets the ring or the caller's
+// arena on return.  The bound is generous and independent of the caller's timeout: copies that were already
+// enqueued cannot be cancelled, only waited for.
+void drain(Ring* r)
 {
+    const auto deadline = Clock::now() + std::chrono::seconds(20);
     for (cudaStream_t s : {r->s_copy, r->s_relay})
         while (cudaStreamQuery(s) == cudaErrorNotReady && Clock::now() < deadline)
             std::this_thread::sleep_for(std::chrono::microseconds(50));
@@ -340,7 +269,7 @@ extern "C" int dr_stage_out(dr_plan* plan, const dr_stage_desc* d, dr_stage_stat
         while (rc == DR_OK && next_issue < g.n_chunks && next_issue - next_done < g.slots) rc = issue(next_issue++);
         if (rc == DR_OK && (rc = complete(next_done)) == DR_OK) st.chunks_done = ++next_done;
     }
-    if (rc) drain(r, Clock::now() + limit);
+    if (rc) drain(r);
     st.elapsed_ms = ms_since(t0);
     st.link_gbs = st.elapsed_ms > 0 ? (double)st.bytes / st.elapsed_ms * 1e-6 : 0;
     if (stats) *stats = st;
@@ -429,7 +358,7 @@ extern "C" int dr_stage_in(dr_plan* plan, const dr_stage_desc* d, dr_stage_stats
         if (next_issue < pieces.size() && next_issue - next_done < g.slots) rc = issue(next_issue++);
         else if ((rc = complete(next_done)) == DR_OK) st.chunks_done = ++next_done;
     }
-    if (rc) drain(r, Clock::now() + limit);
+    if (rc) drain(r);
     st.elapsed_ms = ms_since(t0);
     st.link_gbs = st.elapsed_ms > 0 ? (double)st.bytes / st.elapsed_ms * 1e-6 : 0;
     if (stats) *stats = st;

@@ -176,3 +176,24 @@ def test_staging_argument_errors(plan):
     assert dr.dr_stage_out(plan.handle, mk(budget=8192, chunk=4096, host_arena=host.ctypes.data, host_arena_bytes=100))[0] == B.DR_ERR_SIZE
     assert dr.dr_stage_out(plan.handle, mk(budget=8192, chunk=4096))[0] == B.DR_ERR_INVALID
     assert dr.dr_stage_in(plan.handle, mk(budget=8192, chunk=4096, host_arena=host.ctypes.data, host_arena_bytes=4096, order=[3]))[0] == B.DR_ERR_INVALID
+
+
+def test_wait_that_runs_out_returns_timeout_and_the_transfer_resumes(plan):
+    """A 1 ms bound on a 256 MiB copy (about 5 ms on the link) must run out: the call reports
+    DR_ERR_TIMEOUT with the chunks that did complete, the context stays usable, and resuming from
+    chunks_done with a normal bound delivers the same bytes."""
+    n = 256 * MiB
+    t = torch.empty(n // 4 * 3, dtype=torch.int32, device=dev())
+    synth.cuda_fill_f32(t, 17, synth.BUF_ADAM_M)
+    pinned = torch.zeros(3 * n, dtype=torch.uint8).pin_memory()
+    d = dr.stage_desc([t.data_ptr()], [3 * n], budget=2 * n, chunk=n, host_arena=pinned.data_ptr(),
+                      host_arena_bytes=3 * n, timeout_ms=1)
+    rc, st = dr.dr_stage_out(plan.handle, d)
+    assert rc == B.DR_ERR_TIMEOUT and st.chunks_done < st.n_chunks == 3
+    assert "timed out" in dr.dr_last_error()
+    d.timeout_ms = 0
+    d.first_chunk = st.chunks_done
+    rc, st2 = dr.dr_stage_out(plan.handle, d)
+    assert rc == 0 and st2.chunks_done == 3
+    torch.cuda.synchronize()
+    assert np.array_equal(pinned.numpy().view(np.uint32), synth.fill_f32(17, synth.BUF_ADAM_M, 0, 3 * n // 4))
