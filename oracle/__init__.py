@@ -68,6 +68,10 @@ def _l():
         lib.orc_stage_out.argtypes = [p, p, u64, u64, u64, u64, p, p]
         lib.orc_stage_in.restype = i64
         lib.orc_stage_in.argtypes = [p, p, u64, p, u64, u64, p, p]
+        lib.orc_restage_out.restype = None
+        lib.orc_restage_out.argtypes = [p, u64, u64, u64, p]
+        lib.orc_restage_in.restype = None
+        lib.orc_restage_in.argtypes = [p, u64, u64, u64, p]
         _lib = lib
     return _lib
 
@@ -198,3 +202,18 @@ def stage_in(bufs: list[np.ndarray], source: np.ndarray, budget: int, chunk: int
     if n < 0:
         raise ValueError("oracle: budget cannot hold two slots")
     return int(n), list(done)
+
+
+def restage(old_shards: list[np.ndarray], n: int, w_new: int) -> list[np.ndarray]:
+    """Old shards (world = len(old_shards)) -> new shards for world w_new, through a flat host image."""
+    w_old = len(old_shards)
+    image = np.zeros(n, dtype=np.uint32)
+    for r, sh in enumerate(old_shards):
+        assert sh.dtype == np.uint32 and sh.size == -(-n // w_old)
+        _l().orc_restage_out(sh.ctypes.data, n, w_old, r, image.ctypes.data)
+    out = []
+    for q in range(w_new):
+        new = np.empty(-(-n // w_new), dtype=np.uint32)
+        _l().orc_restage_in(image.ctypes.data, n, w_new, q, new.ctypes.data)
+        out.append(new)
+    return out

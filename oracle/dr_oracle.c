@@ -559,3 +559,28 @@ int64_t orc_stage_in(uint8_t *const *bufs, const uint64_t *bytes, uint64_t n_buf
     free(ring);
     return (int64_t)pieces;
 }
+
+/* ---- Re-sharding the training state across a changed world size (Sec. 3.3) -----------------
+ * Old training ranks hold shards of a flat buffer of N elements cut for world W_old
+ * (S_old = ceil(N / W_old), the last shard padded); the new topology cuts the same flat buffer for
+ * W_new.  Staged through a host image of the flat buffer: old rank r writes its real elements to
+ * image[r S_old ...], new rank q reads image[q S_new ...]; elements past N are padding and read as
+ * zero.  Written here element by element (4-byte words).
+ */
+void orc_restage_out(const uint32_t *old_shard, uint64_t N, uint64_t W_old, uint64_t r, uint32_t *image)
+{
+    uint64_t S = (N + W_old - 1) / W_old, i;
+    for (i = 0; i < S; ++i) {
+        uint64_t f = r * S + i;
+        if (f < N) image[f] = old_shard[i];
+    }
+}
+
+void orc_restage_in(const uint32_t *image, uint64_t N, uint64_t W_new, uint64_t q, uint32_t *new_shard)
+{
+    uint64_t S = (N + W_new - 1) / W_new, i;
+    for (i = 0; i < S; ++i) {
+        uint64_t f = q * S + i;
+        new_shard[i] = f < N ? image[f] : 0u;
+    }
+}

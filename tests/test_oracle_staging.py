@@ -60,3 +60,18 @@ def test_budget_must_hold_two_slots():
         oracle.stage_out(bufs, 1000, 600)
     with pytest.raises(ValueError):
         oracle.stage_out(bufs, 4096)  # default chunk rounds down to 0
+
+
+@pytest.mark.parametrize("n,w_old,w_new", [(1000, 6, 4), (1001, 4, 6), (17, 3, 5), (4096, 2, 8), (5, 8, 3)])
+def test_restage_across_world_sizes_is_split_of_the_concatenation(n, w_old, w_new):
+    """The new shards are what numpy's own split of the (zero padded) flat buffer gives."""
+    rng = np.random.default_rng(n)
+    flat = rng.integers(1, 1 << 32, size=n, dtype=np.uint64).astype(np.uint32)
+    s_old, s_new = -(-n // w_old), -(-n // w_new)
+    padded_old = np.concatenate([flat, np.full(w_old * s_old - n, 0xDEAD, dtype=np.uint32)])  # old padding is garbage
+    old = [a.copy() for a in np.split(padded_old, w_old)]
+    new = oracle.restage(old, n, w_new)
+    padded_new = np.concatenate([flat, np.zeros(w_new * s_new - n, dtype=np.uint32)])
+    for got, want in zip(new, np.split(padded_new, w_new)):
+        assert np.array_equal(got, want)
+    assert np.array_equal(np.concatenate(new)[:n], flat)
