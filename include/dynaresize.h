@@ -226,8 +226,17 @@ typedef struct dr_stage_desc {
     void* ready_events[DR_MAX_STAGE_BUFS]; /* stage-in: caller's cudaEvent_t recorded on the copy
                                               stream right after buffer i's last copy; NULL = none   */
     uint32_t timeout_ms;                /* bound on every internal wait; 0 = 60 000                   */
-    uint32_t flags;                     /* 0                                                          */
+    uint32_t flags;                     /* 0 or DR_STAGE_HOST_OFFSETS                                 */
+    uint64_t host_offset[DR_MAX_STAGE_BUFS]; /* with DR_STAGE_HOST_OFFSETS: buffer i rests at
+                                           host_arena + host_offset[i] instead of at its position in
+                                           the stream; regions must not overlap (arena sinks only)    */
 } dr_stage_desc;
+
+/* Buffer i of a stage call rests at host_arena + host_offset[i].  This is how training state crosses a
+ * change of the training world size (Sec. 3.3, old ranks -> new ranks through host memory): every old
+ * rank stages its shard out to its place in one flat host image, every new rank stages its own,
+ * differently cut, range back in (see dr_shard_range). */
+#define DR_STAGE_HOST_OFFSETS 1u
 
 typedef struct dr_stage_stats {
     uint64_t bytes;                    /* bytes moved by this call                                    */
@@ -258,6 +267,18 @@ int dr_stage_out(dr_plan* plan, const dr_stage_desc* desc, dr_stage_stats* stats
  * ready_events[i] tell when buffer i became usable.  Same pump, errors and threading as above.
  */
 int dr_stage_in(dr_plan* plan, const dr_stage_desc* desc, dr_stage_stats* stats);
+
+/*
+ * dr_shard_range -- the flat elements [*begin, *end) that rank `rank` of `world` really holds
+ * (S = ceil(flat_elems / world) per rank; the last ranks' padding past flat_elems is excluded, so
+ * *end - *begin can be smaller than S, or zero).  With it a caller lays out a re-shard across a changed
+ * world size (Sec. 3.3: e.g. 6 training GPUs -> 4): the old rank stages out [begin, end) of its shard
+ * to host_offset = 4 * begin of a flat host image, the new rank stages in its own range from there, and
+ * the part of the new range the GPU already holds can go through a relay sink without touching the
+ * image.  Host arithmetic only.  DR_ERR_INVALID for world == 0, rank >= world or NULL outputs.
+ */
+int dr_shard_range(uint64_t flat_elems, uint32_t world, uint32_t rank, uint64_t* begin, uint64_t* end,
+                   uint64_t* shard_elems);
 
 /* Synchronises the plan's own streams, frees its ring, table and streams.  NULL is accepted. */
 int dr_plan_destroy(dr_plan* plan);

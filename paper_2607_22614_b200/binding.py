@@ -15,9 +15,10 @@ DR_SRC_FSDP_FLAT = 1
 DR_DST_ROLLOUT_FUSED = 1
 DR_F32, DR_BF16 = 1, 2
 DR_MAX_STAGE_BUFS = 8
+DR_STAGE_HOST_OFFSETS = 1
 
 EXPORTS = ["dr_plan_create", "dr_plan_create_host", "dr_plan_query", "dr_plan_tensor", "dr_plan_segment",
-           "dr_reshard", "dr_reshard_inverse", "dr_reshard_static", "dr_stage_out", "dr_stage_in", "dr_plan_destroy", "dr_strerror",
+           "dr_reshard", "dr_reshard_inverse", "dr_reshard_static", "dr_shard_range", "dr_stage_out", "dr_stage_in", "dr_plan_destroy", "dr_strerror",
            "dr_last_error"]
 
 u8, u32, u64, i64, vp = C.c_uint8, C.c_uint32, C.c_uint64, C.c_int64, C.c_void_p
@@ -59,7 +60,8 @@ class dr_stage_desc(C.Structure):
     _fields_ = [("struct_size", u32), ("n_bufs", u32), ("dev_ptr", vp * 8), ("bytes", u64 * 8), ("order", u32 * 8),
                 ("budget_bytes", u64), ("chunk_bytes", u64), ("host_arena", vp), ("host_arena_bytes", u64),
                 ("callback", dr_chunk_fn), ("user", vp), ("relay_dev", vp * 8), ("first_chunk", u64),
-                ("wait_event", vp), ("ready_events", vp * 8), ("timeout_ms", u32), ("flags", u32)]
+                ("wait_event", vp), ("ready_events", vp * 8), ("timeout_ms", u32), ("flags", u32),
+                ("host_offset", u64 * 8)]
 
 
 class dr_stage_stats(C.Structure):
@@ -96,6 +98,7 @@ def lib() -> C.CDLL:
         L.dr_stage_out.argtypes = [vp, P(dr_stage_desc), P(dr_stage_stats)]
         L.dr_stage_in.argtypes = [vp, P(dr_stage_desc), P(dr_stage_stats)]
         L.dr_plan_destroy.argtypes = [vp]
+        L.dr_shard_range.argtypes = [u64, u32, u32, P(u64), P(u64), P(u64)]
         for n in EXPORTS:
             getattr(L, n).restype = C.c_int
         L.dr_strerror.argtypes = [C.c_int]
@@ -126,7 +129,8 @@ def dst_layout(dtype=DR_BF16, arena_align_bytes=256, moe_tp=1) -> dr_dst_layout:
 
 
 def stage_desc(dev_ptrs, sizes, budget, chunk=0, order=None, host_arena=None, host_arena_bytes=0, callback=None,
-               relay_dev=None, first_chunk=0, wait_event=None, ready_events=None, timeout_ms=0) -> dr_stage_desc:
+               relay_dev=None, first_chunk=0, wait_event=None, ready_events=None, timeout_ms=0,
+               host_offsets=None) -> dr_stage_desc:
     d = dr_stage_desc()
     d.struct_size = C.sizeof(dr_stage_desc)
     d.n_bufs = len(dev_ptrs)
@@ -144,6 +148,10 @@ def stage_desc(dev_ptrs, sizes, budget, chunk=0, order=None, host_arena=None, ho
     d.wait_event = wait_event
     for i, e in enumerate(ready_events or []):
         d.ready_events[i] = e
+    if host_offsets is not None:
+        d.flags |= DR_STAGE_HOST_OFFSETS
+        for i, o in enumerate(host_offsets):
+            d.host_offset[i] = o
     return d
 
 
@@ -198,6 +206,12 @@ def dr_stage_out(plan, desc):
 def dr_stage_in(plan, desc):
     st = dr_stage_stats()
     return lib().dr_stage_in(plan, C.byref(desc), C.byref(st)), st
+
+
+def dr_shard_range(flat_elems, world, rank):
+    b, e, s = u64(), u64(), u64()
+    rc = lib().dr_shard_range(flat_elems, world, rank, C.byref(b), C.byref(e), C.byref(s))
+    return rc, b.value, e.value, s.value
 
 
 def dr_plan_destroy(plan):

@@ -217,6 +217,21 @@ int dr_reshard_inverse(const dr_plan* plan, const void* rollout_dev, uint64_t ro
     return launch_reshard(plan, true, nullptr, flat_dev, rollout_dev, cuda_stream);
 }
 
+int dr_shard_range(uint64_t flat_elems, uint32_t world, uint32_t rank, uint64_t* begin, uint64_t* end,
+                   uint64_t* shard_elems)
+{
+    if (!world || rank >= world || !begin || !end) {
+        set_error("bad world/rank or NULL output");
+        return DR_ERR_INVALID;
+    }
+    const uint64_t S = (flat_elems + world - 1) / world;
+    const uint64_t lo = (uint64_t)rank * S, hi = lo + S;
+    *begin = lo < flat_elems ? lo : flat_elems;
+    *end = hi < flat_elems ? hi : flat_elems;
+    if (shard_elems) *shard_elems = S;
+    return DR_OK;
+}
+
 int dr_plan_destroy(dr_plan* plan)
 {
     if (!plan) return DR_OK;

@@ -61,6 +61,8 @@ struct Geometry {
     uint64_t total = 0, chunk = 0, n_chunks = 0;
     uint32_t slots = 0;
     uint64_t prefix[DR_MAX_STAGE_BUFS + 1] = {0};
+    uint64_t host_at[DR_MAX_STAGE_BUFS] = {0};  // where buffer i rests inside the host arena
+    bool scattered = false;                      // host positions differ from stream positions
 };
 
 int geometry(const dr_stage_desc* d, Geometry* g)
@@ -77,6 +79,8 @@ int geometry(const dr_stage_desc* d, Geometry* g)
         g->prefix[i + 1] = g->prefix[i] + d->bytes[i];
     }
     g->total = g->prefix[d->n_bufs];
+    g->scattered = (d->flags & DR_STAGE_HOST_OFFSETS) != 0;
+    for (uint32_t i = 0; i < d->n_bufs; ++i) g->host_at[i] = g->scattered ? d->host_offset[i] : g->prefix[i];
     g->chunk = d->chunk_bytes ? d->chunk_bytes : d->budget_bytes / 2 / 4096 * 4096;
     if (g->chunk == 0 || d->budget_bytes / g->chunk < 2) {
         set_error("budget %llu cannot hold two slots of %llu bytes", (unsigned long long)d->budget_bytes,
@@ -174,10 +178,28 @@ int check_common(dr_plan* p, const dr_stage_desc* d, const Geometry& g, bool out
         set_error("exactly one of callback, relay_dev, host_arena must be given");
         return DR_ERR_INVALID;
     }
-    if (d->host_arena && d->host_arena_bytes < g.total) {
+    if (g.scattered && !d->host_arena) {
+        set_error("DR_STAGE_HOST_OFFSETS needs a host arena");
+        return DR_ERR_INVALID;
+    }
+    if (d->host_arena && !g.scattered && d->host_arena_bytes < g.total) {
         set_error("host arena holds %llu bytes, stream is %llu", (unsigned long long)d->host_arena_bytes,
                   (unsigned long long)g.total);
         return DR_ERR_SIZE;
+    }
+    if (g.scattered) {
+        for (uint32_t i = 0; i < d->n_bufs; ++i) {
+            if (g.host_at[i] + d->bytes[i] > d->host_arena_bytes) {
+                set_error("buffer %u does not fit the host arena at its offset", i);
+                return DR_ERR_SIZE;
+            }
+            for (uint32_t j = 0; j < i; ++j)
+                if (d->bytes[i] && d->bytes[j] && g.host_at[i] < g.host_at[j] + d->bytes[j] &&
+                    g.host_at[j] < g.host_at[i] + d->bytes[i]) {
+                    set_error("host regions of buffers %u and %u overlap", j, i);
+                    return DR_ERR_INVALID;
+                }
+        }
     }
     int dev = -1;
     if (cudaGetDevice(&dev) != cudaSuccess || dev != p->device) {
@@ -215,19 +237,19 @@ extern "C" int dr_stage_out(dr_plan* plan, const dr_stage_desc* d, dr_stage_stat
     st.pinned_high_water_bytes = direct ? 0 : g.chunk * g.slots;
     if (d->wait_event) DR_CUDA(cudaStreamWaitEvent(r->s_copy, (cudaEvent_t)d->wait_event, 0));
 
-    auto slot_ptr = [&](uint64_t k) -> char* {
-        return direct ? (char*)d->host_arena + k * g.chunk : r->base + (k % g.slots) * g.chunk;
-    };
+    // ring slot of chunk k (unused when chunks are copied straight into a pinned arena)
+    auto slot_ptr = [&](uint64_t k) -> char* { return r->base + (k % g.slots) * g.chunk; };
     // enqueue the copies of chunk k: one per buffer it touches
     auto issue = [&](uint64_t k) -> int {
         uint64_t lo = k * g.chunk, hi = std::min(lo + g.chunk, g.total);
         uint32_t s = (uint32_t)(k % g.slots);
-        char* host = slot_ptr(k);
+        char* host = direct ? nullptr : slot_ptr(k);
         for (uint32_t b = 0; b < d->n_bufs; ++b) {
             uint64_t a = std::max(lo, g.prefix[b]), e = std::min(hi, g.prefix[b + 1]);
             if (a >= e) continue;
-            DR_CUDA(cudaMemcpyAsync(host + (a - lo), (const char*)d->dev_ptr[b] + (a - g.prefix[b]), e - a,
-                                    cudaMemcpyDeviceToHost, r->s_copy));
+            char* to = direct ? (char*)d->host_arena + g.host_at[b] + (a - g.prefix[b]) : host + (a - lo);
+            DR_CUDA(cudaMemcpyAsync(to, (const char*)d->dev_ptr[b] + (a - g.prefix[b]), e - a, cudaMemcpyDeviceToHost,
+                                    r->s_copy));
         }
         DR_CUDA(cudaEventRecord(r->ev_copy[s], r->s_copy));
         if (relay) {
@@ -258,7 +280,10 @@ extern "C" int dr_stage_out(dr_plan* plan, const dr_stage_desc* d, dr_stage_stat
                 return DR_ERR_SINK;
             }
         } else if (!relay && !direct) {
-            r->pool->copy((char*)d->host_arena + lo, slot_ptr(k), n);
+            for (uint32_t b = 0; b < d->n_bufs; ++b) {  // one copy per buffer the chunk touches
+                uint64_t a = std::max(lo, g.prefix[b]), e = std::min(lo + n, g.prefix[b + 1]);
+                if (a < e) r->pool->copy((char*)d->host_arena + g.host_at[b] + (a - g.prefix[b]), slot_ptr(k) + (a - lo), e - a);
+            }
         }
         st.bytes += n;
         return DR_OK;
@@ -324,10 +349,11 @@ extern "C" int dr_stage_in(dr_plan* plan, const dr_stage_desc* d, dr_stage_stats
     auto issue = [&](uint64_t i) -> int {
         const Piece& pc = pieces[i];
         uint32_t s = (uint32_t)(i % g.slots);
-        uint64_t off = g.prefix[pc.buf] + pc.pos;
+        uint64_t off = g.prefix[pc.buf] + pc.pos;            // position in the stream (what a callback sees)
+        uint64_t at = g.host_at[pc.buf] + pc.pos;            // position in the host arena
         const char* host;
         if (direct) {
-            host = (const char*)d->host_arena + off;
+            host = (const char*)d->host_arena + at;
         } else {
             char* slot = r->base + (uint64_t)s * g.chunk;
             if (d->callback) {
@@ -336,7 +362,7 @@ extern "C" int dr_stage_in(dr_plan* plan, const dr_stage_desc* d, dr_stage_stats
                     return DR_ERR_SINK;
                 }
             } else {
-                r->pool->copy(slot, (const char*)d->host_arena + off, pc.n);
+                r->pool->copy(slot, (const char*)d->host_arena + at, pc.n);
             }
             host = slot;
         }

@@ -197,3 +197,69 @@ def test_wait_that_runs_out_returns_timeout_and_the_transfer_resumes(plan):
     assert rc == 0 and st2.chunks_done == 3
     torch.cuda.synchronize()
     assert np.array_equal(pinned.numpy().view(np.uint32), synth.fill_f32(17, synth.BUF_ADAM_M, 0, 3 * n // 4))
+
+
+def _split(flat, w):
+    s = -(-flat.size // w)
+    padded = np.concatenate([flat, np.full(w * s - flat.size, 0xDEAD, dtype=np.uint32)])
+    return [a.copy() for a in np.split(padded, w)]
+
+
+@pytest.mark.parametrize("n,w_old,w_new,pinned", [(3_000_001, 6, 4, True), (3_000_001, 4, 6, False), (1_000_000, 3, 5, False)])
+def test_reshard_state_across_world_sizes_through_one_host_image(plan, n, w_old, w_new, pinned):
+    """Six training GPUs become four (the paper's 6:2 -> 4:4 resize): every old rank stages its shard of
+    master, m and v out to its place in a flat host image, every new rank stages its own range back in.
+    Ranks run one after the other on this GPU; the result must be the oracle's re-sharding."""
+    kinds = (synth.BUF_MASTER, synth.BUF_ADAM_M, synth.BUF_ADAM_V)
+    flats = [synth.fill_f32(23, k, 0, n) for k in kinds]
+    image = torch.zeros(3 * 4 * n, dtype=torch.uint8)
+    if pinned:
+        image = image.pin_memory()
+    for r in range(w_old):
+        rc, lo, hi, s_old = dr.dr_shard_range(n, w_old, r)
+        assert rc == 0
+        shards = [to_dev_u32(_split(f, w_old)[r]) for f in flats]
+        d = dr.stage_desc([t.data_ptr() for t in shards], [4 * (hi - lo)] * 3, budget=1 * MiB, chunk=256 * 1024,
+                          host_arena=image.data_ptr(), host_arena_bytes=image.numel(),
+                          host_offsets=[4 * (k * n + lo) for k in range(3)])
+        st = plan.stage_out(d)
+        assert st.bytes == 12 * (hi - lo)
+    want = [oracle.restage(_split(f, w_old), n, w_new) for f in flats]
+    for q in range(w_new):
+        rc, lo, hi, s_new = dr.dr_shard_range(n, w_new, q)
+        new = [torch.zeros(s_new, dtype=torch.int32, device=dev()) for _ in kinds]
+        d = dr.stage_desc([t.data_ptr() for t in new], [4 * (hi - lo)] * 3, budget=1 * MiB, chunk=256 * 1024,
+                          host_arena=image.data_ptr(), host_arena_bytes=image.numel(),
+                          host_offsets=[4 * (k * n + lo) for k in range(3)], order=[0, 1, 2])
+        st = plan.stage_in(d)
+        assert 0 < st.ready_ms[0] <= st.ready_ms[1] <= st.ready_ms[2] or hi == lo
+        for k in range(3):
+            assert np.array_equal(new[k].cpu().numpy().view(np.uint32), want[k][q])
+
+
+def test_part_of_the_new_shard_already_on_this_gpu_moves_through_the_relay(plan):
+    """Old rank 1 of 6 becomes new rank 1 of 4: the overlap of the two ranges never rests on the host."""
+    n = 2_400_000
+    flat = synth.fill_f32(29, synth.BUF_MASTER, 0, n)
+    _, olo, ohi, _ = dr.dr_shard_range(n, 6, 1)
+    _, nlo, nhi, s_new = dr.dr_shard_range(n, 4, 1)
+    lo, hi = max(olo, nlo), min(ohi, nhi)
+    assert lo < hi
+    old = to_dev_u32(flat[olo:ohi].copy())
+    new = torch.zeros(s_new, dtype=torch.int32, device=dev())
+    d = dr.stage_desc([old.data_ptr() + 4 * (lo - olo)], [4 * (hi - lo)], budget=1 * MiB, chunk=128 * 1024,
+                      relay_dev=[new.data_ptr() + 4 * (lo - nlo)])
+    plan.stage_out(d)
+    got = new.cpu().numpy().view(np.uint32)
+    assert np.array_equal(got[lo - nlo:hi - nlo], flat[lo:hi])
+    assert (got[:lo - nlo] == 0).all() and (got[hi - nlo:] == 0).all()
+
+
+def test_host_offset_errors(plan):
+    t = torch.zeros(2048, dtype=torch.int32, device=dev())
+    host = np.zeros(16384, dtype=np.uint8)
+    mk = lambda offs, nbytes=host.size: dr.stage_desc([t.data_ptr(), t.data_ptr() + 4096], [4096, 4096], budget=8192, chunk=4096,
+                                                      host_arena=host.ctypes.data, host_arena_bytes=nbytes, host_offsets=offs)
+    assert dr.dr_stage_out(plan.handle, mk([0, 2048]))[0] == B.DR_ERR_INVALID      # regions overlap
+    assert dr.dr_stage_out(plan.handle, mk([0, 14000]))[0] == B.DR_ERR_SIZE        # runs past the arena
+    assert dr.dr_stage_out(plan.handle, mk([8192, 0]))[0] == 0                     # any order of regions is fine

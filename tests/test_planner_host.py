@@ -124,7 +124,7 @@ def test_library_exports_every_declared_symbol():
 
 def test_struct_sizes_match_the_header_layout():
     assert C.sizeof(dr.dr_model_spec) == 48 and C.sizeof(dr.dr_src_layout) == 28 and C.sizeof(dr.dr_dst_layout) == 20
-    assert C.sizeof(dr.dr_plan_info) == 80 and C.sizeof(dr.dr_tensor_desc) == 96 and C.sizeof(dr.dr_segment_desc) == 56
+    assert C.sizeof(dr.dr_stage_desc) == 432 and C.sizeof(dr.dr_stage_stats) == 112 and C.sizeof(dr.dr_plan_info) == 80 and C.sizeof(dr.dr_tensor_desc) == 96 and C.sizeof(dr.dr_segment_desc) == 56
 
 
 def test_error_codes():
@@ -156,3 +156,15 @@ def test_error_codes():
     assert dr.dr_plan_tensor(p.handle, 10_000)[0] == dr.binding.DR_ERR_INVALID
     assert "budget" in dr.dr_strerror(dr.binding.DR_ERR_BUDGET)
     assert dr.dr_plan_destroy(None) == 0
+
+
+def test_shard_range():
+    assert dr.dr_shard_range(1000, 6, 0) == (0, 0, 167, 167)
+    assert dr.dr_shard_range(1000, 6, 5) == (0, 835, 1000, 167)      # last shard holds 165 real elements
+    assert dr.dr_shard_range(5, 8, 4) == (0, 4, 5, 1)
+    assert dr.dr_shard_range(5, 8, 7) == (0, 5, 5, 1)                # all padding
+    assert dr.dr_shard_range(5, 8, 8)[0] == dr.binding.DR_ERR_INVALID
+    assert dr.dr_shard_range(5, 0, 0)[0] == dr.binding.DR_ERR_INVALID
+    for n, w in ((1_975_808, 2), (14_768_307_200, 4), (17, 3)):
+        ends = [dr.dr_shard_range(n, w, r)[1:3] for r in range(w)]
+        assert ends[0][0] == 0 and ends[-1][1] == n and all(a[1] == b[0] for a, b in zip(ends, ends[1:]))
