@@ -511,6 +511,21 @@ def staging_sections(args, cfg, plan, master, arena, seed, base, dev, world, lin
                              "all_state_resident_deferred": st_in.elapsed_ms},
     }
 
+    # re-shard across a changed training world size (Sec. 3.3): the image above is the flat state; a new rank 1 of a
+    # world of 4 stages its own range of master, m, v in (weights first), then the old cut is put back
+    if len(bufs) == 3 and not cfg["gathered"] is False:
+        rc, lo, hi, s4 = dr.dr_shard_range(n, 4, 1)
+        d4 = dr.stage_desc(ptrs, [4 * (hi - lo)] * 3, budget=budget, host_arena=image.data_ptr(),
+                           host_arena_bytes=image.numel(), host_offsets=[4 * (k * n + lo) for k in range(3)], order=[0, 1, 2])
+        r4 = [plan.stage_in(d4) for _ in range(2)]
+        ok4 = all(synth.cuda_mismatch_f32(b[:hi - lo], seed, bid, start=base + lo) == 0 for b, bid in zip(bufs, ids))
+        best = max(r4, key=lambda x: x.link_gbs)
+        out["restage"] = {"what": "new rank 1 of world 4 stages its range of master, m, v in from the flat host image",
+                          "bytes": int(best.bytes), "stage_in_gbs": best.link_gbs, "frac_of_link": best.link_gbs / link_h2d,
+                          "weights_resident_ms": best.ready_ms[0], "all_state_resident_ms": best.elapsed_ms,
+                          "matches_generator": bool(ok4)}
+        plan.stage_in(desc(ptrs, image, order=order))
+
     # the same engine with a pageable resting place: chunks go through the pinned ring and worker threads
     if mem_available_bytes() > 4 * n * 1.5:
         pageable = torch.empty(4 * n, dtype=torch.uint8)

@@ -30,6 +30,10 @@ class _Spec(ctypes.Structure):
         "n_experts", "moe_ffn", "tied", "qk_norm")]
 
 
+class _Opts(ctypes.Structure):
+    _fields_ = [(n, ctypes.c_uint32) for n in ("kv_replicate", "vocab_pad", "moe_tp", "moe_ep", "moe_ep_rank")]
+
+
 _lib = None
 
 
@@ -47,6 +51,8 @@ def _l():
         lib.orc_widen_bf16.argtypes = [ctypes.c_uint16]
         lib.orc_model_create.restype = p
         lib.orc_model_create.argtypes = [ctypes.POINTER(_Spec), u64, u64, u64, u64, u64, u64]
+        lib.orc_model_create_ex.restype = p
+        lib.orc_model_create_ex.argtypes = [ctypes.POINTER(_Spec), u64, u64, u64, u64, u64, u64, ctypes.POINTER(_Opts)]
         lib.orc_model_destroy.restype = None
         lib.orc_model_destroy.argtypes = [p]
         for n in ("orc_n_src", "orc_n_dst", "orc_flat_elems", "orc_shard_elems", "orc_arena_bytes"):
@@ -114,9 +120,12 @@ class Model:
     """Source (D1, D2) and rollout (D3) layouts of one model spec at (W, T, t)."""
 
     def __init__(self, spec: dict, *, align: int = 1, world: int = 1, tp: int = 1, tp_rank: int = 0,
-                 elem_size: int = 2, arena_align: int = 256):
+                 elem_size: int = 2, arena_align: int = 256, kv_replicate: bool = False, vocab_pad: int = 0,
+                 moe_tp: int = 1, moe_ep: int = 1, moe_ep_rank: int = 0):
         s = _Spec(**{k: int(spec.get(k, 0)) for k, _ in _Spec._fields_})
-        self._h = _l().orc_model_create(ctypes.byref(s), align, world, tp, tp_rank, elem_size, arena_align)
+        o = _Opts(int(kv_replicate), vocab_pad, moe_tp, moe_ep, moe_ep_rank)
+        self._h = _l().orc_model_create_ex(ctypes.byref(s), align, world, tp, tp_rank, elem_size, arena_align,
+                                           ctypes.byref(o))
         if not self._h:
             raise ValueError("oracle: unsupported spec / layout")
         self.elem_size = elem_size

@@ -58,8 +58,21 @@ typedef struct {
     orc_part *parts;
 } orc_dst;
 
+/* Rollout layout variants beyond the base definition (all off / 1 by default):
+ *   kv_replicate  tp may exceed the kv heads (tp % n_kv_heads == 0): rank t holds the one kv head
+ *                 t / (tp / n_kv_heads), i.e. each kv head is replicated on tp / n_kv_heads ranks
+ *   vocab_pad     embed / lm_head rows are padded up to a multiple of vocab_pad before slicing; the
+ *                 padding rows exist in the arena but have no source element (never written)
+ *   moe_tp        1: experts unsliced; == tp: expert FFN width sliced like the dense MLP
+ *   moe_ep, moe_ep_rank   expert parallelism: the rank keeps the contiguous block of
+ *                 n_experts / moe_ep experts number moe_ep_rank */
+typedef struct {
+    uint32_t kv_replicate, vocab_pad, moe_tp, moe_ep, moe_ep_rank;
+} orc_opts;
+
 typedef struct {
     orc_spec spec;
+    orc_opts opt;
     uint64_t align, world, tp, tp_rank, elem_size, arena_align;
     uint64_t n_src, n_dst;
     orc_src *src;
@@ -221,9 +234,22 @@ static void build_dst(orc_model *m)
     orc_dst *d;
     int64_t embed_index;
 
-    /* embed_t = embed[t V/T : (t+1) V/T, :] */
+    /* vocabulary rows of this rank: [t Vp/T, (t+1) Vp/T) of the matrix padded to Vp rows; only rows < V exist */
+    const uint64_t Vp = m->opt.vocab_pad ? align_up(V, m->opt.vocab_pad) : V;
+    const uint64_t v_lo = t * (Vp / T), v_hi = (t + 1) * (Vp / T);
+    const uint64_t v_real = v_lo >= V ? 0 : (v_hi <= V ? v_hi - v_lo : V - v_lo);
+    /* kv heads of this rank: nkv / T of them, or with replication the single head t / (T / nkv) */
+    const int kv_rep = m->opt.kv_replicate && T > nkv;
+    const uint64_t kv_rows = kv_rep ? hd : (nkv / T) * hd;
+    const uint64_t kv_row0 = kv_rep ? (t / (T / nkv)) * hd : t * (nkv / T) * hd;
+    /* experts of this rank and their width */
+    const uint64_t EP = m->opt.moe_ep ? m->opt.moe_ep : 1, E_loc = c->n_experts / EP, e0 = m->opt.moe_ep_rank * E_loc;
+    const uint64_t MT = m->opt.moe_tp > 1 ? T : 1, mt = m->opt.moe_tp > 1 ? t : 0;
+
+    /* embed_t = embed[t Vp/T : (t+1) Vp/T, :] */
     d = push_dst(m, &cap, "embed", H);
-    add_part(d, find_src(m, -1, "embed"), t * (V / T), 0, V / T);
+    if (v_real) add_part(d, find_src(m, -1, "embed"), v_lo, 0, v_real);
+    d->rows = Vp / T;
     embed_index = (int64_t)m->n_dst - 1;
 
     for (l = 0; l < c->n_layers; ++l) {
@@ -234,8 +260,8 @@ static void build_dst(orc_model *m)
         /* qkv = [ q rows of rank t ; k rows of rank t ; v rows of rank t ] */
         d = D("qkv", H);
         add_part(d, S("q"), t * (nq / T) * hd, 0, (nq / T) * hd);
-        add_part(d, S("k"), t * (nkv / T) * hd, 0, (nkv / T) * hd);
-        add_part(d, S("v"), t * (nkv / T) * hd, 0, (nkv / T) * hd);
+        add_part(d, S("k"), kv_row0, 0, kv_rows);
+        add_part(d, S("v"), kv_row0, 0, kv_rows);
         if (c->qk_norm) {
             d = D("q_norm", hd);
             add_part(d, S("q_norm"), 0, 0, 1);
@@ -256,22 +282,22 @@ static void build_dst(orc_model *m)
             d = D("down", F / T);
             add_part(d, S("down"), 0, t * (F / T), H);
         } else {
-            const uint64_t Fm = c->moe_ffn;
+            const uint64_t Fm = c->moe_ffn, Fs = Fm / MT; /* width kept per expert */
             d = D("router", H);
             add_part(d, S("router"), 0, 0, c->n_experts);
-            /* w13[e] = [gate_e ; up_e], expert-major, experts not sliced */
+            /* w13[j] = [gate_e rows of this rank ; up_e rows of this rank], e = e0 + j, expert-major */
             d = D("w13", H);
-            for (e = 0; e < c->n_experts; ++e) {
+            for (e = (uint32_t)e0; e < e0 + E_loc; ++e) {
                 snprintf(sn, sizeof sn, "layers.%u.experts.%u.gate", l, e);
-                add_part(d, find_src(m, l, sn), 0, 0, Fm);
+                add_part(d, find_src(m, l, sn), mt * Fs, 0, Fs);
                 snprintf(sn, sizeof sn, "layers.%u.experts.%u.up", l, e);
-                add_part(d, find_src(m, l, sn), 0, 0, Fm);
+                add_part(d, find_src(m, l, sn), mt * Fs, 0, Fs);
             }
-            /* w2[e] = down_e */
-            d = D("w2", Fm);
-            for (e = 0; e < c->n_experts; ++e) {
+            /* w2[j] = down_e columns of this rank */
+            d = D("w2", Fs);
+            for (e = (uint32_t)e0; e < e0 + E_loc; ++e) {
                 snprintf(sn, sizeof sn, "layers.%u.experts.%u.down", l, e);
-                add_part(d, find_src(m, l, sn), 0, 0, H);
+                add_part(d, find_src(m, l, sn), 0, mt * Fs, H);
             }
         }
 #undef D
@@ -284,7 +310,8 @@ static void build_dst(orc_model *m)
         d->alias_of = embed_index;
         d->rows = m->dst[embed_index].rows;
     } else {
-        add_part(d, find_src(m, -1, "lm_head"), t * (V / T), 0, V / T);
+        if (v_real) add_part(d, find_src(m, -1, "lm_head"), v_lo, 0, v_real);
+        d->rows = Vp / T;
     }
     /* arena offsets: tensors in order, each start aligned up to arena_align bytes */
     for (i = 0; i < m->n_dst; ++i) {
@@ -300,17 +327,28 @@ static void build_dst(orc_model *m)
     m->arena_bytes = off;
 }
 
-/* Returns NULL when the shapes do not divide by T (no KV-head replication, no padding). */
-orc_model *orc_model_create(const orc_spec *spec, uint64_t align, uint64_t world, uint64_t tp, uint64_t tp_rank,
-                            uint64_t elem_size, uint64_t arena_align)
+/* Returns NULL when the shapes do not divide as the chosen options need. */
+orc_model *orc_model_create_ex(const orc_spec *spec, uint64_t align, uint64_t world, uint64_t tp, uint64_t tp_rank,
+                               uint64_t elem_size, uint64_t arena_align, const orc_opts *opt)
 {
     orc_model *m;
+    orc_opts o = {0, 0, 1, 1, 0};
+    uint64_t Vp;
+    if (opt) o = *opt;
     if (!spec || align == 0 || world == 0 || tp == 0 || tp_rank >= tp || arena_align == 0) return NULL;
     if (elem_size != 2 && elem_size != 4) return NULL;
-    if (spec->n_q_heads % tp || spec->n_kv_heads % tp || spec->vocab % tp) return NULL;
+    if (spec->n_q_heads % tp) return NULL;
+    if (spec->n_kv_heads % tp && !(o.kv_replicate && tp > spec->n_kv_heads && tp % spec->n_kv_heads == 0)) return NULL;
+    Vp = o.vocab_pad ? align_up(spec->vocab, o.vocab_pad) : spec->vocab;
+    if (Vp % tp) return NULL;
     if (spec->n_experts == 0 && spec->ffn % tp) return NULL;
+    if (o.moe_tp != 1 && o.moe_tp != tp) return NULL;
+    if (spec->n_experts && o.moe_tp > 1 && spec->moe_ffn % tp) return NULL;
+    if (o.moe_ep == 0) o.moe_ep = 1;
+    if (spec->n_experts % o.moe_ep || o.moe_ep_rank >= o.moe_ep) return NULL;
     m = (orc_model *)calloc(1, sizeof *m);
     m->spec = *spec;
+    m->opt = o;
     m->align = align;
     m->world = world;
     m->tp = tp;
@@ -320,6 +358,12 @@ orc_model *orc_model_create(const orc_spec *spec, uint64_t align, uint64_t world
     enumerate_src(m);
     build_dst(m);
     return m;
+}
+
+orc_model *orc_model_create(const orc_spec *spec, uint64_t align, uint64_t world, uint64_t tp, uint64_t tp_rank,
+                            uint64_t elem_size, uint64_t arena_align)
+{
+    return orc_model_create_ex(spec, align, world, tp, tp_rank, elem_size, arena_align, NULL);
 }
 
 void orc_model_destroy(orc_model *m)

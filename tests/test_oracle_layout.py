@@ -173,3 +173,56 @@ def test_unsupported_divisibility_is_rejected():
         oracle.Model(spec, tp=4)  # 2 kv heads cannot be split 4 ways: no replication
     with pytest.raises(ValueError):
         oracle.Model(spec, tp=3)
+
+
+VARIANTS = [
+    # (spec, tp, options)
+    (dict(BRUTE[0]["spec"], ffn=12), 4, dict(kv_replicate=True, vocab_pad=8)),   # 2 kv heads on 4 ranks; vocab 6 -> 8
+    (MID[0]["spec"], 16, dict(kv_replicate=True)),                               # 8 kv heads on 16 ranks
+    (MID[1]["spec"], 4, dict(vocab_pad=64)),                                     # vocab 5000 -> 5056, tied
+    (dict(MID[1]["spec"], tied=0), 2, dict(vocab_pad=1024)),                     # last rank partly padding
+    (BRUTE[2]["spec"], 2, dict(moe_tp=2)),                                       # expert FFN sliced
+    (BRUTE[2]["spec"], 2, dict(moe_ep=2, moe_ep_rank=1)),                        # expert block 1 of 2
+    (MID[2]["spec"], 4, dict(moe_tp=4, moe_ep=2, moe_ep_rank=0, vocab_pad=64)),
+    (MID[2]["spec"], 8, dict(kv_replicate=True, moe_ep=4, moe_ep_rank=3)),
+]
+
+
+@pytest.mark.parametrize("spec,T,opts", VARIANTS, ids=[f"v{i}" for i in range(len(VARIANTS))])
+def test_layout_variants_equal_torch_chunk_cat(spec, T, opts):
+    N = closed_form(spec)
+    iota = torch.arange(N, dtype=torch.int32)
+    params = named_params(spec, iota)
+    for t in sorted({0, 1, T // 2, T - 1}):
+        m = oracle.Model(spec, tp=T, tp_rank=t, elem_size=4, arena_align=64, **opts)
+        arena = np.full(m.arena_bytes, 0xFF, dtype=np.uint8)  # int32 -1 wherever nothing is written
+        m.forward(iota.numpy().view(np.uint32), arena)
+        want = rollout_state(spec, params, T, t, fill=-1, **opts)
+        for i, d in enumerate(m.dst_tensors()):
+            if d.alias_of >= 0:
+                continue
+            got = _arena_tensor(m, arena, d, np.int32)
+            w = want[d.name].reshape(d.rows, d.cols).numpy()
+            assert np.array_equal(got, w), (d.name, t)
+            assert np.array_equal(m.map_rows(i, 0, d.rows, d.cols), got)  # unmapped padding rows are -1 in both
+        # inverse restores exactly what forward read
+        back = np.full(N, 0x7E7E7E7E, dtype=np.uint32)
+        m.inverse(arena, back)
+        hit = back != 0x7E7E7E7E
+        assert np.array_equal(back[hit], iota.numpy().view(np.uint32)[hit])
+        mapped = np.concatenate([m.map_rows(i, 0, d.rows, d.cols).ravel()
+                                 for i, d in enumerate(m.dst_tensors()) if d.alias_of < 0])
+        assert hit.sum() == np.unique(mapped[mapped >= 0]).size
+
+
+def test_variant_divisibility_rules():
+    with pytest.raises(ValueError):
+        oracle.Model(BRUTE[0]["spec"], tp=4)                              # needs kv_replicate
+    with pytest.raises(ValueError):
+        oracle.Model(MID[0]["spec"], tp=3, kv_replicate=True)             # 3 is not a multiple of 8 kv heads
+    with pytest.raises(ValueError):
+        oracle.Model(MID[1]["spec"], tp=16)                               # vocab 5000 needs padding for 16 ranks
+    with pytest.raises(ValueError):
+        oracle.Model(BRUTE[2]["spec"], tp=2, moe_ep=3)                    # 4 experts, 3 blocks
+    with pytest.raises(ValueError):
+        oracle.Model(BRUTE[2]["spec"], tp=4, kv_replicate=True, moe_tp=2) # moe_tp is 1 or tp

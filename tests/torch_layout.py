@@ -42,14 +42,30 @@ def named_params(spec, flat_values):
     return OrderedDict((n, t.view(s)) for (n, s), t in zip(shapes.items(), pieces))
 
 
-def rollout_state(spec, params, tp, t):
-    """Fused, tensor-parallel-sliced rollout tensors for rank t of tp (values untouched)."""
+def _vocab_rows(w, tp, t, pad_to, fill):
+    """Rows of rank t after padding the vocabulary up to a multiple of pad_to (padding rows = fill)."""
+    if pad_to:
+        extra = -w.shape[0] % pad_to
+        w = torch.nn.functional.pad(w, (0, 0, 0, extra), value=fill)
+    return w.chunk(tp, dim=0)[t]
+
+
+def rollout_state(spec, params, tp, t, kv_replicate=False, vocab_pad=0, moe_tp=1, moe_ep=1, moe_ep_rank=0, fill=-1):
+    """Fused, tensor-parallel-sliced rollout tensors for rank t of tp (values untouched; vocabulary
+    padding rows hold `fill`)."""
     out = OrderedDict()
-    out["embed"] = params["embed"].chunk(tp, dim=0)[t]
+    nkv = spec["n_kv_heads"]
+
+    def kv(w):
+        if kv_replicate and tp > nkv:  # one head per rank, each head on tp / nkv consecutive ranks
+            return w.view(nkv, spec["head_dim"], -1)[t // (tp // nkv)]
+        return w.chunk(tp, dim=0)[t]
+
+    out["embed"] = _vocab_rows(params["embed"], tp, t, vocab_pad, fill)
     for l in range(spec["n_layers"]):
         p = f"layers.{l}."
         out[p + "in_norm"] = params[p + "in_norm"]
-        out[p + "qkv"] = torch.cat([params[p + n].chunk(tp, dim=0)[t] for n in ("q", "k", "v")], dim=0)
+        out[p + "qkv"] = torch.cat([params[p + "q"].chunk(tp, dim=0)[t], kv(params[p + "k"]), kv(params[p + "v"])], dim=0)
         if spec["qk_norm"]:
             out[p + "q_norm"] = params[p + "q_norm"]
             out[p + "k_norm"] = params[p + "k_norm"]
@@ -61,10 +77,13 @@ def rollout_state(spec, params, tp, t):
         else:
             out[p + "router"] = params[p + "router"]
             E = spec["n_experts"]
+            mine = list(torch.arange(E).chunk(moe_ep)[moe_ep_rank])  # expert parallelism: a contiguous block
+            mt, mr = (tp, t) if moe_tp > 1 else (1, 0)                # expert tensor parallelism
             out[p + "w13"] = torch.stack(
-                [torch.cat([params[p + f"experts.{e}.gate"], params[p + f"experts.{e}.up"]], dim=0) for e in range(E)])
-            out[p + "w2"] = torch.stack([params[p + f"experts.{e}.down"] for e in range(E)])
+                [torch.cat([params[p + f"experts.{int(e)}.gate"].chunk(mt, dim=0)[mr],
+                            params[p + f"experts.{int(e)}.up"].chunk(mt, dim=0)[mr]], dim=0) for e in mine])
+            out[p + "w2"] = torch.stack([params[p + f"experts.{int(e)}.down"].chunk(mt, dim=1)[mr] for e in mine])
     out["final_norm"] = params["final_norm"]
     if not spec["tied"]:
-        out["lm_head"] = params["lm_head"].chunk(tp, dim=0)[t]
+        out["lm_head"] = _vocab_rows(params["lm_head"], tp, t, vocab_pad, fill)
     return out
