@@ -83,10 +83,20 @@ typedef struct dr_src_layout {
  *   o columns of this rank, post_norm, dense: gate_up = [gate_t; up_t], down columns of this rank |
  *   MoE: router, w13[e] = [gate_e; up_e] for every expert, w2[e] = down_e;
  *   final_norm; lm_head rows of this rank (an alias of embed when tied).
- * Norms and the router are replicated on every rank; experts are not sliced (moe_tp must be 1). */
+ * Norms and the router are replicated on every rank; by default experts are neither sliced nor
+ * dropped.  The optional fields select the variants rollout engines use (kv-head replication,
+ * vocabulary padding, expert tensor / expert parallelism). */
 typedef struct dr_dst_layout {
     uint32_t struct_size, kind /* DR_DST_ROLLOUT_FUSED */, dtype /* DR_BF16 or DR_F32 */;
-    uint32_t moe_tp /* 1 */, arena_align_bytes /* power of two >= 16, e.g. 256 */;
+    uint32_t moe_tp;            /* 1: experts unsliced; == tp: expert FFN width sliced like the dense MLP
+                                   (gate_e / up_e rows, down_e columns of this rank)                     */
+    uint32_t arena_align_bytes; /* power of two >= 16, e.g. 256                                          */
+    uint32_t kv_replicate;      /* 1: tp may be a multiple of n_kv_heads; rank t then holds the single kv
+                                   head t / (tp / n_kv_heads) (each head on tp / n_kv_heads ranks)       */
+    uint32_t vocab_pad;         /* > 0: embed / lm_head are padded to a multiple of this many rows before
+                                   slicing; padding rows occupy the arena but are never written or read  */
+    uint32_t moe_ep;            /* expert parallel degree (0 or 1: all experts); must divide n_experts   */
+    uint32_t moe_ep_rank;       /* this rank keeps experts [rank * E / ep, (rank + 1) * E / ep)           */
 } dr_dst_layout;
 
 typedef struct dr_plan dr_plan;
@@ -126,8 +136,9 @@ typedef struct dr_segment_desc {
  * dr_plan_create -- compile the un-flatten / fuse / slice map for (spec, src, dst, tp, rank) into a
  * segment table and upload it to the current device (one small H2D copy; synchronous).  This is the
  * metadata a resize prepares ahead of the switch (Sec. 3.2 applies the same idea to communicators).
- * Errors: DR_ERR_INVALID, DR_ERR_UNSUPPORTED (n_q_heads, n_kv_heads, ffn or vocab not divisible by
- * tp; moe_tp != 1), DR_ERR_NOMEM, DR_ERR_CUDA.  *out is NULL on failure.
+ * Errors: DR_ERR_INVALID, DR_ERR_UNSUPPORTED (n_q_heads, ffn, the padded vocabulary or, without
+ * kv_replicate, n_kv_heads not divisible by tp; moe_tp not 1 or tp; moe_ep not dividing n_experts),
+ * DR_ERR_NOMEM, DR_ERR_CUDA.  *out is NULL on failure.
  */
 int dr_plan_create(const dr_model_spec* spec, const dr_src_layout* src, const dr_dst_layout* dst, uint32_t tp,
                    uint32_t rank, dr_plan** out);

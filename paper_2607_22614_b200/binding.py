@@ -36,7 +36,8 @@ class dr_src_layout(C.Structure):
 
 
 class dr_dst_layout(C.Structure):
-    _fields_ = [("struct_size", u32), ("kind", u32), ("dtype", u32), ("moe_tp", u32), ("arena_align_bytes", u32)]
+    _fields_ = [("struct_size", u32), ("kind", u32), ("dtype", u32), ("moe_tp", u32), ("arena_align_bytes", u32),
+                ("kv_replicate", u32), ("vocab_pad", u32), ("moe_ep", u32), ("moe_ep_rank", u32)]
 
 
 class dr_plan_info(C.Structure):
@@ -123,9 +124,11 @@ def src_layout(world=1, rank=0, gathered=True, align_elems=1) -> dr_src_layout:
                          rank=rank, gathered=int(gathered), align_elems=align_elems)
 
 
-def dst_layout(dtype=DR_BF16, arena_align_bytes=256, moe_tp=1) -> dr_dst_layout:
+def dst_layout(dtype=DR_BF16, arena_align_bytes=256, moe_tp=1, kv_replicate=False, vocab_pad=0, moe_ep=1,
+               moe_ep_rank=0) -> dr_dst_layout:
     return dr_dst_layout(struct_size=C.sizeof(dr_dst_layout), kind=DR_DST_ROLLOUT_FUSED, dtype=dtype, moe_tp=moe_tp,
-                         arena_align_bytes=arena_align_bytes)
+                         arena_align_bytes=arena_align_bytes, kv_replicate=int(kv_replicate), vocab_pad=vocab_pad,
+                         moe_ep=moe_ep, moe_ep_rank=moe_ep_rank)
 
 
 def stage_desc(dev_ptrs, sizes, budget, chunk=0, order=None, host_arena=None, host_arena_bytes=0, callback=None,
@@ -231,10 +234,12 @@ class Plan:
     """Owns one ``dr_plan``.  ``host_only=True`` builds the planner's tables without touching CUDA."""
 
     def __init__(self, spec: dict, *, world=1, rank=0, gathered=True, align_elems=1, tp=1, tp_rank=0,
-                 dtype=DR_BF16, arena_align_bytes=256, host_only=False):
+                 dtype=DR_BF16, arena_align_bytes=256, host_only=False, moe_tp=1, kv_replicate=False, vocab_pad=0,
+                 moe_ep=1, moe_ep_rank=0):
         create = dr_plan_create_host if host_only else dr_plan_create
         rc, self.handle = create(model_spec(spec), src_layout(world, rank, gathered, align_elems),
-                                 dst_layout(dtype, arena_align_bytes), tp, tp_rank)
+                                 dst_layout(dtype, arena_align_bytes, moe_tp, kv_replicate, vocab_pad, moe_ep,
+                                            moe_ep_rank), tp, tp_rank)
         if rc:
             self.handle = None
             raise DrError(rc, "dr_plan_create")

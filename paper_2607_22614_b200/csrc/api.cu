@@ -51,12 +51,25 @@ int validate(const dr_model_spec* s, const dr_src_layout* a, const dr_dst_layout
         set_error("arena_align_bytes must be a power of two >= 16");
         return DR_ERR_INVALID;
     }
-    if (b->moe_tp != 1) {
-        set_error("moe_tp must be 1 (experts are not sliced)");
+    if (b->moe_tp != 1 && b->moe_tp != tp) {
+        set_error("moe_tp must be 1 (experts unsliced) or tp");
         return DR_ERR_UNSUPPORTED;
     }
-    if (s->n_q_heads % tp || s->n_kv_heads % tp || s->vocab % tp || (s->n_experts == 0 && s->ffn % tp)) {
-        set_error("n_q_heads, n_kv_heads, ffn and vocab must be divisible by tp (no replication or padding)");
+    const bool kv_ok = s->n_kv_heads % tp == 0 || (b->kv_replicate && tp > s->n_kv_heads && tp % s->n_kv_heads == 0);
+    const uint64_t vp = b->vocab_pad ? ((uint64_t)s->vocab + b->vocab_pad - 1) / b->vocab_pad * b->vocab_pad : s->vocab;
+    if (s->n_q_heads % tp || !kv_ok || vp % tp || (s->n_experts == 0 && s->ffn % tp) ||
+        (s->n_experts && b->moe_tp > 1 && s->moe_ffn % tp)) {
+        set_error("n_q_heads, n_kv_heads (or tp a multiple of it with kv_replicate), ffn and the padded vocabulary "
+                  "must be divisible by tp");
+        return DR_ERR_UNSUPPORTED;
+    }
+    const uint32_t ep = b->moe_ep ? b->moe_ep : 1;
+    if (b->moe_ep_rank >= ep) {
+        set_error("moe_ep_rank out of range");
+        return DR_ERR_INVALID;
+    }
+    if (s->n_experts % ep) {
+        set_error("moe_ep must divide n_experts");
         return DR_ERR_UNSUPPORTED;
     }
     return DR_OK;

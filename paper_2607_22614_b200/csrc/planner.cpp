@@ -60,6 +60,13 @@ struct Emit {
         t.rows += nr;
         arena = t.arena_off + t.rows * t.cols * p->elem_size;
     }
+    // The tensor owns `rows` rows in the arena even if fewer have a source (vocabulary padding).
+    void pad_rows(uint64_t rows)
+    {
+        Tensor& t = p->tensors.back();
+        if (rows > t.rows) t.rows = rows;
+        arena = t.arena_off + t.rows * t.cols * p->elem_size;
+    }
 };
 
 bool contiguous(const HostSeg& g) { return g.rows == 1; }
@@ -200,9 +207,21 @@ int compile_plan(dr_plan* p)
     Emit out{p};
     char nm[64];
 
+    // layout variants
+    const dr_dst_layout& L = p->dst;
+    const uint64_t Vp = L.vocab_pad ? (V + L.vocab_pad - 1) / L.vocab_pad * L.vocab_pad : V;
+    const uint64_t v_lo = t * (Vp / T), v_hi = (t + 1) * (Vp / T);
+    const uint64_t v_real = v_lo >= V ? 0 : std::min(v_hi, V) - v_lo;  // rows of this rank that exist
+    const bool kv_rep = L.kv_replicate && T > nkv;
+    const uint64_t kv_rows = kv_rep ? hd : (nkv / T) * hd;
+    const uint64_t kv_row0 = kv_rep ? (t / (T / nkv)) * hd : t * (nkv / T) * hd;
+    const uint64_t EP = L.moe_ep ? L.moe_ep : 1, E_loc = E / EP, e_first = L.moe_ep_rank * E_loc;
+    const uint64_t MT = L.moe_tp > 1 ? T : 1, mt = L.moe_tp > 1 ? t : 0;
+
     Param embed = flat.take(V, H);
     out.begin("embed", H);
-    out.block(embed, t * (V / T), 0, V / T);
+    out.block(embed, v_lo, 0, v_real);
+    out.pad_rows(Vp / T);
     const int64_t embed_index = 0;
 
     for (uint32_t l = 0; l < s.n_layers; ++l) {
@@ -224,8 +243,8 @@ int compile_plan(dr_plan* p)
         out.block(in_norm, 0, 0, 1);
         out.begin(name("qkv"), H);
         out.block(q, t * (nq / T) * hd, 0, (nq / T) * hd);
-        out.block(k, t * (nkv / T) * hd, 0, (nkv / T) * hd);
-        out.block(v, t * (nkv / T) * hd, 0, (nkv / T) * hd);
+        out.block(k, kv_row0, 0, kv_rows);
+        out.block(v, kv_row0, 0, kv_rows);
         if (s.qk_norm) {
             out.begin(name("q_norm"), hd);
             out.block(q_norm, 0, 0, 1);
@@ -253,13 +272,14 @@ int compile_plan(dr_plan* p)
             }
             out.begin(name("router"), H);
             out.block(router, 0, 0, E);
+            const uint64_t Fs = Fm / MT;  // expert width kept by this rank
             out.begin(name("w13"), H);
-            for (uint64_t e = 0; e < E; ++e) {
-                out.block(ge[e], 0, 0, Fm);
-                out.block(ue[e], 0, 0, Fm);
+            for (uint64_t e = e_first; e < e_first + E_loc; ++e) {
+                out.block(ge[e], mt * Fs, 0, Fs);
+                out.block(ue[e], mt * Fs, 0, Fs);
             }
-            out.begin(name("w2"), Fm);
-            for (uint64_t e = 0; e < E; ++e) out.block(de[e], 0, 0, H);
+            out.begin(name("w2"), Fs);
+            for (uint64_t e = e_first; e < e_first + E_loc; ++e) out.block(de[e], 0, mt * Fs, H);
         }
     }
     Param final_norm = flat.take(1, H);
@@ -276,7 +296,8 @@ int compile_plan(dr_plan* p)
     } else {
         Param lm_head = flat.take(V, H);
         out.begin("lm_head", H);
-        out.block(lm_head, t * (V / T), 0, V / T);
+        out.block(lm_head, v_lo, 0, v_real);
+        out.pad_rows(Vp / T);
     }
 
     const uint64_t N = flat.next, W = p->src.world, S = (N + W - 1) / W;

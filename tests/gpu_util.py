@@ -41,10 +41,11 @@ def make_source(n: int, seed: int, with_specials: bool = True) -> np.ndarray:
 
 
 def forward_both(spec, *, world=1, rank=0, gathered=True, align=1, tp=1, tp_rank=0, dtype=dr.DR_BF16,
-                 arena_align=256, src=None, seed=1, arena_init=None, misalign=0):
+                 arena_align=256, src=None, seed=1, arena_init=None, misalign=0, **opts):
     """Returns (gpu arena bytes, oracle arena bytes, plan, oracle model, src) for one forward call."""
     es = 2 if dtype == dr.DR_BF16 else 4
-    om = oracle.Model(spec, align=align, world=world, tp=tp, tp_rank=tp_rank, elem_size=es, arena_align=arena_align)
+    om = oracle.Model(spec, align=align, world=world, tp=tp, tp_rank=tp_rank, elem_size=es, arena_align=arena_align,
+                      **opts)
     n_src = world * om.shard_elems if gathered else om.shard_elems
     if src is None:
         src = make_source(world * om.shard_elems, seed)
@@ -53,7 +54,7 @@ def forward_both(spec, *, world=1, rank=0, gathered=True, align=1, tp=1, tp_rank
     want = np.full(om.arena_bytes, SENT8, dtype=np.uint8) if arena_init is None else arena_init[0].copy()
     om.forward(local, want, gathered=gathered, rank=rank)
     plan = dr.Plan(spec, world=world, rank=rank, gathered=gathered, align_elems=align, tp=tp, tp_rank=tp_rank,
-                   dtype=dtype, arena_align_bytes=arena_align)
+                   dtype=dtype, arena_align_bytes=arena_align, **opts)
     assert plan.info.dst_bytes == om.arena_bytes and plan.info.src_bytes == 4 * n_src
     # misalign > 0 shifts both device buffers by that many bytes (a multiple of 16) off their 256-byte
     # allocation boundary, which forces the 128-bit access path

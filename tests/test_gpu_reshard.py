@@ -166,3 +166,32 @@ def test_device_generator_equals_host_generator():
     h = torch.empty(n, dtype=torch.int16, device=dev())
     synth.cuda_fill_bf16(h, 99, synth.BUF_ROLLOUT, start=5)
     assert np.array_equal(h.cpu().numpy().view(np.uint16), synth.fill_bf16(99, synth.BUF_ROLLOUT, 5, n))
+
+
+VARIANTS = [
+    (dict(BRUTE[0]["spec"], ffn=12), 4, dict(kv_replicate=True, vocab_pad=8)),
+    (MID[0]["spec"], 16, dict(kv_replicate=True)),
+    (dict(MID[1]["spec"], tied=0), 2, dict(vocab_pad=1024)),
+    (BRUTE[2]["spec"], 2, dict(moe_tp=2)),
+    (MID[2]["spec"], 4, dict(moe_tp=4, moe_ep=2, moe_ep_rank=0, vocab_pad=64)),
+    (MID[2]["spec"], 8, dict(kv_replicate=True, moe_ep=4, moe_ep_rank=3)),
+]
+
+
+@pytest.mark.parametrize("spec,T,opts", VARIANTS, ids=[f"v{i}" for i in range(len(VARIANTS))])
+def test_layout_variants_forward_and_inverse_match_oracle(spec, T, opts):
+    """KV-head replication, vocabulary padding, expert tensor / expert parallelism: forward into a
+    sentinel-filled arena (padding rows must keep the sentinel), then the inverse of that arena."""
+    for t in sorted({0, T // 2, T - 1}):
+        for (W, g) in ((1, True), (3, False)):
+            r = W - 1
+            got, want, plan, om, src = forward_both(spec, world=W, rank=r, gathered=g, tp=T, tp_rank=t, seed=40 + t, **opts)
+            assert first_diff(got, want) is None
+            n = W * om.shard_elems if g else om.shard_elems
+            wflat = np.full(n, 0xDEADBEEF, dtype=np.uint32)
+            om.inverse(want, wflat, gathered=g, rank=r)
+            flat = torch.full((n,), 0xDEADBEEF - (1 << 32), dtype=torch.int32, device=dev())
+            plan.reshard_inverse(torch.from_numpy(got).to(dev()), flat)
+            torch.cuda.synchronize()
+            assert first_diff(flat.cpu().numpy().view(np.uint32), wflat) is None
+            plan.close()

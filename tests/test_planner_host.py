@@ -123,7 +123,7 @@ def test_library_exports_every_declared_symbol():
 
 
 def test_struct_sizes_match_the_header_layout():
-    assert C.sizeof(dr.dr_model_spec) == 48 and C.sizeof(dr.dr_src_layout) == 28 and C.sizeof(dr.dr_dst_layout) == 20
+    assert C.sizeof(dr.dr_model_spec) == 48 and C.sizeof(dr.dr_src_layout) == 28 and C.sizeof(dr.dr_dst_layout) == 36
     assert C.sizeof(dr.dr_stage_desc) == 432 and C.sizeof(dr.dr_stage_stats) == 112 and C.sizeof(dr.dr_plan_info) == 80 and C.sizeof(dr.dr_tensor_desc) == 96 and C.sizeof(dr.dr_segment_desc) == 56
 
 
@@ -168,3 +168,46 @@ def test_shard_range():
     for n, w in ((1_975_808, 2), (14_768_307_200, 4), (17, 3)):
         ends = [dr.dr_shard_range(n, w, r)[1:3] for r in range(w)]
         assert ends[0][0] == 0 and ends[-1][1] == n and all(a[1] == b[0] for a, b in zip(ends, ends[1:]))
+
+
+VARIANTS = [
+    (dict(BRUTE[0]["spec"], ffn=12), 4, dict(kv_replicate=True, vocab_pad=8)),
+    (MID[0]["spec"], 16, dict(kv_replicate=True)),
+    (MID[1]["spec"], 4, dict(vocab_pad=64)),
+    (dict(MID[1]["spec"], tied=0), 2, dict(vocab_pad=1024)),
+    (BRUTE[2]["spec"], 2, dict(moe_tp=2)),
+    (BRUTE[2]["spec"], 2, dict(moe_ep=2, moe_ep_rank=1)),
+    (MID[2]["spec"], 4, dict(moe_tp=4, moe_ep=2, moe_ep_rank=0, vocab_pad=64)),
+    (MID[2]["spec"], 8, dict(kv_replicate=True, moe_ep=4, moe_ep_rank=3)),
+]
+
+
+@pytest.mark.parametrize("spec,T,opts", VARIANTS, ids=[f"v{i}" for i in range(len(VARIANTS))])
+@pytest.mark.parametrize("W,gathered", [(1, True), (3, False)])
+def test_layout_variants_segment_table_is_the_oracle_map(spec, T, opts, W, gathered):
+    for t in sorted({0, 1, T - 1}):
+        r = W - 1
+        p = dr.Plan(spec, world=W, rank=r, gathered=gathered, tp=T, tp_rank=t, arena_align_bytes=64, host_only=True, **opts)
+        om = oracle.Model(spec, world=W, tp=T, tp_rank=t, arena_align=64, **opts)
+        assert p.info.dst_bytes == om.arena_bytes
+        assert np.array_equal(expand(p, 2), oracle_map(om, 2, gathered, r))
+        for a, b in zip(p.tensors(), om.dst_tensors()):
+            assert (a.name.decode(), a.arena_off, a.rows, a.cols, a.alias_of) == (b.name, b.arena_off, b.rows, b.cols, b.alias_of)
+        p.close()
+
+
+def test_layout_variant_errors():
+    E = dr.binding
+    for kw, tp, want in ((dict(), 4, E.DR_ERR_UNSUPPORTED), (dict(kv_replicate=True), 3, E.DR_ERR_UNSUPPORTED)):
+        with pytest.raises(dr.DrError) as e:
+            dr.Plan(MID[0]["spec"] if tp == 3 else dict(BRUTE[0]["spec"], ffn=12), tp=tp, host_only=True, **kw)
+        assert e.value.status == want
+    with pytest.raises(dr.DrError) as e:
+        dr.Plan(BRUTE[2]["spec"], tp=2, moe_ep=3, host_only=True)
+    assert e.value.status == E.DR_ERR_UNSUPPORTED
+    with pytest.raises(dr.DrError) as e:
+        dr.Plan(BRUTE[2]["spec"], tp=2, moe_ep=2, moe_ep_rank=2, host_only=True)
+    assert e.value.status == E.DR_ERR_INVALID
+    with pytest.raises(dr.DrError) as e:
+        dr.Plan(MID[2]["spec"], tp=4, moe_tp=2, host_only=True)
+    assert e.value.status == E.DR_ERR_UNSUPPORTED
