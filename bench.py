@@ -513,7 +513,7 @@ def staging_sections(args, cfg, plan, master, arena, seed, base, dev, world, lin
 
     # re-shard across a changed training world size (Sec. 3.3): the image above is the flat state; a new rank 1 of a
     # world of 4 stages its own range of master, m, v in (weights first), then the old cut is put back
-    if len(bufs) == 3 and not cfg["gathered"] is False:
+    if len(bufs) == 3 and cfg["gathered"]:
         rc, lo, hi, s4 = dr.dr_shard_range(n, 4, 1)
         d4 = dr.stage_desc(ptrs, [4 * (hi - lo)] * 3, budget=budget, host_arena=image.data_ptr(),
                            host_arena_bytes=image.numel(), host_offsets=[4 * (k * n + lo) for k in range(3)], order=[0, 1, 2])
