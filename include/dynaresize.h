@@ -280,6 +280,46 @@ int dr_stage_out(dr_plan* plan, const dr_stage_desc* desc, dr_stage_stats* stats
 int dr_stage_in(dr_plan* plan, const dr_stage_desc* desc, dr_stage_stats* stats);
 
 /*
+ * Streamed repack: Training -> Rollout for a GPU that does not hold the fp32 master.  The flat source
+ * rests in pinned host memory (where dr_stage_out left it); it is copied to the device chunk by chunk
+ * into a caller-provided window of a few chunks, each chunk is repacked as soon as it has arrived, and
+ * (optionally) every range of the rollout arena is copied back to pinned host memory as soon as no later
+ * chunk can write into it.  Host-to-device copies, the repack kernels and device-to-host copies run on
+ * three streams and overlap, so the whole switch takes about as long as the larger of the two copy
+ * directions; the device never holds more than the window of fp32 state (the bounded staging of Sec. 3.3
+ * applied to the device side, with the "asynchronous overlapping of independent operations" of Sec. 3.3).
+ */
+typedef struct dr_stream_desc {
+    uint32_t struct_size, flags;  /* sizeof(dr_stream_desc), 0                                         */
+    const void* host_src;         /* pinned host: the plan's source buffer (dr_plan_query: src_bytes)  */
+    uint64_t host_src_bytes;
+    void* dst_dev;                /* device: the rollout arena                                         */
+    uint64_t dst_bytes;
+    void* host_dst;               /* pinned host copy of the arena, or NULL                            */
+    uint64_t host_dst_bytes;
+    void* window_dev;             /* device scratch the caller owns: slots = floor(window / chunk) >= 2 */
+    uint64_t window_bytes;
+    uint64_t chunk_bytes;         /* multiple of 32; 0: window_bytes / 2 rounded down to 4096          */
+    uint32_t timeout_ms;          /* bound on the final wait; 0 = 60 000                               */
+    uint32_t pad;
+} dr_stream_desc;
+
+typedef struct dr_stream_stats {
+    uint64_t h2d_bytes, d2h_bytes, n_chunks, kernels;
+    double elapsed_ms;            /* first enqueue to everything complete                              */
+} dr_stream_stats;
+
+/*
+ * dr_reshard_stream -- the result in dst_dev (and host_dst) is exactly dr_reshard's on the same source.
+ * Blocking: returns when every copy and kernel has completed (bounded poll, DR_ERR_TIMEOUT).  The first
+ * call with a given chunk size compiles and uploads one small segment table per chunk (device memory
+ * owned by the plan, re-used by later calls).  Errors: DR_ERR_INVALID, DR_ERR_SIZE (a buffer too small),
+ * DR_ERR_ALIGN (pointers not 32-byte aligned), DR_ERR_BUDGET (window below two chunks), DR_ERR_STATE
+ * (host-only plan), DR_ERR_NOMEM, DR_ERR_CUDA, DR_ERR_TIMEOUT.  Calls on one plan must not overlap.
+ */
+int dr_reshard_stream(dr_plan* plan, const dr_stream_desc* desc, dr_stream_stats* stats);
+
+/*
  * dr_shard_range -- the flat elements [*begin, *end) that rank `rank` of `world` really holds
  * (S = ceil(flat_elems / world) per rank; the last ranks' padding past flat_elems is excluded, so
  * *end - *begin can be smaller than S, or zero).  With it a caller lays out a re-shard across a changed

@@ -18,7 +18,7 @@ DR_MAX_STAGE_BUFS = 8
 DR_STAGE_HOST_OFFSETS = 1
 
 EXPORTS = ["dr_plan_create", "dr_plan_create_host", "dr_plan_query", "dr_plan_tensor", "dr_plan_segment",
-           "dr_reshard", "dr_reshard_inverse", "dr_reshard_static", "dr_shard_range", "dr_stage_out", "dr_stage_in", "dr_plan_destroy", "dr_strerror",
+           "dr_reshard", "dr_reshard_inverse", "dr_reshard_static", "dr_reshard_stream", "dr_shard_range", "dr_stage_out", "dr_stage_in", "dr_plan_destroy", "dr_strerror",
            "dr_last_error"]
 
 u8, u32, u64, i64, vp = C.c_uint8, C.c_uint32, C.c_uint64, C.c_int64, C.c_void_p
@@ -70,6 +70,16 @@ class dr_stage_stats(C.Structure):
                 ("link_gbs", C.c_double), ("pinned_high_water_bytes", u64), ("ready_ms", C.c_double * 8)]
 
 
+class dr_stream_desc(C.Structure):
+    _fields_ = [("struct_size", u32), ("flags", u32), ("host_src", vp), ("host_src_bytes", u64), ("dst_dev", vp),
+                ("dst_bytes", u64), ("host_dst", vp), ("host_dst_bytes", u64), ("window_dev", vp), ("window_bytes", u64),
+                ("chunk_bytes", u64), ("timeout_ms", u32), ("pad", u32)]
+
+
+class dr_stream_stats(C.Structure):
+    _fields_ = [("h2d_bytes", u64), ("d2h_bytes", u64), ("n_chunks", u64), ("kernels", u64), ("elapsed_ms", C.c_double)]
+
+
 class DrError(RuntimeError):
     def __init__(self, status: int, where: str):
         self.status = status
@@ -98,6 +108,7 @@ def lib() -> C.CDLL:
         L.dr_reshard_static.argtypes = [vp, vp, u64, vp, u64, vp]
         L.dr_stage_out.argtypes = [vp, P(dr_stage_desc), P(dr_stage_stats)]
         L.dr_stage_in.argtypes = [vp, P(dr_stage_desc), P(dr_stage_stats)]
+        L.dr_reshard_stream.argtypes = [vp, P(dr_stream_desc), P(dr_stream_stats)]
         L.dr_plan_destroy.argtypes = [vp]
         L.dr_shard_range.argtypes = [u64, u32, u32, P(u64), P(u64), P(u64)]
         for n in EXPORTS:
@@ -211,6 +222,18 @@ def dr_stage_in(plan, desc):
     return lib().dr_stage_in(plan, C.byref(desc), C.byref(st)), st
 
 
+def stream_desc(host_src, host_src_bytes, dst_dev, dst_bytes, window_dev, window_bytes, chunk_bytes=0, host_dst=None,
+                host_dst_bytes=0, timeout_ms=0) -> dr_stream_desc:
+    return dr_stream_desc(struct_size=C.sizeof(dr_stream_desc), host_src=host_src, host_src_bytes=host_src_bytes,
+                          dst_dev=dst_dev, dst_bytes=dst_bytes, host_dst=host_dst, host_dst_bytes=host_dst_bytes,
+                          window_dev=window_dev, window_bytes=window_bytes, chunk_bytes=chunk_bytes, timeout_ms=timeout_ms)
+
+
+def dr_reshard_stream(plan, desc):
+    st = dr_stream_stats()
+    return lib().dr_reshard_stream(plan, C.byref(desc), C.byref(st)), st
+
+
 def dr_shard_range(flat_elems, world, rank):
     b, e, s = u64(), u64(), u64()
     rc = lib().dr_shard_range(flat_elems, world, rank, C.byref(b), C.byref(e), C.byref(s))
@@ -291,6 +314,12 @@ class Plan:
                                 flat.data_ptr(), flat.numel() * flat.element_size(), self._stream(stream))
         if rc:
             raise DrError(rc, "dr_reshard_inverse")
+
+    def reshard_stream(self, desc):
+        rc, st = dr_reshard_stream(self.handle, desc)
+        if rc:
+            raise DrError(rc, "dr_reshard_stream")
+        return st
 
     def stage_out(self, desc):
         rc, st = dr_stage_out(self.handle, desc)

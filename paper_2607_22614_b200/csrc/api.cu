@@ -248,6 +248,7 @@ int dr_shard_range(uint64_t flat_elems, uint32_t world, uint32_t rank, uint64_t*
 int dr_plan_destroy(dr_plan* plan)
 {
     if (!plan) return DR_OK;
+    if (plan->stream) stream_destroy(plan->stream);
     if (plan->ring) ring_destroy(plan->ring);
     if (plan->d_segs) cudaFree(plan->d_segs);
     if (plan->d_hints) cudaFree(plan->d_hints);

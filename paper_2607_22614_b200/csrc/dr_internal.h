@@ -54,7 +54,16 @@ struct Tensor {
     int64_t alias_of = -1;
 };
 
-struct Ring;  // pinned staging ring + worker pool (staging.cu)
+// Everything a launch needs besides the buffers.
+struct Tables {
+    std::vector<DevSeg> segs;
+    std::vector<uint32_t> hints;
+    uint32_t hint_shift = 0;
+    uint64_t n_tiles = 0, elems = 0;
+};
+
+struct Ring;    // pinned staging ring + worker pool (staging.cu)
+struct Stream;  // per-chunk tables of a streamed repack (stream.cu)
 
 }  // namespace dr
 
@@ -80,6 +89,7 @@ struct dr_plan {
     // staging
     std::mutex stage_mu;
     dr::Ring* ring = nullptr;
+    dr::Stream* stream = nullptr;
 };
 
 namespace dr {
@@ -90,5 +100,11 @@ int launch_reshard(const dr_plan* p, bool inverse, const void* flat, void* arena
                    void* stream);
 int choose_grid(int device, uint32_t elem_size);  // resident CTAs of the reshard kernel on the whole GPU
 void ring_destroy(Ring* r);
+void stream_destroy(Stream* s);
+int build_tables(const std::vector<HostSeg>& segs, Tables* out);
+std::vector<HostSeg> window_segments(const std::vector<HostSeg>& segs, uint64_t lo, uint64_t hi, uint32_t es);
+// Enqueue the forward kernel for an explicit table (used by the streamed repack).
+int launch_forward_tables(uint32_t elem_size, const DevSeg* d_segs, uint32_t n_segs, const uint32_t* d_hints,
+                          uint32_t hint_shift, uint64_t n_tiles, const void* flat, void* arena, void* stream);
 
 }  // namespace dr

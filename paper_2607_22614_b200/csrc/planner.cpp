@@ -197,6 +197,62 @@ void classify(std::vector<HostSeg>& v, uint32_t es)
 
 }  // namespace
 
+// Device table, tile prefix and hint table for a list of classified segments.
+int build_tables(const std::vector<HostSeg>& segs, Tables* out)
+{
+    uint64_t tiles = 0, moved = 0;
+    out->segs.clear();
+    out->segs.reserve(segs.size());
+    for (const HostSeg& g : segs) {
+        DevSeg d{};
+        d.dst_off = g.dst_off;
+        d.src_off = g.src_off;
+        d.tile0 = tiles;
+        d.units_per_row = (uint32_t)((g.row_len + kUnitElems - 1) / kUnitElems);
+        uint64_t units = g.rows * d.units_per_row;
+        if (units > 0xFFFFFFFFull || g.src_stride > 0xFFFFFFFFull || g.dst_stride > 0xFFFFFFFFull) {
+            set_error("segment too large for the 32-bit unit index");
+            return DR_ERR_UNSUPPORTED;
+        }
+        d.n_units = (uint32_t)units;
+        d.row_len = (uint32_t)g.row_len;
+        d.src_stride = (uint32_t)g.src_stride;
+        d.dst_stride = (uint32_t)g.dst_stride;
+        d.flags = g.flags;
+        out->segs.push_back(d);
+        tiles += (units + kTileUnits - 1) / kTileUnits;
+        moved += g.rows * g.row_len;
+    }
+    // hint table: segment of every (1 << hint_shift)-th tile
+    out->hint_shift = 0;
+    while (((tiles + (1ull << out->hint_shift) - 1) >> out->hint_shift) > kMaxHints) ++out->hint_shift;
+    const uint64_t n_hints = (tiles + (1ull << out->hint_shift) - 1) >> out->hint_shift;
+    out->hints.assign(n_hints ? n_hints : 1, 0);
+    uint32_t si = 0;
+    for (uint64_t h = 0; h < n_hints; ++h) {
+        const uint64_t tile = h << out->hint_shift;
+        while (si + 1 < out->segs.size() && out->segs[si + 1].tile0 <= tile) ++si;
+        out->hints[h] = si;
+    }
+    out->n_tiles = tiles;
+    out->elems = moved;
+    return DR_OK;
+}
+
+// The part of a plan whose source elements lie in [lo, hi), with sources rebased to lo: what one chunk of
+// a streamed source can produce on its own.
+std::vector<HostSeg> window_segments(const std::vector<HostSeg>& segs, uint64_t lo, uint64_t hi, uint32_t es)
+{
+    std::vector<HostSeg> v;
+    for (const HostSeg& g : segs) {  // cheap reject before the exact clip
+        uint64_t a = g.src_off, b = g.src_off + (g.rows - 1) * g.src_stride + g.row_len;
+        if (b > lo && a < hi) v.push_back(g);
+    }
+    clip_to_shard(v, lo, hi, es);
+    classify(v, es);
+    return v;
+}
+
 int compile_plan(dr_plan* p)
 {
     const dr_model_spec& s = p->spec;
@@ -305,43 +361,13 @@ int compile_plan(dr_plan* p)
     if (!p->src.gathered) clip_to_shard(p->segs, (uint64_t)p->src.rank * S, (uint64_t)(p->src.rank + 1) * S, es);
     classify(p->segs, es);
 
-    // device table + tile prefix
-    uint64_t tiles = 0, moved = 0;
-    p->dev_segs.reserve(p->segs.size());
-    for (const HostSeg& g : p->segs) {
-        DevSeg d{};
-        d.dst_off = g.dst_off;
-        d.src_off = g.src_off;
-        d.tile0 = tiles;
-        d.units_per_row = (uint32_t)((g.row_len + kUnitElems - 1) / kUnitElems);
-        uint64_t units = g.rows * d.units_per_row;
-        if (units > 0xFFFFFFFFull || g.src_stride > 0xFFFFFFFFull || g.dst_stride > 0xFFFFFFFFull) {
-            set_error("segment too large for the 32-bit unit index");
-            return DR_ERR_UNSUPPORTED;
-        }
-        d.n_units = (uint32_t)units;
-        d.row_len = (uint32_t)g.row_len;
-        d.src_stride = (uint32_t)g.src_stride;
-        d.dst_stride = (uint32_t)g.dst_stride;
-        d.flags = g.flags;
-        p->dev_segs.push_back(d);
-        tiles += (units + kTileUnits - 1) / kTileUnits;
-        moved += g.rows * g.row_len;
-    }
-
-    // hint table: segment of every (1 << hint_shift)-th tile
-    p->hint_shift = 0;
-    while (((tiles + (1ull << p->hint_shift) - 1) >> p->hint_shift) > kMaxHints) ++p->hint_shift;
-    {
-        const uint64_t n_hints = (tiles + (1ull << p->hint_shift) - 1) >> p->hint_shift;
-        p->hints.resize(n_hints ? n_hints : 1, 0);
-        uint32_t si = 0;
-        for (uint64_t h = 0; h < n_hints; ++h) {
-            const uint64_t tile = h << p->hint_shift;
-            while (si + 1 < p->dev_segs.size() && p->dev_segs[si + 1].tile0 <= tile) ++si;
-            p->hints[h] = si;
-        }
-    }
+    Tables tb;
+    int trc = build_tables(p->segs, &tb);
+    if (trc) return trc;
+    p->dev_segs.swap(tb.segs);
+    p->hints.swap(tb.hints);
+    p->hint_shift = tb.hint_shift;
+    const uint64_t tiles = tb.n_tiles, moved = tb.elems;
 
     dr_plan_info& I = p->info;
     I.flat_elems = N;

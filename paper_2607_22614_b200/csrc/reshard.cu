@@ -331,6 +331,28 @@ int launch_reshard(const dr_plan* p, bool inverse, const void* flat, void* arena
     return DR_OK;
 }
 
+int launch_forward_tables(uint32_t elem_size, const DevSeg* d_segs, uint32_t n_segs, const uint32_t* d_hints,
+                          uint32_t hint_shift, uint64_t n_tiles, const void* flat, void* arena, void* stream)
+{
+    if (n_tiles == 0) return DR_OK;
+    char* f = (char*)flat;
+    char* a = (char*)arena;
+    const int allow256 = (((uintptr_t)f | (uintptr_t)a) & 31) == 0;
+    const uint64_t want = (n_tiles + DR_TILES_PER_CTA - 1) / DR_TILES_PER_CTA;
+    dim3 grid((unsigned)want), block(kThreads);
+    cudaStream_t s = (cudaStream_t)stream;
+    if (elem_size == 2)
+        reshard_kernel<2, false, DR_BLOCKED><<<grid, block, 0, s>>>(d_segs, n_segs, d_hints, hint_shift, n_tiles, f, a, allow256);
+    else
+        reshard_kernel<4, false, DR_BLOCKED><<<grid, block, 0, s>>>(d_segs, n_segs, d_hints, hint_shift, n_tiles, f, a, allow256);
+    cudaError_t e = cudaGetLastError();
+    if (e != cudaSuccess) {
+        set_error("reshard kernel launch: %s", cudaGetErrorString(e));
+        return DR_ERR_CUDA;
+    }
+    return DR_OK;
+}
+
 }  // namespace dr
 
 // ------------------------------------------------------------------------------------------------
