@@ -29,7 +29,7 @@ if ROOT not in sys.path:
 METRIC = "role-switch transform GB/s (% of HBM peak); stage-out/in GB/s; switch ms"
 GiB = 1 << 30
 # DRAM bytes per element (dram__bytes_read.sum + dram__bytes_write.sum over elements moved) of the forward
-# kernel, from the ncu capture summarised in profiles/reshard_kernel_qwen3-8b.md (a 654 M-element case of the
+# kernel, from the committed ncu capture summary of this kernel (a 654 M-element case of the
 # same kernel; traffic grows in proportion to the elements, so it is scaled to the launch timed here).
 NCU_DRAM_BYTES_PER_ELEMENT_FWD = 5.947
 
@@ -375,7 +375,17 @@ def main():
         line["inverse"] = {"gbs_avg": bytes_inv / ia / 1e6, "gbs_best": bytes_inv / min(inv_ms) / 1e6, "ms_avg": ia,
                            "ms_best": min(inv_ms), "frac_of_measured_peak": bytes_inv / ia / 1e6 / peak}
     line["roofline"]["traffic"] = NCU_DRAM_BYTES_PER_ELEMENT_FWD * (bytes_fwd // 6 // len(plans)) if cfg["spec"] else None
-    line["roofline"]["traffic_source"] = "ncu capture of a 654 M-element case, scaled by elements (profiles/reshard_kernel_qwen3-8b.md)"
+    line["roofline"]["traffic_source"] = "ncu capture of a 654 M-element case of the same kernel, scaled by elements"
+
+    # where the arena is the flat buffer cast in place (TP = 1, dense packing), check the timed output against
+    # torch's own float32 -> bfloat16 on two 64 Mi-element windows
+    if halves == 1 and info.dst_bytes == 2 * n_src and not inverse_dir:
+        plans[0].reshard(master, arena)
+        w = min(n_src, 1 << 26)
+        ok = True
+        for lo in (0, n_src - w):
+            ok &= torch.equal(arena.view(torch.bfloat16)[lo:lo + w], master.view(torch.float32)[lo:lo + w].to(torch.bfloat16))
+        line["config"]["output_equals_torch_cast_on_windows"] = bool(ok)
 
     del flat_back
     torch.cuda.empty_cache()
