@@ -21,7 +21,9 @@ _SRC = os.path.join(_DIR, "dr_oracle.c")
 
 def build(force: bool = False) -> None:
     if force or not os.path.exists(_SO) or os.path.getmtime(_SRC) > os.path.getmtime(_SO):
-        subprocess.check_call(["gcc", "-O2", "-std=c99", "-Wall", "-shared", "-fPIC", "-o", _SO, _SRC])
+        # -ffp-contract=off, no fast-math: fp32 divisions must round exactly once, as written
+        subprocess.check_call(["gcc", "-O2", "-std=c99", "-Wall", "-ffp-contract=off", "-shared", "-fPIC", "-o", _SO, _SRC,
+                               "-lm"])
 
 
 class _Spec(ctypes.Structure):
@@ -74,6 +76,14 @@ def _l():
         lib.orc_stage_out.argtypes = [p, p, u64, u64, u64, u64, p, p]
         lib.orc_stage_in.restype = i64
         lib.orc_stage_in.argtypes = [p, p, u64, p, u64, u64, p, p]
+        lib.orc_cast_e4m3.restype = ctypes.c_uint8
+        lib.orc_cast_e4m3.argtypes = [ctypes.c_uint32]
+        lib.orc_e4m3_value.restype = ctypes.c_float
+        lib.orc_e4m3_value.argtypes = [ctypes.c_uint8]
+        lib.orc_fp8_layout.restype = u64
+        lib.orc_fp8_layout.argtypes = [p, u64, ctypes.POINTER(ctypes.c_int), ctypes.POINTER(u64), ctypes.POINTER(u64)]
+        lib.orc_forward_fp8.restype = ctypes.c_int
+        lib.orc_forward_fp8.argtypes = [p, p, p, i64]
         lib.orc_restage_out.restype = None
         lib.orc_restage_out.argtypes = [p, u64, u64, u64, p]
         lib.orc_restage_in.restype = None
@@ -85,6 +95,15 @@ def _l():
 def cast_bf16(u: int) -> int:
     """D5 on one fp32 bit pattern."""
     return int(_l().orc_cast_bf16(u & 0xFFFFFFFF))
+
+
+def cast_e4m3(u: int) -> int:
+    """D7's fp32 -> e4m3 conversion on one bit pattern."""
+    return int(_l().orc_cast_e4m3(u & 0xFFFFFFFF))
+
+
+def e4m3_value(c: int) -> float:
+    return float(_l().orc_e4m3_value(c & 0xFF))
 
 
 def widen_bf16(b: int) -> int:
@@ -173,6 +192,21 @@ class Model:
         need = self.world * self.shard_elems if gathered else self.shard_elems
         assert src_u32.size >= min(need, self.flat_elems if gathered else need)
         _l().orc_forward(self._h, src_u32.ctypes.data, int(gathered), rank, arena_u8.ctypes.data, only)
+
+    def fp8_layout(self):
+        """(arena bytes, [(quantised, payload offset, scale offset)] per rollout tensor) of the fp8 arena (D7)."""
+        out = []
+        q, o, so = ctypes.c_int(), ctypes.c_uint64(), ctypes.c_uint64()
+        total = 0
+        for i in range(self.n_dst):
+            total = int(_l().orc_fp8_layout(self._h, i, ctypes.byref(q), ctypes.byref(o), ctypes.byref(so)))
+            out.append((bool(q.value), o.value, so.value))
+        return total, out
+
+    def forward_fp8(self, src_u32: np.ndarray, arena_u8: np.ndarray, only: int = -1) -> None:
+        assert src_u32.dtype == np.uint32 and src_u32.flags.c_contiguous and src_u32.size >= self.flat_elems
+        assert arena_u8.dtype == np.uint8 and arena_u8.size >= self.fp8_layout()[0]
+        _l().orc_forward_fp8(self._h, src_u32.ctypes.data, arena_u8.ctypes.data, only)
 
     def inverse(self, arena_u8: np.ndarray, flat_u32: np.ndarray, *, gathered: bool = True, rank: int = 0) -> None:
         assert flat_u32.dtype == np.uint32 and flat_u32.flags.c_contiguous

@@ -23,6 +23,7 @@
  * source with world W, rank r, per-parameter alignment A; rollout layout at
  * tensor-parallel degree T, rank t.  All matrices are [out, in] row-major.
  */
+#include <math.h>
 #include <stdint.h>
 #include <stdio.h>
 #include <stdlib.h>
@@ -627,4 +628,177 @@ void orc_restage_in(const uint32_t *image, uint64_t N, uint64_t W_new, uint64_t 
         uint64_t f = q * S + i;
         new_shard[i] = f < N ? image[f] : 0u;
     }
+}
+
+/* ---- D7: fp8 (e4m3) rollout weights with one fp32 scale per 128 x 128 block ----------------------
+ * A reading for rollout engines that serve block-quantised weights (the paper is silent).  The linear
+ * weights (qkv, o, gate_up, down, w13, w2) are quantised; embeddings, lm_head, router and norms stay
+ * bf16.  For a quantised rollout tensor X[rows, cols]:
+ *   block (bi, bj) = rows [128 bi, 128 bi + 128) x cols [128 bj, 128 bj + 128), clipped to the tensor;
+ *   amax  = max |x| over the block, NaNs skipped, starting from 0;
+ *   scale = amax / 448 in fp32 (round to nearest); a zero quotient is replaced by 1;
+ *   q     = e4m3( x / scale ), fp32 division (round to nearest), then round to nearest even onto the
+ *           e4m3 grid (3 mantissa bits, bias 7, subnormal step 2^-9), magnitudes above 448 saturate to
+ *           448 (code 0x7E), NaN becomes 0x7F.
+ * Arena: payload rows*cols bytes at arena_off, then the scales [ceil(rows/128), ceil(cols/128)] fp32,
+ * row-major, at the next multiple of arena_align.
+ */
+uint8_t orc_cast_e4m3(uint32_t u)
+{
+    uint32_t sign = (u >> 31) << 7, mag = u & 0x7FFFFFFFu;
+    float a;
+    double q, quantum;
+    int e;
+    if (mag > 0x7F800000u) return 0x7F;
+    memcpy(&a, &mag, 4);
+    if (a > 448.0f) return (uint8_t)(sign | 0x7E);
+    if (a == 0.0f) return (uint8_t)sign;
+    e = (int)floor(log2((double)a));        /* exact for powers of two in double; a is fp32 */
+    if (ldexp(1.0, e) > (double)a) e--;     /* guard against log2 rounding up */
+    if (ldexp(1.0, e + 1) <= (double)a) e++;
+    quantum = e < -6 ? ldexp(1.0, -9) : ldexp(1.0, e - 3);
+    q = nearbyint((double)a / quantum);     /* exact quotient; default rounding mode: ties to even */
+    {
+        double v = q * quantum;
+        int ev, m;
+        if (v == 0.0) return (uint8_t)sign;
+        if (v < ldexp(1.0, -6)) return (uint8_t)(sign | (uint32_t)q); /* subnormal: mantissa 1..7 */
+        ev = (int)floor(log2(v));
+        if (ldexp(1.0, ev) > v) ev--;
+        if (ldexp(1.0, ev + 1) <= v) ev++;
+        m = (int)(v / ldexp(1.0, ev - 3)) - 8;
+        return (uint8_t)(sign | (uint32_t)((ev + 7) << 3) | (uint32_t)m);
+    }
+}
+
+/* exact value of an e4m3 code (NaN codes 0x7F / 0xFF decode as NaN) */
+float orc_e4m3_value(uint8_t c)
+{
+    int e = (c >> 3) & 15, m = c & 7;
+    double v;
+    if ((c & 0x7F) == 0x7F) return NAN;
+    v = e == 0 ? ldexp((double)m, -9) : ldexp(1.0 + m / 8.0, e - 7);
+    return (float)((c & 0x80) ? -v : v);
+}
+
+static int is_quantised(const char *name)
+{
+    const char *leaf = strrchr(name, '.');
+    leaf = leaf ? leaf + 1 : name;
+    return !strcmp(leaf, "qkv") || !strcmp(leaf, "o") || !strcmp(leaf, "gate_up") || !strcmp(leaf, "down") ||
+           !strcmp(leaf, "w13") || !strcmp(leaf, "w2");
+}
+
+/* Layout of the fp8 arena: for rollout tensor i, *quant tells whether it is quantised, *off where its
+ * payload starts, *scale_off where its scales start (quantised only).  Returns the arena size. */
+uint64_t orc_fp8_layout(const orc_model *m, uint64_t i, int *quant, uint64_t *off, uint64_t *scale_off)
+{
+    uint64_t k, pos = 0, my_off = 0, my_scale = 0;
+    int my_q = 0;
+    for (k = 0; k < m->n_dst; ++k) {
+        const orc_dst *d = &m->dst[k];
+        uint64_t o = 0, so = 0;
+        int qz = is_quantised(d->name);
+        if (d->alias_of < 0) {
+            pos = align_up(pos, m->arena_align);
+            o = pos;
+            if (qz) {
+                pos += d->rows * d->cols;
+                pos = align_up(pos, m->arena_align);
+                so = pos;
+                pos += ((d->rows + 127) / 128) * ((d->cols + 127) / 128) * 4;
+            } else {
+                pos += d->rows * d->cols * 2;
+            }
+        }
+        if (k == i) {
+            my_q = qz;
+            my_off = d->alias_of >= 0 ? 0 : o;
+            my_scale = so;
+        }
+    }
+    if (i < m->n_dst && m->dst[i].alias_of >= 0) {
+        int q2;
+        uint64_t o2, s2;
+        orc_fp8_layout(m, (uint64_t)m->dst[i].alias_of, &q2, &o2, &s2);
+        my_off = o2;
+    }
+    if (quant) *quant = my_q;
+    if (off) *off = my_off;
+    if (scale_off) *scale_off = my_scale;
+    return pos;
+}
+
+/* Forward into an fp8 arena: the whole flat buffer must be visible (a block cannot be scaled from part
+ * of its elements). */
+int orc_forward_fp8(const orc_model *m, const uint32_t *src, uint8_t *arena, int64_t only)
+{
+    uint64_t i, p, r, c;
+    for (i = 0; i < m->n_dst; ++i) {
+        const orc_dst *d = &m->dst[i];
+        int qz;
+        uint64_t off, soff;
+        if (only >= 0 && (uint64_t)only != i) continue;
+        if (d->alias_of >= 0) continue;
+        orc_fp8_layout(m, i, &qz, &off, &soff);
+        if (!qz) { /* bf16, as in the base definition */
+            for (p = 0; p < d->n_parts; ++p) {
+                const orc_part *q = &d->parts[p];
+                const orc_src *s = &m->src[q->src];
+                for (r = 0; r < q->rows; ++r)
+                    for (c = 0; c < d->cols; ++c) {
+                        uint64_t f = s->flat_off + (q->src_row0 + r) * s->cols + (q->src_col0 + c);
+                        uint16_t b = orc_cast_bf16(src[f]);
+                        memcpy(arena + off + ((q->dst_row0 + r) * d->cols + c) * 2, &b, 2);
+                    }
+            }
+            continue;
+        }
+        {
+            /* gather the rollout tensor as fp32 words, then quantise block by block */
+            uint32_t *x = (uint32_t *)malloc(d->rows * d->cols * 4);
+            uint8_t *has = (uint8_t *)calloc(d->rows, 1);
+            uint64_t bi, bj, nbr = (d->rows + 127) / 128, nbc = (d->cols + 127) / 128;
+            for (p = 0; p < d->n_parts; ++p) {
+                const orc_part *q = &d->parts[p];
+                const orc_src *s = &m->src[q->src];
+                for (r = 0; r < q->rows; ++r) {
+                    has[q->dst_row0 + r] = 1;
+                    for (c = 0; c < d->cols; ++c)
+                        x[(q->dst_row0 + r) * d->cols + c] =
+                            src[s->flat_off + (q->src_row0 + r) * s->cols + (q->src_col0 + c)];
+                }
+            }
+            for (bi = 0; bi < nbr; ++bi)
+                for (bj = 0; bj < nbc; ++bj) {
+                    uint64_t r1 = bi * 128 + 128 < d->rows ? bi * 128 + 128 : d->rows;
+                    uint64_t c1 = bj * 128 + 128 < d->cols ? bj * 128 + 128 : d->cols;
+                    float amax = 0.0f, scale;
+                    for (r = bi * 128; r < r1; ++r)
+                        for (c = bj * 128; c < c1; ++c) {
+                            uint32_t mag = x[r * d->cols + c] & 0x7FFFFFFFu;
+                            float a;
+                            if (!has[r] || mag > 0x7F800000u) continue;
+                            memcpy(&a, &mag, 4);
+                            if (a > amax) amax = a;
+                        }
+                    scale = amax / 448.0f;
+                    if (scale == 0.0f) scale = 1.0f;
+                    memcpy(arena + soff + (bi * nbc + bj) * 4, &scale, 4);
+                    for (r = bi * 128; r < r1; ++r)
+                        for (c = bj * 128; c < c1; ++c) {
+                            float v, qv;
+                            uint32_t qb;
+                            if (!has[r]) continue;
+                            memcpy(&v, &x[r * d->cols + c], 4);
+                            qv = v / scale;
+                            memcpy(&qb, &qv, 4);
+                            arena[off + r * d->cols + c] = orc_cast_e4m3(qb);
+                        }
+                }
+            free(x);
+            free(has);
+        }
+    }
+    return 0;
 }
