@@ -636,10 +636,14 @@ void orc_restage_in(const uint32_t *image, uint64_t N, uint64_t W_new, uint64_t 
  * bf16.  For a quantised rollout tensor X[rows, cols]:
  *   block (bi, bj) = rows [128 bi, 128 bi + 128) x cols [128 bj, 128 bj + 128), clipped to the tensor;
  *   amax  = max |x| over the block, NaNs skipped, starting from 0;
- *   scale = amax / 448 in fp32 (round to nearest); a zero quotient is replaced by 1;
- *   q     = e4m3( x / scale ), fp32 division (round to nearest), then round to nearest even onto the
- *           e4m3 grid (3 mantissa bits, bias 7, subnormal step 2^-9), magnitudes above 448 saturate to
- *           448 (code 0x7E), NaN becomes 0x7F.
+ *   scale = amax / 448 in fp32 (round to nearest), the number a consumer multiplies by to dequantise;
+ *   r     = 448 / amax in fp32 (round to nearest), the number the quantiser multiplies by;
+ *           an all-zero block (amax = 0) takes scale = r = 1;
+ *   q     = e4m3( x * r ), one fp32 multiplication (round to nearest), then round to nearest even onto
+ *           the e4m3 grid (3 mantissa bits, bias 7, subnormal step 2^-9), magnitudes above 448 saturate
+ *           to 448 (code 0x7E), NaN becomes 0x7F.
+ * (The multiply-by-reciprocal form is the one public block-quantisation references use; per element it
+ * costs one multiplication instead of a division.)
  * Arena: payload rows*cols bytes at arena_off, then the scales [ceil(rows/128), ceil(cols/128)] fp32,
  * row-major, at the next multiple of arena_align.
  */
@@ -773,7 +777,7 @@ int orc_forward_fp8(const orc_model *m, const uint32_t *src, uint8_t *arena, int
                 for (bj = 0; bj < nbc; ++bj) {
                     uint64_t r1 = bi * 128 + 128 < d->rows ? bi * 128 + 128 : d->rows;
                     uint64_t c1 = bj * 128 + 128 < d->cols ? bj * 128 + 128 : d->cols;
-                    float amax = 0.0f, scale;
+                    float amax = 0.0f, scale, recip;
                     for (r = bi * 128; r < r1; ++r)
                         for (c = bj * 128; c < c1; ++c) {
                             uint32_t mag = x[r * d->cols + c] & 0x7FFFFFFFu;
@@ -783,7 +787,8 @@ int orc_forward_fp8(const orc_model *m, const uint32_t *src, uint8_t *arena, int
                             if (a > amax) amax = a;
                         }
                     scale = amax / 448.0f;
-                    if (scale == 0.0f) scale = 1.0f;
+                    recip = 448.0f / amax;
+                    if (amax == 0.0f) scale = recip = 1.0f;
                     memcpy(arena + soff + (bi * nbc + bj) * 4, &scale, 4);
                     for (r = bi * 128; r < r1; ++r)
                         for (c = bj * 128; c < c1; ++c) {
@@ -791,7 +796,7 @@ int orc_forward_fp8(const orc_model *m, const uint32_t *src, uint8_t *arena, int
                             uint32_t qb;
                             if (!has[r]) continue;
                             memcpy(&v, &x[r * d->cols + c], 4);
-                            qv = v / scale;
+                            qv = v * recip;
                             memcpy(&qb, &qv, 4);
                             arena[off + r * d->cols + c] = orc_cast_e4m3(qb);
                         }

@@ -69,11 +69,13 @@ def _torch_block_quant(x):
     for bi in range(nbr):
         for bj in range(nbc):
             blk = x[bi * 128:(bi + 1) * 128, bj * 128:(bj + 1) * 128]
-            scale = blk.abs().amax() / torch.tensor(448.0, dtype=torch.float32)
-            if scale == 0:
-                scale = torch.tensor(1.0)
+            amax = blk.abs().amax()
+            scale = amax / torch.tensor(448.0, dtype=torch.float32)
+            recip = torch.tensor(448.0, dtype=torch.float32) / amax
+            if amax == 0:
+                scale = recip = torch.tensor(1.0)
             s[bi, bj] = scale
-            q[bi * 128:(bi + 1) * 128, bj * 128:(bj + 1) * 128] = (blk / scale).to(F8).view(torch.uint8)
+            q[bi * 128:(bi + 1) * 128, bj * 128:(bj + 1) * 128] = (blk * recip).to(F8).view(torch.uint8)
     return q, s
 
 
@@ -129,5 +131,5 @@ def test_zero_block_gets_unit_scale_and_nan_is_skipped_by_amax():
     for d, (qz, off, soff) in zip(m.dst_tensors(), lay):
         if qz:
             body = arena[off:off + d.rows * d.cols]
-            assert set(np.unique(body)) <= {0x7E, 0x7F}                  # 0.5 / (0.5 / 448) = 448; NaN stays NaN
+            assert set(np.unique(body)) <= {0x7E, 0x7F}                  # 0.5 * (448 / 0.5) = 448; NaN stays NaN
             assert arena[soff:soff + 4].view(np.float32)[0] == np.float32(0.5) / np.float32(448)
