@@ -237,6 +237,7 @@ def main():
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--no-staging", action="store_true", help="skip the host-link sections")
     ap.add_argument("--no-cpu", action="store_true", help="skip the CPU oracle baseline")
+    ap.add_argument("--no-fp8", action="store_true", help="skip the fp8 block-quantised variant")
     ap.add_argument("--cpu-seconds", type=float, default=12.0)
     ap.add_argument("--layers", type=int, default=0, help="profiling aid: override the layer count (smaller case)")
     ap.add_argument("--vocab", type=int, default=0, help="profiling aid: override the vocabulary size")
@@ -389,6 +390,32 @@ def main():
 
     del flat_back
     torch.cuda.empty_cache()
+
+    # the fp8 variant of the same switch: linear weights as e4m3 with one scale per 128 x 128 block
+    if cfg["gathered"] and halves == 1 and not args.no_fp8:
+        qplan = dr.Plan(cfg["spec"], world=cfg["world"], rank=cfg["rank"], gathered=True, tp=cfg["tp"],
+                        tp_rank=cfg["tp_rank"], dtype=dr.DR_FP8_E4M3_B128)
+        qarena = torch.empty(qplan.info.dst_bytes, dtype=torch.uint8, device=dev)
+        for _ in range(args.warmup):
+            qplan.reshard(master, qarena)
+        qe = [torch.cuda.Event(enable_timing=True) for _ in range(args.steps + 1)]
+        qe[0].record()
+        for i in range(args.steps):
+            qplan.reshard(master, qarena)
+            qe[i + 1].record()
+        torch.cuda.synchronize()
+        qms = [qe[i].elapsed_time(qe[i + 1]) for i in range(args.steps)]
+        qavg = sum(qms) / len(qms)
+        qb = qplan.info.bytes_moved_fwd
+        line["fp8_forward"] = {"what": "dr_reshard with dtype DR_FP8_E4M3_B128 (copy kernel for bf16 tensors + block-quantisation "
+                                       "kernel), same source", "bytes": int(qb), "quant_elems": int(qplan.info.quant_elems),
+                               "quant_blocks": int(qplan.info.quant_blocks), "gbs_avg": qb / qavg / 1e6,
+                               "gbs_best": qb / min(qms) / 1e6, "ms_avg": qavg, "ms_best": min(qms),
+                               "frac_of_measured_peak": qb / qavg / 1e6 / peak, "frac_of_nominal_8000": qb / qavg / 1e6 / 8000.0,
+                               "algorithmic_bytes_per_quant_elem": 5}
+        qplan.close()
+        del qarena
+        torch.cuda.empty_cache()
 
     # ---- host-link sections ---------------------------------------------------------------------
     if not args.no_staging:

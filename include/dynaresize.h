@@ -53,7 +53,7 @@ typedef enum dr_status {
 
 enum { DR_SRC_FSDP_FLAT = 1 };
 enum { DR_DST_ROLLOUT_FUSED = 1 };
-enum { DR_F32 = 1, DR_BF16 = 2 };
+enum { DR_F32 = 1, DR_BF16 = 2, DR_FP8_E4M3_B128 = 3 };
 
 /* Decoder shape.  Dense when n_experts == 0 (SwiGLU of width ffn), else every layer holds a router
  * [n_experts, hidden] and n_experts SwiGLU experts of width moe_ffn (ffn is ignored). */
@@ -99,6 +99,18 @@ typedef struct dr_dst_layout {
     uint32_t moe_ep_rank;       /* this rank keeps experts [rank * E / ep, (rank + 1) * E / ep)           */
 } dr_dst_layout;
 
+/*
+ * dtype DR_FP8_E4M3_B128 (a rollout-engine layout, no counterpart in the paper): the linear weights
+ * (qkv, o, gate_up, down, w13, w2) are written as fp8 e4m3 with one fp32 scale per 128 x 128 block of
+ * the rollout tensor; embed, lm_head, router and the norms stay bf16.  Per block: amax = max |x| (NaNs
+ * skipped), stored scale = amax / 448 in fp32, q = e4m3(x * (448 / amax)) with the reciprocal and the
+ * product each rounded once in fp32 (an all-zero block takes scale 1), round to nearest even,
+ * magnitudes above 448 saturating to 448, NaN -> 0x7F.  A quantised tensor
+ * occupies rows * cols bytes at arena_off, then its scales, row-major, at scale_off (the next multiple
+ * of arena_align_bytes).  Needs the whole flat buffer (gathered = 1 or world = 1): a block cannot be
+ * scaled from part of its elements.  dr_reshard only; the inverse, static and streamed calls return
+ * DR_ERR_UNSUPPORTED for such a plan.
+ */
 typedef struct dr_plan dr_plan;
 
 typedef struct dr_plan_info {
@@ -112,6 +124,8 @@ typedef struct dr_plan_info {
     uint64_t elems_moved;     /* elements one dr_reshard / dr_reshard_inverse moves                  */
     uint64_t bytes_moved_fwd; /* algorithmic bytes of dr_reshard: (4 + dst element size) * elems     */
     uint64_t bytes_moved_inv; /* the same for dr_reshard_inverse                                     */
+    uint64_t quant_elems;     /* DR_FP8_E4M3_B128 plans: elements written as fp8 (counted in elems_moved) */
+    uint64_t quant_blocks;    /* and the number of 128 x 128 blocks, one fp32 scale each              */
 } dr_plan_info;
 
 typedef struct dr_tensor_desc {
@@ -119,6 +133,10 @@ typedef struct dr_tensor_desc {
     uint64_t arena_off; /* byte offset of the tensor inside the rollout arena                       */
     uint64_t rows, cols;
     int64_t alias_of;   /* >= 0: index of the rollout tensor whose storage this one shares           */
+    uint32_t elem_size; /* bytes per element of the payload: 4, 2, or 1 (fp8)                         */
+    uint32_t quantised; /* 1: fp8 payload with block scales                                          */
+    uint64_t scale_off; /* quantised: byte offset of the fp32 scales [scale_rows, scale_cols]         */
+    uint64_t scale_rows, scale_cols; /* ceil(rows / 128), ceil(cols / 128)                            */
 } dr_tensor_desc;
 
 /* One entry of the compiled map: rows x row_len elements, row i read from source element

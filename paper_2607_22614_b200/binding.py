@@ -13,7 +13,7 @@ DR_ERR_CUDA, DR_ERR_BUDGET, DR_ERR_SINK, DR_ERR_TIMEOUT, DR_ERR_STATE = -6, -7, 
 DR_VERSION = 1
 DR_SRC_FSDP_FLAT = 1
 DR_DST_ROLLOUT_FUSED = 1
-DR_F32, DR_BF16 = 1, 2
+DR_F32, DR_BF16, DR_FP8_E4M3_B128 = 1, 2, 3
 DR_MAX_STAGE_BUFS = 8
 DR_STAGE_HOST_OFFSETS = 1
 
@@ -42,11 +42,13 @@ class dr_dst_layout(C.Structure):
 
 class dr_plan_info(C.Structure):
     _fields_ = [(n, u64) for n in ("flat_elems", "shard_elems", "src_bytes", "dst_bytes", "n_tensors", "n_segments",
-                                   "n_tiles", "elems_moved", "bytes_moved_fwd", "bytes_moved_inv")]
+                                   "n_tiles", "elems_moved", "bytes_moved_fwd", "bytes_moved_inv",
+                                   "quant_elems", "quant_blocks")]
 
 
 class dr_tensor_desc(C.Structure):
-    _fields_ = [("name", C.c_char * 64), ("arena_off", u64), ("rows", u64), ("cols", u64), ("alias_of", i64)]
+    _fields_ = [("name", C.c_char * 64), ("arena_off", u64), ("rows", u64), ("cols", u64), ("alias_of", i64),
+                ("elem_size", u32), ("quantised", u32), ("scale_off", u64), ("scale_rows", u64), ("scale_cols", u64)]
 
 
 class dr_segment_desc(C.Structure):

@@ -33,7 +33,7 @@ int validate(const dr_model_spec* s, const dr_src_layout* a, const dr_dst_layout
         return DR_ERR_INVALID;
     }
     if (a->kind != DR_SRC_FSDP_FLAT || a->dtype != DR_F32 || b->kind != DR_DST_ROLLOUT_FUSED ||
-        (b->dtype != DR_BF16 && b->dtype != DR_F32)) {
+        (b->dtype != DR_BF16 && b->dtype != DR_F32 && b->dtype != DR_FP8_E4M3_B128)) {
         set_error("unknown layout kind or dtype");
         return DR_ERR_UNSUPPORTED;
     }
@@ -50,6 +50,10 @@ int validate(const dr_model_spec* s, const dr_src_layout* a, const dr_dst_layout
     if (al < 16 || (al & (al - 1))) {
         set_error("arena_align_bytes must be a power of two >= 16");
         return DR_ERR_INVALID;
+    }
+    if (b->dtype == DR_FP8_E4M3_B128 && !a->gathered && a->world > 1) {
+        set_error("fp8 block scaling needs the whole flat buffer (gathered = 1)");
+        return DR_ERR_UNSUPPORTED;
     }
     if (b->moe_tp != 1 && b->moe_tp != tp) {
         set_error("moe_tp must be 1 (experts unsliced) or tp");
@@ -92,7 +96,8 @@ int create(const dr_model_spec* s, const dr_src_layout* a, const dr_dst_layout* 
     p->dst = *b;
     p->tp = tp;
     p->tp_rank = rank;
-    p->elem_size = b->dtype == DR_BF16 ? 2 : 4;
+    p->elem_size = b->dtype == DR_F32 ? 4 : 2;
+    p->fp8 = b->dtype == DR_FP8_E4M3_B128;
     p->host_only = host_only;
     try {
         rc = compile_plan(p);
@@ -107,6 +112,15 @@ int create(const dr_model_spec* s, const dr_src_layout* a, const dr_dst_layout* 
         size_t hbytes = p->hints.size() * sizeof(uint32_t);
         if (e == cudaSuccess) e = cudaMalloc((void**)&p->d_hints, hbytes);
         if (e == cudaSuccess) e = cudaMemcpy(p->d_hints, p->hints.data(), hbytes, cudaMemcpyHostToDevice);
+        auto upload = [&](void** dst, const void* src, size_t n) {
+            if (e == cudaSuccess && n) e = cudaMalloc(dst, n);
+            if (e == cudaSuccess && n) e = cudaMemcpy(*dst, src, n, cudaMemcpyHostToDevice);
+        };
+        if (p->fp8) {
+            upload((void**)&p->d_qtensors, p->qtensors.data(), p->qtensors.size() * sizeof(QTensor));
+            upload((void**)&p->d_qparts, p->qparts.data(), p->qparts.size() * sizeof(QPart));
+            upload((void**)&p->d_qhints, p->qhints.data(), p->qhints.size() * sizeof(uint32_t));
+        }
         if (e == cudaSuccess) p->grid = choose_grid(p->device, p->elem_size);
         if (e != cudaSuccess || p->grid <= 0) {
             set_error("plan upload: %s", cudaGetErrorString(e));
@@ -191,6 +205,11 @@ int dr_plan_tensor(const dr_plan* plan, uint32_t i, dr_tensor_desc* out)
     out->rows = t.rows;
     out->cols = t.cols;
     out->alias_of = t.alias_of;
+    out->elem_size = t.es;
+    out->quantised = t.quant ? 1 : 0;
+    out->scale_off = t.scale_off;
+    out->scale_rows = t.quant ? (t.rows + 127) / 128 : 0;
+    out->scale_cols = t.quant ? (t.cols + 127) / 128 : 0;
     return DR_OK;
 }
 
@@ -218,7 +237,9 @@ int dr_reshard(const dr_plan* plan, const void* src_dev, uint64_t src_bytes, voi
     int rc = check_call(plan, src_dev, src_bytes, plan ? plan->info.src_bytes : 0, dst_dev, dst_bytes,
                         plan ? plan->info.dst_bytes : 0);
     if (rc) return rc;
-    return launch_reshard(plan, false, src_dev, dst_dev, nullptr, cuda_stream);
+    rc = launch_reshard(plan, false, src_dev, dst_dev, nullptr, cuda_stream);
+    if (rc == DR_OK && plan->fp8) rc = launch_quant(plan, src_dev, dst_dev, cuda_stream);
+    return rc;
 }
 
 int dr_reshard_inverse(const dr_plan* plan, const void* rollout_dev, uint64_t rollout_bytes, void* flat_dev,
@@ -227,6 +248,10 @@ int dr_reshard_inverse(const dr_plan* plan, const void* rollout_dev, uint64_t ro
     int rc = check_call(plan, rollout_dev, rollout_bytes, plan ? plan->info.dst_bytes : 0, flat_dev, flat_bytes,
                         plan ? plan->info.src_bytes : 0);
     if (rc) return rc;
+    if (plan->fp8) {
+        set_error("fp8 plans have no inverse map");
+        return DR_ERR_UNSUPPORTED;
+    }
     return launch_reshard(plan, true, nullptr, flat_dev, rollout_dev, cuda_stream);
 }
 
@@ -252,6 +277,9 @@ int dr_plan_destroy(dr_plan* plan)
     if (plan->ring) ring_destroy(plan->ring);
     if (plan->d_segs) cudaFree(plan->d_segs);
     if (plan->d_hints) cudaFree(plan->d_hints);
+    if (plan->d_qtensors) cudaFree(plan->d_qtensors);
+    if (plan->d_qparts) cudaFree(plan->d_qparts);
+    if (plan->d_qhints) cudaFree(plan->d_qhints);
     delete plan;
     return DR_OK;
 }

@@ -43,6 +43,24 @@ struct DevSeg {
 };
 static_assert(sizeof(DevSeg) == 48, "DevSeg layout");
 
+// fp8 block quantisation: one entry per quantised rollout tensor, one per row-block source part.
+struct QPart {
+    uint64_t src_off;   // flat element offset of the part's first row, at the tensor's first column
+    uint32_t dst_row0;  // first rollout row the part fills
+    uint32_t rows;
+    uint32_t src_stride;  // elements between source rows
+    uint32_t pad;
+};
+static_assert(sizeof(QPart) == 24, "QPart layout");
+struct QTensor {
+    uint64_t payload_off, scale_off;  // arena bytes
+    uint64_t block0;                  // index of the tensor's first block
+    uint32_t rows, cols, nbc;         // nbc = column blocks
+    uint32_t part0, n_parts;
+    uint32_t aligned;                 // 1: every source row start and the column count allow 256-bit loads
+};
+static_assert(sizeof(QTensor) == 48, "QTensor layout");
+
 struct HostSeg {
     uint64_t dst_off, src_off, rows, row_len, src_stride, dst_stride;
     uint32_t flags, tensor;
@@ -52,6 +70,9 @@ struct Tensor {
     std::string name;
     uint64_t arena_off = 0, rows = 0, cols = 0;
     int64_t alias_of = -1;
+    uint32_t es = 2;         // payload bytes per element
+    bool quant = false;
+    uint64_t scale_off = 0;  // quantised tensors
 };
 
 // Everything a launch needs besides the buffers.
@@ -80,11 +101,20 @@ struct dr_plan {
     // hints[i] = segment holding tile i << hint_shift: a tile finds its segment with one load plus a short walk
     std::vector<uint32_t> hints;
     uint32_t hint_shift = 0;
+    // fp8 plans: quantised tensors, their parts, and a block -> tensor hint table
+    bool fp8 = false;
+    std::vector<dr::QTensor> qtensors;
+    std::vector<dr::QPart> qparts;
+    std::vector<uint32_t> qhints;
+    uint32_t qhint_shift = 0;
     // device side (absent on a host-only plan)
     bool host_only = true;
     int device = -1;
     dr::DevSeg* d_segs = nullptr;
     uint32_t* d_hints = nullptr;
+    dr::QTensor* d_qtensors = nullptr;
+    dr::QPart* d_qparts = nullptr;
+    uint32_t* d_qhints = nullptr;
     int grid = 0;
     // staging
     std::mutex stage_mu;
@@ -99,6 +129,7 @@ int compile_plan(dr_plan* p);  // planner.cpp: fills tensors, segs, dev_segs, in
 int launch_reshard(const dr_plan* p, bool inverse, const void* flat, void* arena_or_flat_out, const void* arena_in,
                    void* stream);
 int choose_grid(int device, uint32_t elem_size);  // resident CTAs of the reshard kernel on the whole GPU
+int launch_quant(const dr_plan* p, const void* flat, void* arena, void* stream);
 void ring_destroy(Ring* r);
 void stream_destroy(Stream* s);
 int build_tables(const std::vector<HostSeg>& segs, Tables* out);

@@ -25,23 +25,74 @@ struct Builder {
     }
 };
 
+// The linear weights that DR_FP8_E4M3_B128 quantises; everything else stays bf16.
+bool is_linear_weight(const std::string& name)
+{
+    size_t dot = name.rfind('.');
+    std::string leaf = dot == std::string::npos ? name : name.substr(dot + 1);
+    return leaf == "qkv" || leaf == "o" || leaf == "gate_up" || leaf == "down" || leaf == "w13" || leaf == "w2";
+}
+
 struct Emit {
     dr_plan* p;
     uint64_t arena = 0;
+    uint64_t align_up(uint64_t x) const
+    {
+        uint64_t a = p->dst.arena_align_bytes;
+        return (x + a - 1) / a * a;
+    }
+    // Close the tensor being built: a quantised tensor is followed by its block scales.
+    void finish()
+    {
+        if (p->tensors.empty()) return;
+        Tensor& t = p->tensors.back();
+        if (!t.quant || t.alias_of >= 0) return;
+        QTensor& q = p->qtensors.back();
+        q.rows = (uint32_t)t.rows;
+        q.nbc = (uint32_t)((t.cols + 127) / 128);
+        q.n_parts = (uint32_t)p->qparts.size() - q.part0;
+        t.scale_off = align_up(t.arena_off + t.rows * t.cols);
+        q.scale_off = t.scale_off;
+        arena = t.scale_off + ((t.rows + 127) / 128) * q.nbc * 4;
+    }
     void begin(const std::string& name, uint64_t cols)
     {
+        finish();
         Tensor t;
         t.name = name;
         t.cols = cols;
-        uint64_t a = p->dst.arena_align_bytes;
-        arena = (arena + a - 1) / a * a;
+        t.quant = p->fp8 && is_linear_weight(name);
+        t.es = t.quant ? 1 : p->elem_size;
+        arena = align_up(arena);
         t.arena_off = arena;
         p->tensors.push_back(t);
+        if (t.quant) {
+            QTensor q{};
+            q.payload_off = t.arena_off;
+            q.cols = (uint32_t)cols;
+            q.part0 = (uint32_t)p->qparts.size();
+            q.aligned = (cols % 8 == 0 && t.arena_off % 8 == 0) ? 1 : 0;
+            p->qtensors.push_back(q);
+        }
     }
     // Append rows [r0, r0+nr) x cols [c0, c0+cols) of parameter q below what the tensor already holds.
     void block(const Param& q, uint64_t r0, uint64_t c0, uint64_t nr)
     {
         Tensor& t = p->tensors.back();
+        if (t.quant) {  // recorded as a row-block part of a quantised tensor, not as a copy segment
+            if (nr) {
+                QPart qp{};
+                qp.src_off = q.off + r0 * q.cols + c0;
+                qp.dst_row0 = (uint32_t)t.rows;
+                qp.rows = (uint32_t)nr;
+                qp.src_stride = (uint32_t)q.cols;
+                if (qp.src_off % 8 || q.cols % 8) p->qtensors.back().aligned = 0;
+                p->qparts.push_back(qp);
+            }
+            t.rows += nr;
+            arena = t.arena_off + t.rows * t.cols;
+            return;
+        }
         HostSeg g{};
         g.dst_off = t.arena_off + t.rows * t.cols * p->elem_size;
         g.src_off = q.off + r0 * q.cols + c0;
@@ -356,6 +407,7 @@ int compile_plan(dr_plan* p)
         out.pad_rows(Vp / T);
     }
 
+    out.finish();
     const uint64_t N = flat.next, W = p->src.world, S = (N + W - 1) / W;
     merge_adjacent(p->segs, es);
     if (!p->src.gathered) clip_to_shard(p->segs, (uint64_t)p->src.rank * S, (uint64_t)(p->src.rank + 1) * S, es);
@@ -369,6 +421,26 @@ int compile_plan(dr_plan* p)
     p->hint_shift = tb.hint_shift;
     const uint64_t tiles = tb.n_tiles, moved = tb.elems;
 
+    // fp8: block prefix per quantised tensor and a block -> tensor hint table
+    uint64_t qblocks = 0, qelems = 0;
+    for (QTensor& q : p->qtensors) {
+        q.block0 = qblocks;
+        qblocks += (uint64_t)((q.rows + 127) / 128) * q.nbc;
+        qelems += (uint64_t)q.rows * q.cols;
+    }
+    if (p->fp8) {
+        p->qhint_shift = 0;
+        while (((qblocks + (1ull << p->qhint_shift) - 1) >> p->qhint_shift) > kMaxHints) ++p->qhint_shift;
+        const uint64_t n_hints = (qblocks + (1ull << p->qhint_shift) - 1) >> p->qhint_shift;
+        p->qhints.assign(n_hints ? n_hints : 1, 0);
+        uint32_t qi = 0;
+        for (uint64_t h = 0; h < n_hints; ++h) {
+            const uint64_t b = h << p->qhint_shift;
+            while (qi + 1 < p->qtensors.size() && p->qtensors[qi + 1].block0 <= b) ++qi;
+            p->qhints[h] = qi;
+        }
+    }
+
     dr_plan_info& I = p->info;
     I.flat_elems = N;
     I.shard_elems = S;
@@ -377,9 +449,11 @@ int compile_plan(dr_plan* p)
     I.n_tensors = p->tensors.size();
     I.n_segments = p->segs.size();
     I.n_tiles = tiles;
-    I.elems_moved = moved;
-    I.bytes_moved_fwd = moved * (4 + es);
+    I.elems_moved = moved + qelems;
+    I.bytes_moved_fwd = moved * (4 + es) + qelems * 5 + qblocks * 4;
     I.bytes_moved_inv = moved * (4 + es);
+    I.quant_elems = qelems;
+    I.quant_blocks = qblocks;
 
     // Every access the kernels will make is checked here, so a launch cannot leave its buffers.
     const uint64_t src_elems = I.src_bytes / 4;

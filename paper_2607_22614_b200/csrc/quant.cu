@@ -1,0 +1,171 @@
+// fp32 -> fp8 e4m3 with one fp32 scale per 128 x 128 block of the rollout tensor (sm_100a).
+//
+// One CTA per block: 512 threads hold the block's 16 384 values in registers (four 256-bit loads in
+// flight per thread, three CTAs per SM, each row of the block one contiguous 512 B request), reduce |x| to the block
+// maximum with shuffles and one shared-memory step, then
+// multiply by the block's reciprocal scale, convert two values per cvt.rn.satfinite.e4m3x2.f32 and store
+// each row as one contiguous 128 B request.  The bound is HBM: 4 B read + 1 B written per element (+ 4 B
+// per 16 384 elements for the scale).
+#include <cuda_runtime.h>
+
+#include "dr_internal.h"
+
+namespace dr {
+namespace {
+
+#ifndef DR_Q_THREADS
+#define DR_Q_THREADS 512
+#endif
+#ifndef DR_Q_MIN_BLOCKS
+#define DR_Q_MIN_BLOCKS 3
+#endif
+constexpr int kQThreads = DR_Q_THREADS;
+constexpr int kRowsPerPass = kQThreads / 16;   // 16 threads cover one 128-column block row
+constexpr int kPasses = 128 / kRowsPerPass;    // block rows per thread
+static_assert(kQThreads >= 128 && 128 % kRowsPerPass == 0, "thread count must tile the block");
+
+__device__ __forceinline__ void ld256f(const void* p, float (&v)[8])
+{
+    asm volatile("ld.global.nc.L1::no_allocate.v8.f32 {%0,%1,%2,%3,%4,%5,%6,%7}, [%8];"
+                 : "=f"(v[0]), "=f"(v[1]), "=f"(v[2]), "=f"(v[3]), "=f"(v[4]), "=f"(v[5]), "=f"(v[6]), "=f"(v[7])
+                 : "l"(p));
+}
+__device__ __forceinline__ float ld32f(const void* p)
+{
+    float v;
+    asm volatile("ld.global.nc.L1::no_allocate.f32 %0, [%1];" : "=f"(v) : "l"(p));
+    return v;
+}
+// two fp32 -> two e4m3 bytes: round to nearest even, saturate to +-448; a NaN of either sign comes out
+// as 0x7F (checked against the oracle on sources made of every bit pattern)
+__device__ __forceinline__ uint32_t cvt_e4m3x2(float lo, float hi)
+{
+    uint16_t d;
+    asm("cvt.rn.satfinite.e4m3x2.f32 %0, %1, %2;" : "=h"(d) : "f"(hi), "f"(lo));
+    return d;
+}
+__global__ void __launch_bounds__(kQThreads, DR_Q_MIN_BLOCKS)
+    quant_kernel(const QTensor* __restrict__ tensors, uint32_t n_tensors, const QPart* __restrict__ parts,
+                 const uint32_t* __restrict__ hints, uint32_t hint_shift, const char* __restrict__ flat,
+                 char* __restrict__ arena)
+{
+    __shared__ uint64_t row_src[128];  // flat element offset of (row, first column of the tensor)
+    __shared__ float warp_max[kQThreads / 32];
+    __shared__ float s_recip;
+
+    const uint64_t b = blockIdx.x;
+    // block -> tensor: hint plus a short walk (all threads, same addresses: broadcast loads)
+    uint32_t ti = hints[b >> hint_shift];
+    while (ti + 1 < n_tensors && tensors[ti + 1].block0 <= b) ++ti;
+    const QTensor T = tensors[ti];
+    const uint32_t lb = (uint32_t)(b - T.block0);
+    const uint32_t bi = lb / T.nbc, bj = lb - bi * T.nbc;
+    const uint32_t r0 = bi * 128, c0 = bj * 128;
+    const uint32_t nrows = min(128u, T.rows - r0);
+
+    // each of the first 128 threads finds the source row of one block row (binary search over the parts)
+    if (threadIdx.x < 128) {
+        uint64_t off = 0;
+        const uint32_t r = r0 + threadIdx.x;
+        if (threadIdx.x < nrows) {
+            uint32_t lo = T.part0, hi = T.part0 + T.n_parts;  // last part with dst_row0 <= r
+            while (hi - lo > 1) {
+                uint32_t mid = lo + (hi - lo) / 2;
+                if (parts[mid].dst_row0 <= r) lo = mid; else hi = mid;
+            }
+            const QPart P = parts[lo];
+            off = P.src_off + (uint64_t)(r - P.dst_row0) * P.src_stride;
+        }
+        row_src[threadIdx.x] = off;
+    }
+    __syncthreads();
+
+    const uint32_t cu = threadIdx.x & 15;   // 8-column unit inside the block row
+    const uint32_t rb = threadIdx.x >> 4;   // row inside a pass
+    const uint32_t col = c0 + cu * 8;
+    float v[kPasses][8];
+    float amax = 0.0f;
+#pragma unroll
+    for (int p = 0; p < kPasses; ++p) {
+        const uint32_t row = p * kRowsPerPass + rb;
+#pragma unroll
+        for (int k = 0; k < 8; ++k) v[p][k] = 0.0f;
+        if (row < nrows && col < T.cols) {
+            const char* src = flat + (row_src[row] + col) * 4;
+            if (T.aligned) {
+                ld256f(src, v[p]);
+            } else {
+#pragma unroll
+                for (int k = 0; k < 8; ++k)
+                    if (col + k < T.cols) v[p][k] = ld32f(src + 4 * k);
+            }
+        }
+    }
+#pragma unroll
+    for (int p = 0; p < kPasses; ++p)
+#pragma unroll
+        for (int k = 0; k < 8; ++k) amax = fmaxf(amax, fabsf(v[p][k]));  // fmaxf drops NaN operands
+#pragma unroll
+    for (int o = 16; o; o >>= 1) amax = fmaxf(amax, __shfl_xor_sync(0xFFFFFFFFu, amax, o));
+    if ((threadIdx.x & 31) == 0) warp_max[threadIdx.x >> 5] = amax;
+    __syncthreads();
+    if (threadIdx.x == 0) {
+        float m = warp_max[0];
+#pragma unroll
+        for (int w = 1; w < kQThreads / 32; ++w) m = fmaxf(m, warp_max[w]);
+        float scale = __fdiv_rn(m, 448.0f), recip = __fdiv_rn(448.0f, m);
+        if (m == 0.0f) scale = recip = 1.0f;
+        s_recip = recip;
+        *(float*)(arena + T.scale_off + ((uint64_t)bi * T.nbc + bj) * 4) = scale;
+    }
+    __syncthreads();
+    const float recip = s_recip;
+
+#pragma unroll
+    for (int p = 0; p < kPasses; ++p) {
+        const uint32_t row = p * kRowsPerPass + rb;
+        if (row >= nrows || col >= T.cols) continue;
+        uint32_t q[8];
+#pragma unroll
+        for (int k = 0; k < 8; k += 2) {
+            const float a = __fmul_rn(v[p][k], recip), c = __fmul_rn(v[p][k + 1], recip);
+            const uint32_t two = cvt_e4m3x2(a, c);
+            q[k] = two & 0xFF;
+            q[k + 1] = two >> 8;
+        }
+        char* dst = arena + T.payload_off + (uint64_t)(r0 + row) * T.cols + col;
+        if (T.aligned) {
+            uint2 w;
+            w.x = q[0] | (q[1] << 8) | (q[2] << 16) | (q[3] << 24);
+            w.y = q[4] | (q[5] << 8) | (q[6] << 16) | (q[7] << 24);
+            asm volatile("st.global.L1::no_allocate.v2.b32 [%0], {%1,%2};" ::"l"(dst), "r"(w.x), "r"(w.y) : "memory");
+        } else {
+#pragma unroll
+            for (int k = 0; k < 8; ++k)
+                if (col + k < T.cols) dst[k] = (char)q[k];
+        }
+    }
+}
+
+}  // namespace
+
+int launch_quant(const dr_plan* p, const void* flat, void* arena, void* stream)
+{
+    const uint64_t blocks = p->info.quant_blocks;
+    if (blocks == 0) return DR_OK;
+    if (blocks > 0x7FFFFFFFull) {
+        set_error("too many quantisation blocks");
+        return DR_ERR_UNSUPPORTED;
+    }
+    quant_kernel<<<(unsigned)blocks, kQThreads, 0, (cudaStream_t)stream>>>(
+        p->d_qtensors, (uint32_t)p->qtensors.size(), p->d_qparts, p->d_qhints, p->qhint_shift, (const char*)flat,
+        (char*)arena);
+    cudaError_t e = cudaGetLastError();
+    if (e != cudaSuccess) {
+        set_error("quant kernel launch: %s", cudaGetErrorString(e));
+        return DR_ERR_CUDA;
+    }
+    return DR_OK;
+}
+
+}  // namespace dr

@@ -419,6 +419,10 @@ extern "C" int dr_reshard_static(const dr_plan* plan, const void* src_dev, uint6
         return DR_ERR_INVALID;
     }
     const uint64_t n_segs = plan->dev_segs.size();
+    if (plan->fp8) {
+        set_error("fp8 plans are not supported by the static entry point");
+        return DR_ERR_UNSUPPORTED;
+    }
     if (n_segs > kStaticMaxSegs) {
         set_error("plan has %llu segments; the static table holds at most %u (use dr_plan_create + dr_reshard)",
                   (unsigned long long)n_segs, kStaticMaxSegs);

@@ -137,6 +137,10 @@ extern "C" int dr_reshard_stream(dr_plan* plan, const dr_stream_desc* d, dr_stre
         set_error("host-only plan cannot launch");
         return DR_ERR_STATE;
     }
+    if (plan->fp8) {
+        set_error("fp8 plans cannot be streamed: a block needs all of its source rows");
+        return DR_ERR_UNSUPPORTED;
+    }
     if (d->host_src_bytes < plan->info.src_bytes || d->dst_bytes < plan->info.dst_bytes ||
         (d->host_dst && d->host_dst_bytes < plan->info.dst_bytes)) {
         set_error("a buffer is smaller than the plan needs");

@@ -124,7 +124,7 @@ def test_library_exports_every_declared_symbol():
 
 def test_struct_sizes_match_the_header_layout():
     assert C.sizeof(dr.dr_model_spec) == 48 and C.sizeof(dr.dr_src_layout) == 28 and C.sizeof(dr.dr_dst_layout) == 36
-    assert C.sizeof(dr.dr_stage_desc) == 432 and C.sizeof(dr.dr_stage_stats) == 112 and C.sizeof(dr.dr_plan_info) == 80 and C.sizeof(dr.dr_tensor_desc) == 96 and C.sizeof(dr.dr_segment_desc) == 56
+    assert C.sizeof(dr.dr_stage_desc) == 432 and C.sizeof(dr.dr_stage_stats) == 112 and C.sizeof(dr.dr_plan_info) == 96 and C.sizeof(dr.dr_tensor_desc) == 128 and C.sizeof(dr.dr_segment_desc) == 56
 
 
 def test_error_codes():
@@ -211,3 +211,41 @@ def test_layout_variant_errors():
     with pytest.raises(dr.DrError) as e:
         dr.Plan(MID[2]["spec"], tp=4, moe_tp=2, host_only=True)
     assert e.value.status == E.DR_ERR_UNSUPPORTED
+
+
+@pytest.mark.parametrize("spec,T,opts", [(MID[0]["spec"], 2, {}), (MID[2]["spec"], 2, dict(moe_ep=2, moe_ep_rank=1)),
+                                         (dict(BRUTE[0]["spec"], ffn=12), 2, {}), (CONFIGS[2]["spec"], 1, {})],
+                         ids=["mid-dense", "mid-moe-ep", "brute", "qwen3-8b"])
+def test_fp8_plan_layout_matches_oracle(spec, T, opts):
+    for t in range(T):
+        p = dr.Plan(spec, tp=T, tp_rank=t, dtype=dr.DR_FP8_E4M3_B128, arena_align_bytes=64, host_only=True, **opts)
+        om = oracle.Model(spec, tp=T, tp_rank=t, arena_align=64, **opts)
+        total, lay = om.fp8_layout()
+        assert p.info.dst_bytes == total
+        q_elems = q_blocks = 0
+        for a, b, (qz, off, soff) in zip(p.tensors(), om.dst_tensors(), lay):
+            assert (a.name.decode(), a.rows, a.cols, a.alias_of, bool(a.quantised), a.arena_off) == \
+                   (b.name, b.rows, b.cols, b.alias_of, qz and b.alias_of < 0 or qz, off)
+            if qz:
+                assert a.elem_size == 1 and a.scale_off == soff
+                assert (a.scale_rows, a.scale_cols) == (-(-b.rows // 128), -(-b.cols // 128))
+                q_elems += b.rows * b.cols
+                q_blocks += a.scale_rows * a.scale_cols
+            elif b.alias_of < 0:
+                assert a.elem_size == 2
+        assert (p.info.quant_elems, p.info.quant_blocks) == (q_elems, q_blocks)
+        copied = p.info.elems_moved - q_elems
+        assert p.info.bytes_moved_fwd == copied * 6 + q_elems * 5 + q_blocks * 4
+        # the copy segments cover exactly the non-quantised tensors
+        assert sum(s.rows * s.row_len for s in p.segments()) == copied == \
+            sum(b.rows * b.cols for b, (qz, _, _) in zip(om.dst_tensors(), lay) if not qz and b.alias_of < 0)
+        p.close()
+
+
+def test_fp8_plan_restrictions():
+    E = dr.binding
+    with pytest.raises(dr.DrError) as e:
+        dr.Plan(MID[0]["spec"], world=2, rank=0, gathered=False, dtype=dr.DR_FP8_E4M3_B128, host_only=True)
+    assert e.value.status == E.DR_ERR_UNSUPPORTED
+    p = dr.Plan(MID[0]["spec"], world=2, rank=1, gathered=True, dtype=dr.DR_FP8_E4M3_B128, host_only=True)
+    assert p.info.quant_blocks > 0
