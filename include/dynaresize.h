@@ -349,6 +349,31 @@ int dr_reshard_stream(dr_plan* plan, const dr_stream_desc* desc, dr_stream_stats
 int dr_shard_range(uint64_t flat_elems, uint32_t world, uint32_t rank, uint64_t* begin, uint64_t* end,
                    uint64_t* shard_elems);
 
+/*
+ * Hysteresis-guided reconfiguration (Sec. 3.4; host only, no CUDA).  The controller only decides WHEN to
+ * move between pre-specified topologies, listed from most-Training to most-Rollout (e.g. 6:2, 5:3, 4:4).
+ * Per step: imbalance = (t_rollout - t_train) / max(t_rollout, t_train).  A step signals "towards
+ * Rollout" if imbalance > enter_threshold, "towards Training" if < -enter_threshold, is quiet if
+ * |imbalance| < exit_threshold, and otherwise lies in the hysteresis band (the streak of signals neither
+ * grows nor resets).  A move by one position is decided when `consecutive` signals of one direction have
+ * arrived in a row, the topology has been held for dwell_steps, the previous move is cooldown_steps ago
+ * (Sec. 5 Exp#3: more than 10 steps, above the ~11-step break-even) and the neighbour exists.
+ */
+typedef struct dr_ctl_config {
+    uint32_t struct_size, n_topologies, initial;
+    uint32_t consecutive, dwell_steps, cooldown_steps;
+    double enter_threshold, exit_threshold; /* 0 <= exit <= enter, enter > 0 */
+} dr_ctl_config;
+typedef struct dr_ctl dr_ctl;
+
+int dr_ctl_create(const dr_ctl_config* cfg, dr_ctl** out);                /* DR_ERR_INVALID, DR_ERR_NOMEM */
+/* Feed one step.  *move = -1 / 0 / +1, *topology = index after the move.  DR_ERR_INVALID on NaN / negative times. */
+int dr_ctl_observe(dr_ctl* ctl, double t_rollout, double t_train, int32_t* move, uint32_t* topology);
+/* Sustained steps after which one resize has paid for itself: cost / (step_before - step_after) (Exp#3);
+ * infinity when the step did not get faster. */
+int dr_ctl_break_even(double resize_cost_s, double step_before_s, double step_after_s, double* steps);
+int dr_ctl_destroy(dr_ctl* ctl);
+
 /* Synchronises the plan's own streams, frees its ring, table and streams.  NULL is accepted. */
 int dr_plan_destroy(dr_plan* plan);
 

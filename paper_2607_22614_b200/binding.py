@@ -19,7 +19,7 @@ DR_STAGE_HOST_OFFSETS = 1
 
 EXPORTS = ["dr_plan_create", "dr_plan_create_host", "dr_plan_query", "dr_plan_tensor", "dr_plan_segment",
            "dr_reshard", "dr_reshard_inverse", "dr_reshard_static", "dr_reshard_stream", "dr_shard_range", "dr_stage_out", "dr_stage_in", "dr_plan_destroy", "dr_strerror",
-           "dr_last_error"]
+           "dr_last_error", "dr_ctl_create", "dr_ctl_observe", "dr_ctl_break_even", "dr_ctl_destroy"]
 
 u8, u32, u64, i64, vp = C.c_uint8, C.c_uint32, C.c_uint64, C.c_int64, C.c_void_p
 
@@ -82,6 +82,11 @@ class dr_stream_stats(C.Structure):
     _fields_ = [("h2d_bytes", u64), ("d2h_bytes", u64), ("n_chunks", u64), ("kernels", u64), ("elapsed_ms", C.c_double)]
 
 
+class dr_ctl_config(C.Structure):
+    _fields_ = [("struct_size", u32), ("n_topologies", u32), ("initial", u32), ("consecutive", u32), ("dwell_steps", u32),
+                ("cooldown_steps", u32), ("enter_threshold", C.c_double), ("exit_threshold", C.c_double)]
+
+
 class DrError(RuntimeError):
     def __init__(self, status: int, where: str):
         self.status = status
@@ -113,6 +118,10 @@ def lib() -> C.CDLL:
         L.dr_reshard_stream.argtypes = [vp, P(dr_stream_desc), P(dr_stream_stats)]
         L.dr_plan_destroy.argtypes = [vp]
         L.dr_shard_range.argtypes = [u64, u32, u32, P(u64), P(u64), P(u64)]
+        L.dr_ctl_create.argtypes = [P(dr_ctl_config), P(vp)]
+        L.dr_ctl_observe.argtypes = [vp, C.c_double, C.c_double, P(C.c_int32), P(u32)]
+        L.dr_ctl_break_even.argtypes = [C.c_double, C.c_double, C.c_double, P(C.c_double)]
+        L.dr_ctl_destroy.argtypes = [vp]
         for n in EXPORTS:
             getattr(L, n).restype = C.c_int
         L.dr_strerror.argtypes = [C.c_int]
@@ -240,6 +249,29 @@ def dr_shard_range(flat_elems, world, rank):
     b, e, s = u64(), u64(), u64()
     rc = lib().dr_shard_range(flat_elems, world, rank, C.byref(b), C.byref(e), C.byref(s))
     return rc, b.value, e.value, s.value
+
+
+def dr_ctl_create(n_topologies, initial=0, enter=0.2, exit=0.1, consecutive=3, dwell=5, cooldown=11):
+    cfg = dr_ctl_config(struct_size=C.sizeof(dr_ctl_config), n_topologies=n_topologies, initial=initial,
+                        consecutive=consecutive, dwell_steps=dwell, cooldown_steps=cooldown, enter_threshold=enter,
+                        exit_threshold=exit)
+    h = vp()
+    return lib().dr_ctl_create(C.byref(cfg), C.byref(h)), h
+
+
+def dr_ctl_observe(ctl, t_rollout, t_train):
+    move, topo = C.c_int32(), u32()
+    rc = lib().dr_ctl_observe(ctl, t_rollout, t_train, C.byref(move), C.byref(topo))
+    return rc, move.value, topo.value
+
+
+def dr_ctl_break_even(resize_cost_s, step_before_s, step_after_s):
+    out = C.c_double()
+    return lib().dr_ctl_break_even(resize_cost_s, step_before_s, step_after_s, C.byref(out)), out.value
+
+
+def dr_ctl_destroy(ctl):
+    return lib().dr_ctl_destroy(ctl)
 
 
 def dr_plan_destroy(plan):
