@@ -419,7 +419,11 @@ def main():
 
     # ---- host-link sections ---------------------------------------------------------------------
     if not args.no_staging:
-        line.update(staging_sections(args, cfg, plans[0], master, arena, seed, base, dev, world, line, max_over_ranks))
+        try:
+            line.update(staging_sections(args, cfg, plans[0], master, arena, seed, base, dev, world, line, max_over_ranks))
+        except Exception as exc:  # e.g. the box cannot pin this much host memory: keep the device-side line
+            line.setdefault("staging", {})["error"] = f"{type(exc).__name__}: {exc}"[:300]
+            line.setdefault("e2e", {"value": None, "unit": "GB/s", "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0})
 
     if rank == 0 and not args.no_cpu and world == 1:
         gbs, elems, spent, desc = oracle_sample(cfg, args.cpu_seconds)
