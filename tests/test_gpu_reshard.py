@@ -195,3 +195,15 @@ def test_layout_variants_forward_and_inverse_match_oracle(spec, T, opts):
             torch.cuda.synchronize()
             assert first_diff(flat.cpu().numpy().view(np.uint32), wflat) is None
             plan.close()
+
+
+def test_empty_plan_launches_nothing_and_touches_nothing():
+    spec = dict(n_layers=0, hidden=4, n_q_heads=1, n_kv_heads=1, head_dim=2, ffn=4, vocab=2, tied=1, qk_norm=1)
+    p = dr.Plan(spec, world=16, rank=15, gathered=False)
+    src = torch.zeros(8, dtype=torch.int32, device=dev())
+    arena = arena_dev(max(p.info.dst_bytes, 16))
+    p.reshard(src, arena)
+    p.reshard_inverse(arena, src)
+    torch.cuda.synchronize()
+    assert (arena.cpu().numpy() == SENT8).all() and (src.cpu().numpy() == 0).all()
+    p.close()

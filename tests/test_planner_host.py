@@ -249,3 +249,13 @@ def test_fp8_plan_restrictions():
     assert e.value.status == E.DR_ERR_UNSUPPORTED
     p = dr.Plan(MID[0]["spec"], world=2, rank=1, gathered=True, dtype=dr.DR_FP8_E4M3_B128, host_only=True)
     assert p.info.quant_blocks > 0
+
+
+def test_plan_with_nothing_to_move():
+    """More ranks than elements: the last shards hold only padding, the plan is empty and still valid."""
+    spec = dict(n_layers=0, hidden=4, n_q_heads=1, n_kv_heads=1, head_dim=2, ffn=4, vocab=2, tied=1, qk_norm=1)
+    full = dr.Plan(spec, host_only=True)
+    assert full.info.flat_elems == 12
+    p = dr.Plan(spec, world=16, rank=15, gathered=False, host_only=True)
+    assert p.info.shard_elems == 1 and p.info.n_segments == 0 and p.info.n_tiles == 0 and p.info.elems_moved == 0
+    assert p.info.dst_bytes == full.info.dst_bytes
