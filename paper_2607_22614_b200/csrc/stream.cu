@@ -170,31 +170,37 @@ extern "C" int dr_reshard_stream(dr_plan* plan, const dr_stream_desc* d, dr_stre
     dr_stream_stats st{};
     st.n_chunks = s->chunks.size();
 
-    uint64_t copied_below = 0;  // arena bytes already on their way to host_dst
-    DR_CUDA(cudaEventRecord(s->ev_first, s->s_h2d));
-    for (uint64_t k = 0; k < s->chunks.size(); ++k) {
-        const ChunkTables& c = s->chunks[k];
-        const uint32_t slot = (uint32_t)(k % slots);
-        const uint64_t lo = k * chunk, n = std::min(chunk, plan->info.src_bytes - lo);
-        char* win = (char*)d->window_dev + (uint64_t)slot * chunk;
-        if (k >= slots) DR_CUDA(cudaStreamWaitEvent(s->s_h2d, s->ev_done[slot], 0));  // the slot's previous kernel
-        DR_CUDA(cudaMemcpyAsync(win, (const char*)d->host_src + lo, n, cudaMemcpyHostToDevice, s->s_h2d));
-        DR_CUDA(cudaEventRecord(s->ev_arrived[slot], s->s_h2d));
-        st.h2d_bytes += n;
-        DR_CUDA(cudaStreamWaitEvent(s->s_kernel, s->ev_arrived[slot], 0));
-        rc = launch_forward_tables(plan->elem_size, s->d_segs + c.seg_off, c.n_segs, s->d_hints + c.hint_off, c.hint_shift,
-                                   c.n_tiles, win, d->dst_dev, s->s_kernel);
-        if (rc) break;
-        if (c.n_tiles) ++st.kernels;
-        DR_CUDA(cudaEventRecord(s->ev_done[slot], s->s_kernel));
-        if (d->host_dst && c.final_below > copied_below) {
-            DR_CUDA(cudaStreamWaitEvent(s->s_d2h, s->ev_done[slot], 0));
-            DR_CUDA(cudaMemcpyAsync((char*)d->host_dst + copied_below, (const char*)d->dst_dev + copied_below,
-                                    c.final_below - copied_below, cudaMemcpyDeviceToHost, s->s_d2h));
-            st.d2h_bytes += c.final_below - copied_below;
-            copied_below = c.final_below;
+    // Everything is enqueued up front; a failure stops the enqueueing, and what was already enqueued is still
+    // waited for below, so that no copy or kernel of this call is in flight when it returns.
+    auto enqueue = [&]() -> int {
+        uint64_t copied_below = 0;  // arena bytes already on their way to host_dst
+        DR_CUDA(cudaEventRecord(s->ev_first, s->s_h2d));
+        for (uint64_t k = 0; k < s->chunks.size(); ++k) {
+            const ChunkTables& c = s->chunks[k];
+            const uint32_t slot = (uint32_t)(k % slots);
+            const uint64_t lo = k * chunk, n = std::min(chunk, plan->info.src_bytes - lo);
+            char* win = (char*)d->window_dev + (uint64_t)slot * chunk;
+            if (k >= slots) DR_CUDA(cudaStreamWaitEvent(s->s_h2d, s->ev_done[slot], 0));  // the slot's previous kernel
+            DR_CUDA(cudaMemcpyAsync(win, (const char*)d->host_src + lo, n, cudaMemcpyHostToDevice, s->s_h2d));
+            DR_CUDA(cudaEventRecord(s->ev_arrived[slot], s->s_h2d));
+            st.h2d_bytes += n;
+            DR_CUDA(cudaStreamWaitEvent(s->s_kernel, s->ev_arrived[slot], 0));
+            int krc = launch_forward_tables(plan->elem_size, s->d_segs + c.seg_off, c.n_segs, s->d_hints + c.hint_off,
+                                            c.hint_shift, c.n_tiles, win, d->dst_dev, s->s_kernel);
+            if (krc) return krc;
+            if (c.n_tiles) ++st.kernels;
+            DR_CUDA(cudaEventRecord(s->ev_done[slot], s->s_kernel));
+            if (d->host_dst && c.final_below > copied_below) {
+                DR_CUDA(cudaStreamWaitEvent(s->s_d2h, s->ev_done[slot], 0));
+                DR_CUDA(cudaMemcpyAsync((char*)d->host_dst + copied_below, (const char*)d->dst_dev + copied_below,
+                                        c.final_below - copied_below, cudaMemcpyDeviceToHost, s->s_d2h));
+                st.d2h_bytes += c.final_below - copied_below;
+                copied_below = c.final_below;
+            }
         }
-    }
+        return DR_OK;
+    };
+    rc = enqueue();
     // one bounded wait for the tail of each stream
     const auto limit = std::chrono::milliseconds(d->timeout_ms ? d->timeout_ms : 60000);
     const auto deadline = std::chrono::steady_clock::now() + limit;
