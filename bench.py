@@ -286,6 +286,10 @@ def main():
     else:
         plans = [dr.Plan(cfg["spec"], world=cfg["world"], rank=cfg["rank"], gathered=cfg["gathered"], tp=cfg["tp"],
                          tp_rank=cfg["tp_rank"])]
+    t0 = time.perf_counter()  # plan compile (host) + table upload: prepared ahead of a switch, not on its critical path
+    dr.Plan(cfg["spec"], world=cfg["world"], rank=cfg["rank"], gathered=cfg["gathered"], tp=cfg["tp"],
+            tp_rank=cfg["tp_rank"]).close()
+    plan_create_ms = (time.perf_counter() - t0) * 1e3
     info = plans[0].info
     n_src = info.src_bytes // 4
     bytes_fwd = sum(p.info.bytes_moved_fwd for p in plans)
@@ -362,7 +366,7 @@ def main():
                    "elements": int(info.elems_moved if halves == 1 else sum(p.info.elems_moved for p in plans)),
                    "bytes_per_step": int(step_bytes), "l2": "inputs larger than L2 (no flush needed)",
                    "passes": halves, "parallelism": "replicas only" if world > 1 else "1 GPU",
-                   "segments": int(info.n_segments), "tiles": int(info.n_tiles)},
+                   "segments": int(info.n_segments), "tiles": int(info.n_tiles), "plan_create_ms": plan_create_ms},
         "clocks": clocks,
         "gpu_launches": args.steps * (len(plans) + (1 if do_inverse else 0)),
         "forward": {"gbs_avg": ach, "gbs_best": bytes_fwd / min(fwd_ms) / 1e6, "ms_avg": fwd_avg, "ms_best": min(fwd_ms),

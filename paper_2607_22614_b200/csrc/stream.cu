@@ -51,6 +51,7 @@ namespace {
     do {                                                                         \
         cudaError_t e_ = (call);                                                 \
         if (e_ != cudaSuccess) {                                                 \
+            cudaGetLastError(); /* not sticky: clear it for later calls */      \
             set_error("%s: %s", #call, cudaGetErrorString(e_));                  \
             return e_ == cudaErrorMemoryAllocation ? DR_ERR_NOMEM : DR_ERR_CUDA; \
         }                                                                        \

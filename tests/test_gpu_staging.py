@@ -263,3 +263,25 @@ def test_host_offset_errors(plan):
     assert dr.dr_stage_out(plan.handle, mk([0, 2048]))[0] == B.DR_ERR_INVALID      # regions overlap
     assert dr.dr_stage_out(plan.handle, mk([0, 14000]))[0] == B.DR_ERR_SIZE        # runs past the arena
     assert dr.dr_stage_out(plan.handle, mk([8192, 0]))[0] == 0                     # any order of regions is fine
+
+
+def test_pinned_ring_allocation_failure_is_reported_and_the_plan_stays_usable(plan):
+    """A budget no machine can pin: the ring allocation fails on the host side, the call returns an
+    out-of-memory (or CUDA) error, nothing was copied, and the same plan still works afterwards."""
+    t = torch.arange(4096, dtype=torch.int32, device=dev())
+    host = np.zeros(16384, dtype=np.uint8)
+    d = dr.stage_desc([t.data_ptr()], [16384], budget=1 << 47, chunk=1 << 46, host_arena=host.ctypes.data,
+                      host_arena_bytes=host.size)
+    rc, st = dr.dr_stage_out(plan.handle, d)
+    assert rc in (B.DR_ERR_NOMEM, B.DR_ERR_CUDA) and st.bytes == 0
+    assert (host == 0).all()
+    d = dr.stage_desc([t.data_ptr()], [16384], budget=8192, chunk=4096, host_arena=host.ctypes.data, host_arena_bytes=host.size)
+    assert plan.stage_out(d).bytes == 16384
+    assert np.array_equal(host.view(np.int32), np.arange(4096, dtype=np.int32))
+    # and a kernel launch after the failed allocation sees no stale error
+    p2 = dr.Plan(MID[2]["spec"])
+    src = torch.zeros(p2.info.src_bytes // 4, dtype=torch.int32, device=dev())
+    arena = torch.zeros(p2.info.dst_bytes, dtype=torch.uint8, device=dev())
+    p2.reshard(src, arena)
+    torch.cuda.synchronize()
+    p2.close()
