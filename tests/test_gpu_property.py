@@ -13,7 +13,7 @@ from test_planner_property import cases
 pytestmark = pytest.mark.gpu
 
 
-@settings(max_examples=60, deadline=None, derandomize=True, suppress_health_check=list(HealthCheck))
+@settings(max_examples=60, deadline=None, derandomize=True, database=None, suppress_health_check=list(HealthCheck))
 @given(cases())
 def test_random_plans_on_the_gpu(c):
     es = 2 if c["dtype"] == dr.DR_BF16 else 4
@@ -71,7 +71,7 @@ def staging_cases(draw):
     return dict(sizes=sizes, chunk=chunk, budget=chunk * slots + draw(st.integers(0, chunk - 1)), sink=sink, order=list(order))
 
 
-@settings(max_examples=40, deadline=None, derandomize=True, suppress_health_check=list(HealthCheck))
+@settings(max_examples=40, deadline=None, derandomize=True, database=None, suppress_health_check=list(HealthCheck))
 @given(staging_cases())
 def test_random_staging_geometries(c):
     """Random buffer sizes (odd byte counts included), chunk sizes, slot counts, sinks and restore orders:
