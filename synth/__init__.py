@@ -60,9 +60,11 @@ def bits(seed: int, buffer_id: int, index: int) -> int:
     return int(_h().synth_bits(seed, buffer_id, index))
 
 
-def fill_f32(seed: int, buffer_id: int, start: int, n: int) -> np.ndarray:
-    """uint32 bit patterns of fp32 elements start..start+n."""
-    out = np.empty(n, dtype=np.uint32)
+def fill_f32(seed: int, buffer_id: int, start: int, n: int, out: np.ndarray | None = None) -> np.ndarray:
+    """uint32 bit patterns of fp32 elements start..start+n (written into ``out`` when given)."""
+    if out is None:
+        out = np.empty(n, dtype=np.uint32)
+    assert out.dtype == np.uint32 and out.size == n and out.flags.c_contiguous
     _h().synth_fill_f32(out.ctypes.data, seed, buffer_id, start, n)
     return out
 

@@ -169,3 +169,114 @@ def test_cfg4_moe_two_half_shards_sampled():
     slots = torch.from_numpy(_arena_slots(om, ti, rows, cols)).to(DEV)
     got = arena.view(torch.int16)[slots].cpu().numpy().view(np.uint16)
     assert np.array_equal(got, want)
+
+
+def _host_room_gb():
+    with open("/proc/meminfo") as f:
+        for line in f:
+            if line.startswith("MemAvailable:"):
+                return int(line.split()[1]) / 1e6
+    return 0
+
+
+def test_cfg2_whole_arena_equals_oracle():
+    """All 8.19 G elements of the Qwen3-8B-shaped switch against the oracle (needs about 70 GB of host memory)."""
+    _need(55)
+    if _host_room_gb() < 90:
+        pytest.skip("needs 90 GB of free host memory")
+    cfg = CONFIGS[2]
+    plan, om = _models(cfg)
+    seed = seed_of(2)
+    src = torch.empty(plan.info.src_bytes // 4, dtype=torch.int32, device=DEV)
+    synth.cuda_fill_f32(src, seed, synth.BUF_MASTER)
+    arena = torch.full((plan.info.dst_bytes,), 0xA5, dtype=torch.uint8, device=DEV)
+    plan.reshard(src, arena)
+    torch.cuda.synchronize()
+    del src
+    flat = synth.fill_f32(seed, synth.BUF_MASTER, 0, om.flat_elems)
+    want = np.full(om.arena_bytes, 0xA5, dtype=np.uint8)
+    om.forward(flat, want)
+    del flat
+    got = arena.cpu().numpy()
+    assert np.array_equal(got, want)
+    plan.close()
+
+
+def test_cfg3_whole_shard_equals_oracle_inverse():
+    """The complete Rollout -> Training result of the Qwen3-14B-shaped workload: every word of FSDP shard 1 of 4,
+    written or not, against the oracle's inverse."""
+    _need(26)
+    if _host_room_gb() < 50:
+        pytest.skip("needs 50 GB of free host memory")
+    cfg = CONFIGS[3]
+    plan, om = _models(cfg)
+    seed = seed_of(3)
+    S, r = plan.info.shard_elems, cfg["rank"]
+    arena = torch.empty(plan.info.dst_bytes // 2, dtype=torch.int16, device=DEV)
+    synth.cuda_fill_bf16(arena, seed, synth.BUF_ROLLOUT)
+    sent = 0xDEADBEEF - (1 << 32)
+    flat = torch.full((S,), sent, dtype=torch.int32, device=DEV)
+    plan.reshard_inverse(arena, flat)
+    torch.cuda.synchronize()
+    del arena
+    h_arena = synth.fill_bf16(seed, synth.BUF_ROLLOUT, 0, om.arena_bytes // 2).view(np.uint8)
+    want = np.full(S, 0xDEADBEEF, dtype=np.uint32)
+    om.inverse(h_arena, want, gathered=False, rank=r)
+    assert np.array_equal(flat.cpu().numpy().view(np.uint32), want)
+    plan.close()
+
+
+def test_cfg4_whole_arena_equals_oracle_streamed_by_layer():
+    """All 29.8 G elements of the Qwen3-30B-A3B-shaped MoE switch.  Neither the 122 GB source nor the 59.5 GB
+    arena is held on the host: the oracle runs tensor by tensor on lazily committed mappings, one layer's
+    source at a time, and each rollout tensor is compared and released."""
+    import mmap
+    _need(125)
+    if _host_room_gb() < 24:
+        pytest.skip("needs 24 GB of free host memory")
+    cfg = CONFIGS[4]
+    seed = seed_of(4)
+    om = oracle.Model(cfg["spec"], world=2, tp=cfg["tp"], tp_rank=cfg["tp_rank"])
+    S = om.shard_elems
+    arena = torch.full((om.arena_bytes,), 0xA5, dtype=torch.uint8, device=DEV)
+    shard = torch.empty(S, dtype=torch.int32, device=DEV)
+    for half in (0, 1):
+        plan, _ = _models(cfg, world=2, rank=half, gathered=False)
+        synth.cuda_fill_f32(shard, seed, synth.BUF_MASTER, start=half * S)
+        plan.reshard(shard, arena)
+        torch.cuda.synchronize()
+        plan.close()
+    del shard
+    page = mmap.PAGESIZE
+    mm_src = mmap.mmap(-1, -(-4 * 2 * S // page) * page)
+    mm_dst = mmap.mmap(-1, -(-om.arena_bytes // page) * page)
+    flat = np.frombuffer(mm_src, dtype=np.uint32)
+    want = np.frombuffer(mm_dst, dtype=np.uint8)
+
+    def release(mm, lo, hi):  # give whole pages inside [lo, hi) back
+        a, b = -(-lo // page) * page, hi // page * page
+        if b > a:
+            mm.madvise(mmap.MADV_DONTNEED, a, b - a)
+
+    srcs = om.src_tensors()
+    dst = om.dst_tensors()
+    groups = ["embed"] + [f"layers.{l}." for l in range(cfg["spec"]["n_layers"])] + ["final_norm", "lm_head"]
+    checked = 0
+    for g in groups:
+        mine = [s for s in srcs if s.name == g or (g.endswith(".") and s.name.startswith(g))]
+        lo = min(s.flat_off for s in mine)
+        hi = max(s.flat_off + s.rows * s.cols for s in mine)
+        synth.fill_f32(seed, synth.BUF_MASTER, lo, hi - lo, out=flat[lo:hi])
+        for i, d in enumerate(dst):
+            if d.alias_of >= 0 or not (d.name == g or (g.endswith(".") and d.name.startswith(g))):
+                continue
+            nbytes = d.rows * d.cols * 2
+            want[d.arena_off:d.arena_off + nbytes] = 0xA5
+            om.forward(flat, want, gathered=True, only=i)
+            got = arena[d.arena_off:d.arena_off + nbytes].cpu().numpy()
+            assert np.array_equal(got, want[d.arena_off:d.arena_off + nbytes]), d.name
+            release(mm_dst, d.arena_off, d.arena_off + nbytes)
+            checked += d.rows * d.cols
+        release(mm_src, 4 * lo, 4 * hi)
+    assert checked == 29_767_972_864
+    del flat, want
