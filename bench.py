@@ -392,6 +392,26 @@ def main():
             ok &= torch.equal(arena.view(torch.bfloat16)[lo:lo + w], master.view(torch.float32)[lo:lo + w].to(torch.bfloat16))
         line["config"]["output_equals_torch_cast_on_windows"] = bool(ok)
 
+    # context: what torch's own streaming kernels reach on this GPU in this run (the measured-peak file is a
+    # torch copy too); 1 Gi-element buffers, best of 5
+    if halves == 1 and n_src >= (1 << 30):
+        a16, b16 = master.view(torch.bfloat16)[:1 << 30], arena.view(torch.bfloat16)[:1 << 30] if info.dst_bytes >= (2 << 30) else None
+        def best(fn, nbytes):
+            ts = []
+            for _ in range(5):
+                e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+                e0.record(); fn(); e1.record(); torch.cuda.synchronize()
+                ts.append(e0.elapsed_time(e1))
+            return nbytes / min(ts) / 1e6
+        ctx_peaks = {"torch_read_sum_gbs": best(lambda: master.view(torch.float32)[:1 << 30].sum(), 4 << 30)}
+        if b16 is not None:
+            saved = b16.clone()
+            ctx_peaks["torch_copy_gbs"] = best(lambda: b16.copy_(a16), 4 << 30)
+            ctx_peaks["torch_fill_gbs"] = best(lambda: b16.zero_(), 2 << 30)
+            b16.copy_(saved)
+            del saved
+        line["context_ceilings"] = ctx_peaks
+
     del flat_back
     torch.cuda.empty_cache()
 

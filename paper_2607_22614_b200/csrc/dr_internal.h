@@ -122,6 +122,18 @@ struct dr_plan {
     dr::Stream* stream = nullptr;
 };
 
+// Run a CUDA runtime call inside a function (or lambda) that returns a dr_status; on failure record the
+// message, clear the (non-sticky) error so that later launches do not see it, and return.
+#define DR_CUDA(call)                                                             \
+    do {                                                                          \
+        cudaError_t e_ = (call);                                                  \
+        if (e_ != cudaSuccess) {                                                  \
+            cudaGetLastError();                                                   \
+            dr::set_error("%s: %s", #call, cudaGetErrorString(e_));               \
+            return e_ == cudaErrorMemoryAllocation ? DR_ERR_NOMEM : DR_ERR_CUDA;  \
+        }                                                                         \
+    } while (0)
+
 namespace dr {
 
 void set_error(const char* fmt, ...);

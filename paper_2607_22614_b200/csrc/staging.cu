@@ -48,16 +48,6 @@ void ring_destroy(Ring* r)
 
 namespace {
 
-#define DR_CUDA(call)                                                        \
-    do {                                                                     \
-        cudaError_t e_ = (call);                                             \
-        if (e_ != cudaSuccess) {                                             \
-            cudaGetLastError(); /* not sticky: clear it for later calls */  \
-            set_error("%s: %s", #call, cudaGetErrorString(e_));              \
-            return e_ == cudaErrorMemoryAllocation ? DR_ERR_NOMEM : DR_ERR_CUDA; \
-        }                                                                    \
-    } while (0)
-
 struct Geometry {
     uint64_t total = 0, chunk = 0, n_chunks = 0;
     uint32_t slots = 0;

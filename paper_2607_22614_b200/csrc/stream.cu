@@ -47,16 +47,6 @@ void stream_destroy(Stream* s)
 
 namespace {
 
-#define DR_CUDA(call)                                                            \
-    do {                                                                         \
-        cudaError_t e_ = (call);                                                 \
-        if (e_ != cudaSuccess) {                                                 \
-            cudaGetLastError(); /* not sticky: clear it for later calls */      \
-            set_error("%s: %s", #call, cudaGetErrorString(e_));                  \
-            return e_ == cudaErrorMemoryAllocation ? DR_ERR_NOMEM : DR_ERR_CUDA; \
-        }                                                                        \
-    } while (0)
-
 // Per-chunk tables for a given chunk size, compiled once and kept on the device.
 int prepare(dr_plan* p, uint64_t chunk_bytes, uint32_t slots)
 {

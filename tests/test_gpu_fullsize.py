@@ -280,3 +280,30 @@ def test_cfg4_whole_arena_equals_oracle_streamed_by_layer():
         release(mm_src, 4 * lo, 4 * hi)
     assert checked == 29_767_972_864
     del flat, want
+
+
+def test_cfg1_streamed_repack_equals_resident_repack():
+    """The 6.9 GB source of the Qwen3-1.7B-shaped workload streamed from pinned host memory through a 512 MiB
+    window: the arena on the device and its copy on the host equal the resident dr_reshard result
+    (itself compared whole with the oracle above)."""
+    _need(12)
+    cfg = CONFIGS[1]
+    plan, om = _models(cfg)
+    seed = seed_of(1)
+    src = torch.empty(plan.info.src_bytes // 4, dtype=torch.int32, device=DEV)
+    synth.cuda_fill_f32(src, seed, synth.BUF_MASTER)
+    ref = torch.full((plan.info.dst_bytes,), 0xA5, dtype=torch.uint8, device=DEV)
+    plan.reshard(src, ref)
+    h_src = torch.empty(plan.info.src_bytes, dtype=torch.uint8, pin_memory=True)
+    h_src.copy_(src.view(torch.uint8))
+    del src
+    h_dst = torch.zeros(plan.info.dst_bytes, dtype=torch.uint8, pin_memory=True)
+    arena = torch.full((plan.info.dst_bytes,), 0xA5, dtype=torch.uint8, device=DEV)
+    window = torch.empty(512 << 20, dtype=torch.uint8, device=DEV)
+    st = plan.reshard_stream(dr.stream_desc(h_src.data_ptr(), plan.info.src_bytes, arena.data_ptr(), plan.info.dst_bytes,
+                                            window.data_ptr(), 512 << 20, chunk_bytes=64 << 20, host_dst=h_dst.data_ptr(),
+                                            host_dst_bytes=plan.info.dst_bytes))
+    assert st.n_chunks == -(-plan.info.src_bytes // (64 << 20)) and st.d2h_bytes == plan.info.dst_bytes
+    assert torch.equal(arena, ref)
+    assert torch.equal(h_dst, ref.cpu())
+    plan.close()
