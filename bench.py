@@ -189,6 +189,7 @@ def oracle_sample(cfg, seconds: float, max_layers: int = 1 << 30):
         flat[lo:hi] = synth.fill_f32(seed, synth.BUF_MASTER, lo, hi - lo)
         for i, d in enumerate(dst):
             if d.name.startswith(f"layers.{layer}.") and d.alias_of < 0:
+                arena[d.arena_off:d.arena_off + d.rows * d.cols * 2].fill(0)  # commit the output pages before timing
                 t0 = time.perf_counter()
                 om.forward(flat, arena, gathered=True, only=i)
                 spent += time.perf_counter() - t0
@@ -198,6 +199,42 @@ def oracle_sample(cfg, seconds: float, max_layers: int = 1 << 30):
             break
     gbs = elems * 6 / spent / 1e9
     return gbs, elems, spent, f"forward transform of rollout layers 0..{layers - 1} of {cfg['name']} ({elems} elements)"
+
+
+def oracle_sample_all_cores(cfg, layers: int = 8):
+    """The same oracle, one thread per rollout tensor over all host cores (the C loop releases the GIL):
+    layers 0..layers-1 of the workload.  Returns (GB/s, threads, elements, seconds)."""
+    from concurrent.futures import ThreadPoolExecutor
+
+    import numpy as np
+
+    import oracle
+    import synth
+
+    om = oracle.Model(cfg["spec"], world=cfg["world"], tp=cfg["tp"], tp_rank=cfg["tp_rank"])
+    srcs = {s.name: s for s in om.src_tensors()}
+    flat = np.empty(om.world * om.shard_elems, dtype=np.uint32)
+    arena = np.empty(om.arena_bytes, dtype=np.uint8)
+    seed = synth.SEED_BASE + cfg["index"]
+    layers = min(layers, cfg["spec"]["n_layers"])
+    work = []
+    for layer in range(layers):
+        names = [n for n in srcs if n.startswith(f"layers.{layer}.")]
+        lo = min(srcs[n].flat_off for n in names)
+        hi = max(srcs[n].flat_off + srcs[n].rows * srcs[n].cols for n in names)
+        synth.fill_f32(seed, synth.BUF_MASTER, lo, hi - lo, out=flat[lo:hi])
+        for i, d in enumerate(om.dst_tensors()):
+            if d.name.startswith(f"layers.{layer}.") and d.alias_of < 0:
+                arena[d.arena_off:d.arena_off + d.rows * d.cols * 2].fill(0)  # commit the output pages before timing
+                work.append((i, d.rows * d.cols))
+    work.sort(key=lambda w: -w[1])  # big tensors first
+    threads = os.cpu_count() or 1
+    t0 = time.perf_counter()
+    with ThreadPoolExecutor(max_workers=threads) as ex:
+        list(ex.map(lambda w: om.forward(flat, arena, gathered=True, only=w[0]), work))
+    spent = time.perf_counter() - t0
+    elems = sum(w[1] for w in work)
+    return elems * 6 / spent / 1e9, threads, elems, spent
 
 
 def run_reference(args, cfg):
@@ -453,6 +490,10 @@ def main():
         gbs, elems, spent, desc = oracle_sample(cfg, args.cpu_seconds)
         line["cpu_baseline"] = {"value": gbs, "unit": "GB/s", "cores": 1, "kind": "oracle", "sample": desc,
                                 "seconds": spent}
+        g2, threads, e2, s2 = oracle_sample_all_cores(cfg)
+        line["cpu_baseline_all_cores"] = {"value": g2, "unit": "GB/s", "cores": threads, "kind": "oracle",
+                                          "sample": f"the same oracle, one thread per rollout tensor, {e2} elements",
+                                          "seconds": s2}
     for p in plans:
         p.close()
     ctx.close()
