@@ -166,6 +166,12 @@ int dr_plan_create(const dr_model_spec* spec, const dr_src_layout* src, const dr
 int dr_plan_create_host(const dr_model_spec* spec, const dr_src_layout* src, const dr_dst_layout* dst, uint32_t tp,
                         uint32_t rank, dr_plan** out);
 
+/* The part of `plan` whose source elements lie in [src_elem_lo, src_elem_hi) of the buffer the plan reads,
+ * as a host-only plan whose source buffer is that window alone (what one chunk of dr_reshard_stream
+ * repacks).  For inspection and checks; not for fp8 plans (DR_ERR_UNSUPPORTED).  DR_ERR_INVALID if the
+ * window is empty or leaves the source buffer. */
+int dr_plan_window_host(const dr_plan* plan, uint64_t src_elem_lo, uint64_t src_elem_hi, dr_plan** out);
+
 int dr_plan_query(const dr_plan* plan, dr_plan_info* out);
 int dr_plan_tensor(const dr_plan* plan, uint32_t i, dr_tensor_desc* out);   /* DR_ERR_INVALID if i >= n_tensors  */
 int dr_plan_segment(const dr_plan* plan, uint64_t i, dr_segment_desc* out); /* DR_ERR_INVALID if i >= n_segments */

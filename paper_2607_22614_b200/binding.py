@@ -17,7 +17,7 @@ DR_F32, DR_BF16, DR_FP8_E4M3_B128 = 1, 2, 3
 DR_MAX_STAGE_BUFS = 8
 DR_STAGE_HOST_OFFSETS = 1
 
-EXPORTS = ["dr_plan_create", "dr_plan_create_host", "dr_plan_query", "dr_plan_tensor", "dr_plan_segment",
+EXPORTS = ["dr_plan_create", "dr_plan_create_host", "dr_plan_window_host", "dr_plan_query", "dr_plan_tensor", "dr_plan_segment",
            "dr_reshard", "dr_reshard_inverse", "dr_reshard_static", "dr_reshard_stream", "dr_shard_range", "dr_stage_out", "dr_stage_in", "dr_plan_destroy", "dr_strerror",
            "dr_last_error", "dr_ctl_create", "dr_ctl_observe", "dr_ctl_break_even", "dr_ctl_destroy"]
 
@@ -107,6 +107,7 @@ def lib() -> C.CDLL:
         P = C.POINTER
         L.dr_plan_create.argtypes = [P(dr_model_spec), P(dr_src_layout), P(dr_dst_layout), u32, u32, P(vp)]
         L.dr_plan_create_host.argtypes = L.dr_plan_create.argtypes
+        L.dr_plan_window_host.argtypes = [vp, u64, u64, P(vp)]
         L.dr_plan_query.argtypes = [vp, P(dr_plan_info)]
         L.dr_plan_tensor.argtypes = [vp, u32, P(dr_tensor_desc)]
         L.dr_plan_segment.argtypes = [vp, u64, P(dr_segment_desc)]
@@ -191,6 +192,11 @@ def dr_plan_create_host(spec, src, dst, tp, rank):
     h = vp()
     rc = lib().dr_plan_create_host(C.byref(spec), C.byref(src), C.byref(dst), tp, rank, C.byref(h))
     return rc, h
+
+
+def dr_plan_window_host(plan, src_elem_lo, src_elem_hi):
+    h = vp()
+    return lib().dr_plan_window_host(plan, src_elem_lo, src_elem_hi, C.byref(h)), h
 
 
 def dr_plan_query(plan):
@@ -303,6 +309,16 @@ class Plan:
         rc, self.info = dr_plan_query(self.handle)
         if rc:
             raise DrError(rc, "dr_plan_query")
+
+    def window(self, src_elem_lo, src_elem_hi):
+        """Host-only plan for the source window [lo, hi) (what one chunk of the streamed repack covers)."""
+        rc, h = dr_plan_window_host(self.handle, src_elem_lo, src_elem_hi)
+        if rc:
+            raise DrError(rc, "dr_plan_window_host")
+        w = Plan.__new__(Plan)
+        w.handle = h
+        rc, w.info = dr_plan_query(h)
+        return w
 
     def close(self):
         if getattr(self, "handle", None):

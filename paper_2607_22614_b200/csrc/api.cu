@@ -182,6 +182,58 @@ int dr_plan_create_host(const dr_model_spec* spec, const dr_src_layout* src, con
     return create(spec, src, dst, tp, rank, true, out);
 }
 
+int dr_plan_window_host(const dr_plan* plan, uint64_t src_elem_lo, uint64_t src_elem_hi, dr_plan** out)
+{
+    if (!plan || !out) {
+        set_error("NULL argument");
+        return DR_ERR_INVALID;
+    }
+    *out = nullptr;
+    if (plan->fp8) {
+        set_error("fp8 plans have no source windows");
+        return DR_ERR_UNSUPPORTED;
+    }
+    if (src_elem_lo >= src_elem_hi || src_elem_hi > plan->info.src_bytes / 4) {
+        set_error("window is empty or outside the source buffer");
+        return DR_ERR_INVALID;
+    }
+    dr_plan* w = new (std::nothrow) dr_plan();
+    if (!w) return DR_ERR_NOMEM;
+    w->spec = plan->spec;
+    w->src = plan->src;
+    w->dst = plan->dst;
+    w->tp = plan->tp;
+    w->tp_rank = plan->tp_rank;
+    w->elem_size = plan->elem_size;
+    w->host_only = true;
+    int rc = DR_OK;
+    try {
+        w->tensors = plan->tensors;
+        w->segs = window_segments(plan->segs, src_elem_lo, src_elem_hi, plan->elem_size);
+        Tables tb;
+        rc = build_tables(w->segs, &tb);
+        if (rc == DR_OK) {
+            w->dev_segs.swap(tb.segs);
+            w->hints.swap(tb.hints);
+            w->hint_shift = tb.hint_shift;
+            w->info = plan->info;
+            w->info.src_bytes = 4 * (src_elem_hi - src_elem_lo);
+            w->info.n_segments = w->segs.size();
+            w->info.n_tiles = tb.n_tiles;
+            w->info.elems_moved = tb.elems;
+            w->info.bytes_moved_fwd = w->info.bytes_moved_inv = tb.elems * (4 + plan->elem_size);
+        }
+    } catch (const std::bad_alloc&) {
+        rc = DR_ERR_NOMEM;
+    }
+    if (rc) {
+        dr_plan_destroy(w);
+        return rc;
+    }
+    *out = w;
+    return DR_OK;
+}
+
 int dr_plan_query(const dr_plan* plan, dr_plan_info* out)
 {
     if (!plan || !out) {

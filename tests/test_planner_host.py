@@ -259,3 +259,33 @@ def test_plan_with_nothing_to_move():
     p = dr.Plan(spec, world=16, rank=15, gathered=False, host_only=True)
     assert p.info.shard_elems == 1 and p.info.n_segments == 0 and p.info.n_tiles == 0 and p.info.elems_moved == 0
     assert p.info.dst_bytes == full.info.dst_bytes
+
+
+@pytest.mark.parametrize("spec,kw,chunk", [
+    (MID[0]["spec"], dict(tp=2, tp_rank=1), 2_499_992), (MID[2]["spec"], dict(tp=2, tp_rank=0, moe_ep=2, moe_ep_rank=1), 1_000_003),
+    (BRUTE[0]["spec"], dict(tp=2, tp_rank=1, align_elems=3), 16), (MID[1]["spec"], dict(world=3, rank=1, gathered=False, tp=2), 600_001),
+    (BRUTE[2]["spec"], dict(dtype=dr.DR_F32), 7)], ids=["dense-tp2", "moe-ep", "brute", "shard-local", "brute-moe-f32"])
+def test_source_windows_partition_the_plan(spec, kw, chunk):
+    """The per-chunk plans of the streamed repack: together they write exactly what the whole plan writes, each
+    from inside its own window, and nothing twice."""
+    es = 4 if kw.get("dtype") == dr.DR_F32 else 2
+    p = dr.Plan(spec, arena_align_bytes=64, host_only=True, **kw)
+    whole = expand(p, es)
+    n_src = p.info.src_bytes // 4
+    union = np.full_like(whole, -1)
+    moved = 0
+    for lo in range(0, n_src, chunk):
+        hi = min(lo + chunk, n_src)
+        w = p.window(lo, hi)
+        assert w.info.src_bytes == 4 * (hi - lo) and w.info.dst_bytes == p.info.dst_bytes
+        m = expand(w, es)                      # indices relative to the window
+        hit = m >= 0
+        assert (m[hit] < hi - lo).all()
+        assert (union[hit] == -1).all()        # no arena element comes from two windows
+        union[hit] = m[hit] + lo
+        moved += w.info.elems_moved
+        w.close()
+    assert np.array_equal(union, whole) and moved == p.info.elems_moved
+    assert dr.dr_plan_window_host(p.handle, 5, 5)[0] == dr.binding.DR_ERR_INVALID
+    assert dr.dr_plan_window_host(p.handle, 0, n_src + 1)[0] == dr.binding.DR_ERR_INVALID
+    p.close()
