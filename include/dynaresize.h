@@ -186,7 +186,9 @@ int dr_plan_segment(const dr_plan* plan, uint64_t i, dr_segment_desc* out); /* D
  * subnormals are rounded, not flushed), or a bit copy when the plan's dst dtype is DR_F32.
  * Errors (all found before launch): DR_ERR_SIZE if src_bytes / dst_bytes are below the plan's
  * requirement, DR_ERR_ALIGN if a base pointer is not 16-byte aligned, DR_ERR_STATE, DR_ERR_CUDA.
- * The plan is not modified: concurrent calls on different streams are allowed.
+ * The plan is not modified: concurrent calls on different streams are allowed.  The call only enqueues
+ * kernels, so (after one ordinary call has loaded the module) it may be recorded into a CUDA graph by
+ * stream capture and replayed; the same holds for dr_reshard_inverse.
  */
 int dr_reshard(const dr_plan* plan, const void* src_dev, uint64_t src_bytes, void* dst_dev, uint64_t dst_bytes,
                void* cuda_stream);

@@ -207,3 +207,58 @@ def test_empty_plan_launches_nothing_and_touches_nothing():
     torch.cuda.synchronize()
     assert (arena.cpu().numpy() == SENT8).all() and (src.cpu().numpy() == 0).all()
     p.close()
+
+
+def test_one_plan_on_two_streams_at_once():
+    """A plan is immutable: two repacks of different sources run concurrently on two streams."""
+    spec = MID[0]["spec"]
+    plan = dr.Plan(spec, tp=2, tp_rank=0)
+    om = oracle.Model(spec, tp=2, tp_rank=0)
+    srcs = [make_source(om.flat_elems, s) for s in (91, 92)]
+    wants = []
+    for s in srcs:
+        w = np.full(om.arena_bytes, SENT8, dtype=np.uint8)
+        om.forward(s, w)
+        wants.append(w)
+    devs = [to_dev_u32(s) for s in srcs]
+    arenas = [arena_dev(om.arena_bytes) for _ in srcs]
+    streams = [torch.cuda.Stream(), torch.cuda.Stream()]
+    torch.cuda.synchronize()
+    for _ in range(3):
+        for d, a, st in zip(devs, arenas, streams):
+            plan.reshard(d, a, stream=st)
+    torch.cuda.synchronize()
+    for a, w in zip(arenas, wants):
+        assert first_diff(a.cpu().numpy(), w) is None
+    plan.close()
+
+
+def test_repack_and_inverse_replay_from_a_cuda_graph():
+    """dr_reshard / dr_reshard_inverse only enqueue kernels, so a switch can be captured once and replayed."""
+    spec = MID[2]["spec"]
+    plan = dr.Plan(spec, tp=2, tp_rank=1)
+    om = oracle.Model(spec, tp=2, tp_rank=1)
+    src = to_dev_u32(make_source(om.flat_elems, 93))
+    arena = arena_dev(om.arena_bytes)
+    back = torch.full((om.flat_elems,), 0x5A5A5A5A, dtype=torch.int32, device=dev())
+    plan.reshard(src, arena)          # warm-up outside the capture (module load)
+    torch.cuda.synchronize()
+    arena.fill_(SENT8)
+    graph = torch.cuda.CUDAGraph()
+    with torch.cuda.graph(graph):
+        plan.reshard(src, arena)      # enqueued on the capturing stream (the current stream inside the context)
+        plan.reshard_inverse(arena, back)
+    torch.cuda.synchronize()
+    assert (arena.cpu().numpy() == SENT8).all()   # capture enqueues nothing
+    for seed in (94, 95):             # new weights in the same buffers, same graph
+        host = make_source(om.flat_elems, seed)
+        src.copy_(torch.from_numpy(host.view(np.int32)))
+        graph.replay()
+        torch.cuda.synchronize()
+        want = np.full(om.arena_bytes, SENT8, dtype=np.uint8)
+        om.forward(host, want)
+        assert first_diff(arena.cpu().numpy(), want) is None
+        wflat = np.full(om.flat_elems, 0x5A5A5A5A, dtype=np.uint32)
+        om.inverse(want, wflat)
+        assert first_diff(back.cpu().numpy().view(np.uint32), wflat) is None
+    plan.close()
