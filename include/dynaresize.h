@@ -1,17 +1,18 @@
 /*
  * dynaresize.h -- C ABI of the per-GPU role-switch state transform for sm_100a (B200).
  *
- * When runtime GPU reallocation turns a Training GPU into a Rollout GPU (or back), the GPU must
- * "flush old parameters and ingest new weights and optimizer states" (paper Sec. 1, challenge 2) and
- * "reload the states required by the new topology" (Sec. 3.3).  This library is that per-GPU step:
+ * When runtime GPU reallocation turns a Training GPU into a Rollout GPU (or back), the GPU has to drop
+ * the state of its old role and take in the weights and optimizer state of the new one (paper Sec. 1,
+ * challenge 2), i.e. bring in whatever state the new topology asks for (Sec. 3.3).  This library is
+ * that per-GPU step:
  *
  *   Training -> Rollout : read the FSDP-style flat fp32 master buffer, un-flatten it, fuse Q/K/V and
  *                         gate/up, slice for a tensor-parallel degree and rank, cast to bf16
  *                         (round to nearest, ties to even) into a contiguous rollout arena;
  *   Rollout -> Training : the inverse layout map (bf16 widened exactly to fp32);
  *   both directions     : stream optimizer state (fp32 master, Adam m, Adam v) to and from host
- *                         memory in fixed chunks through a bounded pinned ring (the "chunked
- *                         streaming ... through host-memory buffers" of Sec. 3.3), weights first
+ *                         memory in fixed chunks through a bounded pinned ring (the chunk-wise
+ *                         streaming through host buffers of Sec. 3.3), weights first
  *                         on the way back (the deferred optimizer reload of Sec. 3.3).
  *
  * Conventions
@@ -177,7 +178,7 @@ int dr_plan_tensor(const dr_plan* plan, uint32_t i, dr_tensor_desc* out);   /* D
 int dr_plan_segment(const dr_plan* plan, uint64_t i, dr_segment_desc* out); /* DR_ERR_INVALID if i >= n_segments */
 
 /*
- * dr_reshard -- Training -> Rollout (Sec. 1 challenge 2: "ingest new weights").  Enqueues the
+ * dr_reshard -- Training -> Rollout (Sec. 1 challenge 2: taking in the new role's weights).  Enqueues the
  * gather / cast kernel on cuda_stream and returns; nothing is synchronised.
  *   src_dev : fp32 flat buffer (whole, or this rank's shard when gathered = 0), read only
  *   dst_dev : rollout arena; only mapped elements are written, gaps and (for gathered = 0) elements
@@ -194,8 +195,8 @@ int dr_reshard(const dr_plan* plan, const void* src_dev, uint64_t src_bytes, voi
                void* cuda_stream);
 
 /*
- * dr_reshard_inverse -- Rollout -> Training (Sec. 3.3: "reload the states required by the new
- * topology").  Scatters the rollout arena back to the flat positions it was taken from, widening
+ * dr_reshard_inverse -- Rollout -> Training (Sec. 3.3: bringing back the state the new topology
+ * needs)..  Scatters the rollout arena back to the flat positions it was taken from, widening
  * bf16 to fp32 exactly (bits << 16).  Only positions covered by this TP rank (and, for gathered = 0,
  * lying in this shard) are written; padding and everything else keep their bytes.  Asynchronous on
  * cuda_stream; same errors as dr_reshard.
@@ -313,7 +314,7 @@ int dr_stage_in(dr_plan* plan, const dr_stage_desc* desc, dr_stage_stats* stats)
  * chunk can write into it.  Host-to-device copies, the repack kernels and device-to-host copies run on
  * three streams and overlap, so the whole switch takes about as long as the larger of the two copy
  * directions; the device never holds more than the window of fp32 state (the bounded staging of Sec. 3.3
- * applied to the device side, with the "asynchronous overlapping of independent operations" of Sec. 3.3).
+ * applied to the device side, and Sec. 3.3's overlap of operations that do not depend on one another).
  */
 typedef struct dr_stream_desc {
     uint32_t struct_size, flags;  /* sizeof(dr_stream_desc), 0                                         */

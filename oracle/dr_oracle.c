@@ -2,9 +2,10 @@
  * TEST INFRASTRUCTURE -- NOT PART OF THE PRODUCT PATH.
  *
  * Plain, slow, single-threaded CPU statement of the per-GPU state transform
- * that a Training<->Rollout role switch needs ("flush old parameters and
- * ingest new weights and optimizer states", paper Sec. 1 challenge 2; "reload
- * the states required by the new topology", Sec. 3.3) and of the bounded
+ * that a Training<->Rollout role switch needs (dropping the old role's
+ * parameters and taking in the new role's weights and optimizer state, paper
+ * Sec. 1 challenge 2; bringing in the state the new topology asks for,
+ * Sec. 3.3) and of the bounded
  * chunked host staging of Sec. 3.3.  The paper gives no formula for the
  * layout map, so the definitions D1-D6 below are the ones this repository
  * adopts; every one is written out element by element, with no segment
