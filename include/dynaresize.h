@@ -148,7 +148,7 @@ typedef struct dr_segment_desc {
     uint64_t src_off;  /* elements, relative to the source buffer the call receives                 */
     uint64_t rows, row_len, src_row_stride, dst_row_stride; /* elements                              */
     uint32_t vector_bytes; /* 32 / 16: source access width the kernel may use; 0: scalar path        */
-    uint32_t tensor;       /* rollout tensor it belongs to                                           */
+    uint32_t tensor;       /* rollout tensor its first element belongs to (merged runs span several)  */
 } dr_segment_desc;
 
 /*
