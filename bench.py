@@ -262,6 +262,26 @@ def run_reference(args, cfg):
     print(json.dumps(line))
 
 
+def run_all(args):
+    """The per-workload table: each workload in a process of its own (device memory is returned in between)."""
+    for i in range(5):
+        cmd = [sys.executable, os.path.abspath(__file__), "--cfg", str(i), "--steps", str(args.steps), "--warmup",
+               str(args.warmup), "--no-cpu"] + (["--no-staging"] if args.no_staging or i == 4 else [])
+        r = subprocess.run(cmd, capture_output=True, text=True)
+        lines = [l for l in r.stdout.splitlines() if l.startswith("{")]
+        if r.returncode or not lines:
+            print(json.dumps({"cfg": i, "error": (r.stderr or r.stdout)[-300:]}))
+            continue
+        d = json.loads(lines[-1])
+        st = d.get("staging", {})
+        print(json.dumps({"cfg": i, "workload": d["config"]["workload"], "value": d["value"],
+                          "forward_gbs": d["forward"]["gbs_avg"], "forward_ms": d["forward"]["ms_avg"],
+                          "inverse_gbs": d.get("inverse", {}).get("gbs_avg"), "frac_of_measured_peak": d["roofline"]["frac"],
+                          "fp8_forward_gbs": d.get("fp8_forward", {}).get("gbs_avg"),
+                          "stage_out_gbs": st.get("stage_out_gbs"), "stage_in_gbs": st.get("stage_in_gbs"),
+                          "e2e_gbs": d.get("e2e", {}).get("value"), "switch_ms": d.get("switch_ms")}), flush=True)
+
+
 # ------------------------------------------------------------------------------------------------
 # CUDA path
 # ------------------------------------------------------------------------------------------------
@@ -279,6 +299,8 @@ def main():
     ap.add_argument("--layers", type=int, default=0, help="profiling aid: override the layer count (smaller case)")
     ap.add_argument("--vocab", type=int, default=0, help="profiling aid: override the vocabulary size")
     ap.add_argument("--profile", action="store_true", help="profiling aid: allow fewer than 3 warm-up steps")
+    ap.add_argument("--all", action="store_true", help="run the five workloads one after the other (one process each) "
+                                                       "and print one summary line per workload")
     args = ap.parse_args()
     if args.impl == "ours" and not args.profile:
         args.warmup = max(args.warmup, 3)
@@ -289,6 +311,9 @@ def main():
         cfg["spec"] = dict(cfg["spec"], n_layers=args.layers or cfg["spec"]["n_layers"],
                            vocab=args.vocab or cfg["spec"]["vocab"])
         cfg["name"] += f" (reduced: {cfg['spec']['n_layers']} layers, vocab {cfg['spec']['vocab']})"
+    if args.all:
+        run_all(args)
+        return
     if args.impl == "reference":
         run_reference(args, cfg)
         return
