@@ -127,6 +127,7 @@ typedef struct dr_plan_info {
     uint64_t bytes_moved_inv; /* the same for dr_reshard_inverse                                     */
     uint64_t quant_elems;     /* DR_FP8_E4M3_B128 plans: elements written as fp8 (counted in elems_moved) */
     uint64_t quant_blocks;    /* and the number of 128 x 128 blocks, one fp32 scale each              */
+    uint64_t n_groups;        /* n_layers + 2: embed, every layer, final norm with lm_head            */
 } dr_plan_info;
 
 typedef struct dr_tensor_desc {
@@ -203,6 +204,26 @@ int dr_reshard(const dr_plan* plan, const void* src_dev, uint64_t src_bytes, voi
  */
 int dr_reshard_inverse(const dr_plan* plan, const void* rollout_dev, uint64_t rollout_bytes, void* flat_dev,
                        uint64_t flat_bytes, void* cuda_stream);
+
+/* A group of rollout tensors that can be repacked on its own: group 0 is embed, group l + 1 is layer l,
+ * the last group holds final_norm and lm_head. */
+typedef struct dr_group_desc {
+    uint32_t first_tensor, n_tensors; /* rollout tensors [first_tensor, first_tensor + n_tensors)        */
+    uint64_t elems;                   /* elements the group moves (0 when its sources lie in other shards) */
+    uint64_t bytes_moved;             /* algorithmic bytes: (4 + rollout element size) * elems            */
+} dr_group_desc;
+int dr_plan_group(const dr_plan* plan, uint32_t g, dr_group_desc* out); /* DR_ERR_INVALID if g >= n_groups */
+
+/*
+ * dr_reshard_groups -- dr_reshard restricted to groups [first, first + count): one layer (or a few) at a
+ * time, so that whatever follows the repack of a layer (handing it to the rollout engine, sending it to
+ * other GPUs) can overlap the repack of the next ones; this is the switch split into the fine-grained,
+ * overlappable operations Sec. 3.1 and 3.3 argue for.  Elements of other groups keep their bytes;
+ * running every group once, in any order, gives exactly dr_reshard's result.  Same arguments and errors
+ * as dr_reshard, plus DR_ERR_INVALID for a range outside the groups and DR_ERR_UNSUPPORTED for fp8 plans.
+ */
+int dr_reshard_groups(const dr_plan* plan, uint32_t first, uint32_t count, const void* src_dev, uint64_t src_bytes,
+                      void* dst_dev, uint64_t dst_bytes, void* cuda_stream);
 
 /*
  * dr_reshard_static -- dr_reshard for callers that must not allocate device memory.  (The paper has

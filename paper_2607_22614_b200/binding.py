@@ -18,7 +18,7 @@ DR_MAX_STAGE_BUFS = 8
 DR_STAGE_HOST_OFFSETS = 1
 
 EXPORTS = ["dr_plan_create", "dr_plan_create_host", "dr_plan_window_host", "dr_plan_query", "dr_plan_tensor", "dr_plan_segment",
-           "dr_reshard", "dr_reshard_inverse", "dr_reshard_static", "dr_reshard_stream", "dr_shard_range", "dr_stage_out", "dr_stage_in", "dr_plan_destroy", "dr_strerror",
+           "dr_reshard", "dr_reshard_inverse", "dr_plan_group", "dr_reshard_groups", "dr_reshard_static", "dr_reshard_stream", "dr_shard_range", "dr_stage_out", "dr_stage_in", "dr_plan_destroy", "dr_strerror",
            "dr_last_error", "dr_ctl_create", "dr_ctl_observe", "dr_ctl_break_even", "dr_ctl_destroy"]
 
 u8, u32, u64, i64, vp = C.c_uint8, C.c_uint32, C.c_uint64, C.c_int64, C.c_void_p
@@ -43,7 +43,11 @@ class dr_dst_layout(C.Structure):
 class dr_plan_info(C.Structure):
     _fields_ = [(n, u64) for n in ("flat_elems", "shard_elems", "src_bytes", "dst_bytes", "n_tensors", "n_segments",
                                    "n_tiles", "elems_moved", "bytes_moved_fwd", "bytes_moved_inv",
-                                   "quant_elems", "quant_blocks")]
+                                   "quant_elems", "quant_blocks", "n_groups")]
+
+
+class dr_group_desc(C.Structure):
+    _fields_ = [("first_tensor", u32), ("n_tensors", u32), ("elems", u64), ("bytes_moved", u64)]
 
 
 class dr_tensor_desc(C.Structure):
@@ -114,6 +118,8 @@ def lib() -> C.CDLL:
         L.dr_reshard.argtypes = [vp, vp, u64, vp, u64, vp]
         L.dr_reshard_inverse.argtypes = [vp, vp, u64, vp, u64, vp]
         L.dr_reshard_static.argtypes = [vp, vp, u64, vp, u64, vp]
+        L.dr_plan_group.argtypes = [vp, u32, P(dr_group_desc)]
+        L.dr_reshard_groups.argtypes = [vp, u32, u32, vp, u64, vp, u64, vp]
         L.dr_stage_out.argtypes = [vp, P(dr_stage_desc), P(dr_stage_stats)]
         L.dr_stage_in.argtypes = [vp, P(dr_stage_desc), P(dr_stage_stats)]
         L.dr_reshard_stream.argtypes = [vp, P(dr_stream_desc), P(dr_stream_stats)]
@@ -220,6 +226,15 @@ def dr_reshard(plan, src_dev, src_bytes, dst_dev, dst_bytes, cuda_stream):
 
 def dr_reshard_inverse(plan, rollout_dev, rollout_bytes, flat_dev, flat_bytes, cuda_stream):
     return lib().dr_reshard_inverse(plan, rollout_dev, rollout_bytes, flat_dev, flat_bytes, cuda_stream)
+
+
+def dr_plan_group(plan, g):
+    d = dr_group_desc()
+    return lib().dr_plan_group(plan, g, C.byref(d)), d
+
+
+def dr_reshard_groups(plan, first, count, src_dev, src_bytes, dst_dev, dst_bytes, cuda_stream):
+    return lib().dr_reshard_groups(plan, first, count, src_dev, src_bytes, dst_dev, dst_bytes, cuda_stream)
 
 
 def dr_reshard_static(plan, src_dev, src_bytes, dst_dev, dst_bytes, cuda_stream):
@@ -358,6 +373,13 @@ class Plan:
                         dst.numel() * dst.element_size(), self._stream(stream))
         if rc:
             raise DrError(rc, "dr_reshard")
+
+    def reshard_groups(self, first, count, src, dst, stream=None):
+        """Repack only groups [first, first + count) (0: embed, l + 1: layer l, last: final norm and lm_head)."""
+        rc = dr_reshard_groups(self.handle, first, count, src.data_ptr(), src.numel() * src.element_size(), dst.data_ptr(),
+                               dst.numel() * dst.element_size(), self._stream(stream))
+        if rc:
+            raise DrError(rc, "dr_reshard_groups")
 
     def reshard_inverse(self, rollout, flat, stream=None):
         rc = dr_reshard_inverse(self.handle, rollout.data_ptr(), rollout.numel() * rollout.element_size(),

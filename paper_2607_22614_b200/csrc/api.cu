@@ -294,6 +294,47 @@ int dr_reshard(const dr_plan* plan, const void* src_dev, uint64_t src_bytes, voi
     return rc;
 }
 
+int dr_plan_group(const dr_plan* plan, uint32_t g, dr_group_desc* out)
+{
+    if (!plan || !out || g >= plan->groups.size()) {
+        set_error("bad group index");
+        return DR_ERR_INVALID;
+    }
+    const Group& G = plan->groups[g];
+    out->first_tensor = G.first_tensor;
+    out->n_tensors = G.n_tensors;
+    out->elems = G.elems;
+    out->bytes_moved = G.elems * (4 + plan->elem_size);
+    return DR_OK;
+}
+
+int dr_reshard_groups(const dr_plan* plan, uint32_t first, uint32_t count, const void* src_dev, uint64_t src_bytes,
+                      void* dst_dev, uint64_t dst_bytes, void* cuda_stream)
+{
+    int rc = check_call(plan, src_dev, src_bytes, plan ? plan->info.src_bytes : 0, dst_dev, dst_bytes,
+                        plan ? plan->info.dst_bytes : 0);
+    if (rc) return rc;
+    if (plan->fp8) {
+        set_error("fp8 plans are repacked whole");
+        return DR_ERR_UNSUPPORTED;
+    }
+    if (count == 0 || first >= plan->groups.size() || count > plan->groups.size() - first) {
+        set_error("group range outside the plan's %zu groups", plan->groups.size());
+        return DR_ERR_INVALID;
+    }
+    // groups own consecutive tile ranges: the union of the non-empty ones is one range
+    uint64_t lo = ~0ull, hi = 0;
+    for (uint32_t g = first; g < first + count; ++g) {
+        const Group& G = plan->groups[g];
+        if (G.tile_hi > G.tile_lo) {
+            lo = G.tile_lo < lo ? G.tile_lo : lo;
+            hi = G.tile_hi > hi ? G.tile_hi : hi;
+        }
+    }
+    if (hi == 0) return DR_OK;  // nothing of these groups lies in this shard
+    return launch_reshard(plan, false, src_dev, dst_dev, nullptr, cuda_stream, lo, hi);
+}
+
 int dr_reshard_inverse(const dr_plan* plan, const void* rollout_dev, uint64_t rollout_bytes, void* flat_dev,
                        uint64_t flat_bytes, void* cuda_stream)
 {

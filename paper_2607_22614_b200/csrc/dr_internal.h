@@ -14,7 +14,7 @@ namespace dr {
 // A work unit is 8 consecutive elements of one row (32 B of fp32, 16 B of bf16); a tile is
 // kTileUnits consecutive units of one segment.  One CTA iteration processes one tile.
 #ifndef DR_TILE_UNITS
-#define DR_TILE_UNITS 512
+#define DR_TILE_UNITS 1536
 #endif
 constexpr uint32_t kUnitElems = 8;
 constexpr uint32_t kTileUnits = DR_TILE_UNITS;
@@ -64,12 +64,20 @@ static_assert(sizeof(QTensor) == 48, "QTensor layout");
 struct HostSeg {
     uint64_t dst_off, src_off, rows, row_len, src_stride, dst_stride;
     uint32_t flags, tensor;
+    uint32_t group = 0;  // 0: embed, 1..L: layers, L+1: final norm and lm_head
+};
+
+// A group of rollout tensors that can be repacked on its own (tiles [tile_lo, tile_hi) of the plan).
+struct Group {
+    uint64_t tile_lo = 0, tile_hi = 0, elems = 0;
+    uint32_t first_tensor = 0, n_tensors = 0;
 };
 
 struct Tensor {
     std::string name;
     uint64_t arena_off = 0, rows = 0, cols = 0;
     int64_t alias_of = -1;
+    uint32_t group = 0;
     uint32_t es = 2;         // payload bytes per element
     bool quant = false;
     uint64_t scale_off = 0;  // quantised tensors
@@ -98,6 +106,7 @@ struct dr_plan {
     std::vector<dr::Tensor> tensors;
     std::vector<dr::HostSeg> segs;
     std::vector<dr::DevSeg> dev_segs;  // host copy of the device table
+    std::vector<dr::Group> groups;
     // hints[i] = segment holding tile i << hint_shift: a tile finds its segment with one load plus a short walk
     std::vector<uint32_t> hints;
     uint32_t hint_shift = 0;
@@ -138,8 +147,9 @@ namespace dr {
 
 void set_error(const char* fmt, ...);
 int compile_plan(dr_plan* p);  // planner.cpp: fills tensors, segs, dev_segs, info
+// Tiles [tile_lo, min(tile_hi, all)) of the plan.
 int launch_reshard(const dr_plan* p, bool inverse, const void* flat, void* arena_or_flat_out, const void* arena_in,
-                   void* stream);
+                   void* stream, uint64_t tile_lo = 0, uint64_t tile_hi = ~0ull);
 int choose_grid(int device, uint32_t elem_size);  // resident CTAs of the reshard kernel on the whole GPU
 int launch_quant(const dr_plan* p, const void* flat, void* arena, void* stream);
 void ring_destroy(Ring* r);

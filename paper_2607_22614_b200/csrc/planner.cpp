@@ -36,6 +36,7 @@ bool is_linear_weight(const std::string& name)
 struct Emit {
     dr_plan* p;
     uint64_t arena = 0;
+    uint32_t group = 0;  // group of the tensors begun from now on
     uint64_t align_up(uint64_t x) const
     {
         uint64_t a = p->dst.arena_align_bytes;
@@ -61,6 +62,7 @@ struct Emit {
         Tensor t;
         t.name = name;
         t.cols = cols;
+        t.group = group;
         t.quant = p->fp8 && is_linear_weight(name);
         t.es = t.quant ? 1 : p->elem_size;
         arena = align_up(arena);
@@ -97,6 +99,7 @@ struct Emit {
         g.dst_off = t.arena_off + t.rows * t.cols * p->elem_size;
         g.src_off = q.off + r0 * q.cols + c0;
         g.tensor = (uint32_t)(p->tensors.size() - 1);
+        g.group = t.group;
         if (t.cols == q.cols) {  // whole rows: one contiguous run
             g.rows = 1;
             g.row_len = nr * t.cols;
@@ -129,7 +132,7 @@ void merge_adjacent(std::vector<HostSeg>& v, uint32_t es)
     for (const HostSeg& g : v) {
         if (!out.empty()) {
             HostSeg& b = out.back();
-            if (contiguous(b) && contiguous(g) && b.src_off + b.row_len == g.src_off &&
+            if (b.group == g.group && contiguous(b) && contiguous(g) && b.src_off + b.row_len == g.src_off &&
                 b.dst_off + b.row_len * es == g.dst_off) {
                 b.row_len += g.row_len;
                 b.src_stride = b.dst_stride = b.row_len;
@@ -336,6 +339,7 @@ int compile_plan(dr_plan* p)
             snprintf(nm, sizeof nm, "layers.%u.%s", l, leaf);
             return std::string(nm);
         };
+        out.group = l + 1;
         Param in_norm = flat.take(1, H);
         Param q = flat.take(nq * hd, H), k = flat.take(nkv * hd, H), v = flat.take(nkv * hd, H);
         Param q_norm{}, k_norm{};
@@ -389,6 +393,7 @@ int compile_plan(dr_plan* p)
             for (uint64_t e = e_first; e < e_first + E_loc; ++e) out.block(de[e], 0, mt * Fs, H);
         }
     }
+    out.group = s.n_layers + 1;
     Param final_norm = flat.take(1, H);
     out.begin("final_norm", H);
     out.block(final_norm, 0, 0, 1);
@@ -399,6 +404,7 @@ int compile_plan(dr_plan* p)
         a.arena_off = p->tensors[embed_index].arena_off;
         a.rows = p->tensors[embed_index].rows;
         a.cols = H;
+        a.group = out.group;
         p->tensors.push_back(a);
     } else {
         Param lm_head = flat.take(V, H);
@@ -420,6 +426,31 @@ int compile_plan(dr_plan* p)
     p->hints.swap(tb.hints);
     p->hint_shift = tb.hint_shift;
     const uint64_t tiles = tb.n_tiles, moved = tb.elems;
+    // tile range, tensors and element count of every group (segments are in group order)
+    p->groups.assign(s.n_layers + 2, Group{});
+    for (size_t i = 0; i < p->tensors.size(); ++i) {
+        Group& G = p->groups[p->tensors[i].group];
+        if (G.n_tensors == 0) G.first_tensor = (uint32_t)i;
+        G.n_tensors++;
+    }
+    {
+        uint64_t at = 0;
+        for (Group& G : p->groups) G.tile_lo = G.tile_hi = 0;
+        std::vector<bool> seen(p->groups.size(), false);
+        for (size_t i = 0; i < p->segs.size(); ++i) {
+            Group& G = p->groups[p->segs[i].group];
+            const uint64_t t0 = p->dev_segs[i].tile0;
+            const uint64_t t1 = i + 1 < p->segs.size() ? p->dev_segs[i + 1].tile0 : tiles;
+            if (!seen[p->segs[i].group]) {
+                G.tile_lo = t0;
+                seen[p->segs[i].group] = true;
+            }
+            G.tile_hi = t1;
+            G.elems += p->segs[i].rows * p->segs[i].row_len;
+            at = t1;
+        }
+        (void)at;
+    }
 
     // fp8: block prefix per quantised tensor and a block -> tensor hint table
     uint64_t qblocks = 0, qelems = 0;
@@ -452,6 +483,7 @@ int compile_plan(dr_plan* p)
     I.elems_moved = moved + qelems;
     I.bytes_moved_fwd = moved * (4 + es) + qelems * 5 + qblocks * 4;
     I.bytes_moved_inv = moved * (4 + es);
+    I.n_groups = p->groups.size();
     I.quant_elems = qelems;
     I.quant_blocks = qblocks;
 

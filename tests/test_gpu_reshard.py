@@ -262,3 +262,44 @@ def test_repack_and_inverse_replay_from_a_cuda_graph():
         om.inverse(want, wflat)
         assert first_diff(back.cpu().numpy().view(np.uint32), wflat) is None
     plan.close()
+
+
+@pytest.mark.parametrize("spec,kw", [(MID[0]["spec"], dict(tp=2, tp_rank=1)), (MID[2]["spec"], dict(tp=1)),
+                                     (MID[1]["spec"], dict(world=3, rank=1, gathered=False, tp=2, tp_rank=0)),
+                                     (BRUTE[1]["spec"], dict(tp=2, tp_rank=0, align=3))],
+                         ids=["dense-tp2", "moe", "shard-local-tied", "brute-tied"])
+def test_groups_in_any_order_build_up_the_full_repack(spec, kw):
+    """One layer at a time, in a shuffled order: after every call the arena holds exactly the oracle's tensors
+    of the groups done so far and the sentinel everywhere else; at the end it is dr_reshard's result."""
+    kw = dict(kw)
+    world, rank, gathered, align = kw.pop("world", 1), kw.pop("rank", 0), kw.pop("gathered", True), kw.pop("align", 1)
+    om = oracle.Model(spec, align=align, world=world, **kw)
+    full = make_source(world * om.shard_elems, 123)
+    local = full if gathered else full[rank * om.shard_elems:(rank + 1) * om.shard_elems].copy()
+    plan = dr.Plan(spec, world=world, rank=rank, gathered=gathered, align_elems=align, **kw)
+    src = to_dev_u32(local)
+    arena = arena_dev(om.arena_bytes)
+    want = np.full(om.arena_bytes, SENT8, dtype=np.uint8)
+    order = np.random.default_rng(5).permutation(plan.info.n_groups)
+    for g in order:
+        rc, d = dr.dr_plan_group(plan.handle, int(g))
+        for i in range(d.first_tensor, d.first_tensor + d.n_tensors):
+            om.forward(local, want, gathered=gathered, rank=rank, only=i)
+        plan.reshard_groups(int(g), 1, src, arena)
+        torch.cuda.synchronize()
+        assert first_diff(arena.cpu().numpy(), want) is None
+    ref = arena_dev(om.arena_bytes)
+    plan.reshard(src, ref)
+    torch.cuda.synchronize()
+    assert torch.equal(ref, arena)
+    # several groups in one call, and the argument checks
+    arena2 = arena_dev(om.arena_bytes)
+    half = plan.info.n_groups // 2
+    plan.reshard_groups(0, half, src, arena2)
+    plan.reshard_groups(half, plan.info.n_groups - half, src, arena2)
+    torch.cuda.synchronize()
+    assert torch.equal(ref, arena2)
+    s = torch.cuda.current_stream().cuda_stream
+    bad = dr.dr_reshard_groups(plan.handle, 1, plan.info.n_groups, src.data_ptr(), src.numel() * 4, arena.data_ptr(), arena.numel(), s)
+    assert bad == dr.binding.DR_ERR_INVALID
+    plan.close()

@@ -124,7 +124,7 @@ def test_library_exports_every_declared_symbol():
 
 def test_struct_sizes_match_the_header_layout():
     assert C.sizeof(dr.dr_model_spec) == 48 and C.sizeof(dr.dr_src_layout) == 28 and C.sizeof(dr.dr_dst_layout) == 36
-    assert C.sizeof(dr.dr_stage_desc) == 432 and C.sizeof(dr.dr_stage_stats) == 112 and C.sizeof(dr.dr_plan_info) == 96 and C.sizeof(dr.dr_tensor_desc) == 128 and C.sizeof(dr.dr_segment_desc) == 56
+    assert C.sizeof(dr.dr_stage_desc) == 432 and C.sizeof(dr.dr_stage_stats) == 112 and C.sizeof(dr.dr_plan_info) == 104 and C.sizeof(dr.dr_tensor_desc) == 128 and C.sizeof(dr.dr_segment_desc) == 56
 
 
 def test_error_codes():
@@ -289,3 +289,31 @@ def test_source_windows_partition_the_plan(spec, kw, chunk):
     assert dr.dr_plan_window_host(p.handle, 5, 5)[0] == dr.binding.DR_ERR_INVALID
     assert dr.dr_plan_window_host(p.handle, 0, n_src + 1)[0] == dr.binding.DR_ERR_INVALID
     p.close()
+
+
+def test_groups_partition_the_plan():
+    for cfg, kw in ((CONFIGS[2], {}), (CONFIGS[4], {}), (MID[1], dict(world=3, rank=2, gathered=False, tp=2)),
+                    (BRUTE[2], dict(tp=2, tp_rank=1))):
+        kw = dict(kw)
+        if "world" in cfg and not kw:
+            kw = dict(world=cfg["world"], rank=cfg["rank"], gathered=cfg["gathered"], tp=cfg["tp"], tp_rank=cfg["tp_rank"])
+        p = dr.Plan(cfg["spec"], host_only=True, **kw)
+        L = cfg["spec"]["n_layers"]
+        assert p.info.n_groups == L + 2
+        names = [t.name.decode() for t in p.tensors()]
+        nxt, elems = 0, 0
+        for g in range(p.info.n_groups):
+            rc, d = dr.dr_plan_group(p.handle, g)
+            assert rc == 0 and d.first_tensor == nxt and d.bytes_moved == d.elems * 6
+            mine = names[d.first_tensor:d.first_tensor + d.n_tensors]
+            if g == 0:
+                assert mine == ["embed"]
+            elif g <= L:
+                assert mine and all(n.startswith(f"layers.{g - 1}.") for n in mine)
+            else:
+                assert mine == ["final_norm", "lm_head"]
+            nxt += d.n_tensors
+            elems += d.elems
+        assert nxt == len(names) and elems == p.info.elems_moved
+        assert dr.dr_plan_group(p.handle, p.info.n_groups)[0] == dr.binding.DR_ERR_INVALID
+        p.close()
