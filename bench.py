@@ -440,7 +440,8 @@ def main():
     if inv_ms:
         ia = sum(inv_ms) / len(inv_ms)
         line["inverse"] = {"gbs_avg": bytes_inv / ia / 1e6, "gbs_best": bytes_inv / min(inv_ms) / 1e6, "ms_avg": ia,
-                           "ms_best": min(inv_ms), "frac_of_measured_peak": bytes_inv / ia / 1e6 / peak}
+                           "ms_best": min(inv_ms), "ms_median": median(inv_ms),
+                           "frac_of_measured_peak": bytes_inv / ia / 1e6 / peak}
     line["roofline"]["traffic"] = NCU_DRAM_BYTES_PER_ELEMENT_FWD * (bytes_fwd // 6 // len(plans)) if cfg["spec"] else None
     line["roofline"]["traffic_source"] = "ncu capture of a 654 M-element case of the same kernel, scaled by elements"
 
