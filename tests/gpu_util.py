@@ -62,15 +62,16 @@ def forward_both(spec, *, world=1, rank=0, gathered=True, align=1, tp=1, tp_rank
     s_buf = torch.zeros(n_src + pad, dtype=torch.int32, device=dev())
     s_dev = s_buf[pad:]
     s_dev.copy_(torch.from_numpy(local.view(np.int32)))
-    a_buf = arena_dev(om.arena_bytes + misalign)
-    a_dev = a_buf[misalign:]
+    # guard bands of 256 sentinel bytes on both sides of the arena: a write outside the arena would show there
+    G = 256
+    a_buf = arena_dev(G + misalign + om.arena_bytes + G)
+    a_dev = a_buf[G + misalign:G + misalign + om.arena_bytes]
     if arena_init is not None:
         a_dev.copy_(arena_init[1])
     plan.reshard(s_dev, a_dev)
     torch.cuda.synchronize()
     got = a_dev.cpu().numpy()
-    if misalign:
-        assert (a_buf[:misalign].cpu().numpy() == SENT8).all()
+    assert (a_buf[:G + misalign].cpu().numpy() == SENT8).all() and (a_buf[G + misalign + om.arena_bytes:].cpu().numpy() == SENT8).all()
     return got, want, plan, om, src
 
 
