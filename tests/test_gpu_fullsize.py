@@ -3,6 +3,8 @@
 cfg 1 is compared whole against the oracle (the oracle finishes it in seconds).  cfg 2-4 are too big
 for that: they are checked on sampled outputs that the oracle computes one by one, on whole small
 tensors, on row blocks at the edges of the big tensors, and by counting what the call touched."""
+import os
+
 import numpy as np
 import pytest
 import torch
@@ -261,12 +263,14 @@ def test_cfg4_whole_arena_equals_oracle_streamed_by_layer():
     srcs = om.src_tensors()
     dst = om.dst_tensors()
     groups = ["embed"] + [f"layers.{l}." for l in range(cfg["spec"]["n_layers"])] + ["final_norm", "lm_head"]
-    checked = 0
-    for g in groups:
+
+    def check_group(g):
+        """Generate the group's source, run the oracle on its rollout tensors, compare with the GPU arena, release."""
         mine = [s for s in srcs if s.name == g or (g.endswith(".") and s.name.startswith(g))]
         lo = min(s.flat_off for s in mine)
         hi = max(s.flat_off + s.rows * s.cols for s in mine)
         synth.fill_f32(seed, synth.BUF_MASTER, lo, hi - lo, out=flat[lo:hi])
+        n = 0
         for i, d in enumerate(dst):
             if d.alias_of >= 0 or not (d.name == g or (g.endswith(".") and d.name.startswith(g))):
                 continue
@@ -276,8 +280,14 @@ def test_cfg4_whole_arena_equals_oracle_streamed_by_layer():
             got = arena[d.arena_off:d.arena_off + nbytes].cpu().numpy()
             assert np.array_equal(got, want[d.arena_off:d.arena_off + nbytes]), d.name
             release(mm_dst, d.arena_off, d.arena_off + nbytes)
-            checked += d.rows * d.cols
+            n += d.rows * d.cols
         release(mm_src, 4 * lo, 4 * hi)
+        return n
+
+    # the groups are independent: several run at once on the host cores (the oracle itself stays single-threaded)
+    from concurrent.futures import ThreadPoolExecutor
+    with ThreadPoolExecutor(max_workers=min(6, os.cpu_count() or 1)) as ex:
+        checked = sum(ex.map(check_group, groups))
     assert checked == 29_767_972_864
     del flat, want
 
