@@ -23,6 +23,18 @@
  *     table, its pinned staging ring and two internal streams.
  *   - Streams and events are passed as void* holding a cudaStream_t / cudaEvent_t (NULL stream =
  *     the legacy default stream).
+ *   - Stream ordering.  dr_reshard, dr_reshard_inverse, dr_reshard_groups and dr_reshard_static run on
+ *     the stream they are given and need nothing more.  dr_stage_out, dr_stage_in and
+ *     dr_reshard_stream copy on streams the plan owns (created non-blocking, so not even the legacy
+ *     default stream orders them).  On entry they therefore make their streams wait for everything
+ *     already enqueued on desc->caller_stream (or, when desc->wait_event is set, for that event
+ *     alone), so that device buffers the caller has just filled, zeroed or freed-and-reallocated on
+ *     that stream are ready before the first copy touches them.  Work the caller has pending on any
+ *     OTHER stream that touches those buffers must be covered by wait_event or a synchronise.  The
+ *     three calls block until all of their copies and kernels have completed, so whatever the caller
+ *     enqueues after they return, on any stream, sees the result; done_event is recorded for callers
+ *     that hand the ordering to a third stream.  None of the three may be called while caller_stream
+ *     is being captured into a CUDA graph.
  *   - There is no CPU fallback: without a CUDA device every compute call fails with DR_ERR_CUDA.
  *   - Matrices are [out_features, in_features], row-major.
  */
@@ -188,6 +200,8 @@ int dr_plan_segment(const dr_plan* plan, uint64_t i, dr_segment_desc* out); /* D
  * subnormals are rounded, not flushed), or a bit copy when the plan's dst dtype is DR_F32.
  * Errors (all found before launch): DR_ERR_SIZE if src_bytes / dst_bytes are below the plan's
  * requirement, DR_ERR_ALIGN if a base pointer is not 16-byte aligned, DR_ERR_STATE, DR_ERR_CUDA.
+ * Bases that are 32-byte aligned let the kernels (the fp8 one included) use 256-bit accesses; with
+ * 16-byte aligned bases they fall back to 128-bit ones, same result.
  * The plan is not modified: concurrent calls on different streams are allowed.  The call only enqueues
  * kernels, so (after one ordinary call has loaded the module) it may be recorded into a CUDA graph by
  * stream capture and replayed; the same holds for dr_reshard_inverse.
@@ -239,8 +253,11 @@ int dr_reshard_groups(const dr_plan* plan, uint32_t first, uint32_t count, const
  * runs from there.  The call itself allocates nothing, on host or device.
  *
  * Same arguments, result and errors as dr_reshard, plus DR_ERR_SIZE when the plan has more than
- * 16 384 segments (dr_plan_query: n_segments).  The first call on each device looks up the table's
- * device address; make that first call outside any stream capture.  All calls share the one table and
+ * 16 384 segments (dr_plan_query: n_segments).  Unlike dr_reshard the call is not purely an enqueue:
+ * the table is uploaded from ordinary (pageable) host memory with cudaMemcpyAsync, which the driver may
+ * stage and for which it may make the host wait until earlier work on cuda_stream has drained.  The
+ * first call on each device looks up the table's device address; make that first call outside any
+ * stream capture.  All calls share the one table and
  * it keeps the previous call's entries: each call rewrites the entries it uses, in stream order,
  * before its kernel reads them, so calls on one stream are safe back to back, while calls that can
  * overlap on the GPU (different streams, or different threads on different streams) race on the table
@@ -281,14 +298,24 @@ typedef struct dr_stage_desc {
     void* user;
     void* relay_dev[DR_MAX_STAGE_BUFS];
     uint64_t first_chunk;               /* resume: chunks / pieces below this index are skipped       */
-    void* wait_event;                   /* cudaEvent_t the first copy waits for (producer), or NULL   */
+    void* wait_event;                   /* cudaEvent_t the first copy waits for INSTEAD of
+                                           caller_stream's pending work: the overlap recipe records
+                                           it before enqueueing dr_reshard, so that stage-out starts
+                                           while the repack runs (both only read).  NULL: none      */
     void* ready_events[DR_MAX_STAGE_BUFS]; /* stage-in: caller's cudaEvent_t recorded on the copy
                                               stream right after buffer i's last copy; NULL = none   */
     uint32_t timeout_ms;                /* bound on every internal wait; 0 = 60 000                   */
-    uint32_t flags;                     /* 0 or DR_STAGE_HOST_OFFSETS                                 */
+    uint32_t flags;                     /* DR_STAGE_HOST_OFFSETS | DR_STAGE_UNORDERED, or 0           */
     uint64_t host_offset[DR_MAX_STAGE_BUFS]; /* with DR_STAGE_HOST_OFFSETS: buffer i rests at
                                            host_arena + host_offset[i] instead of at its position in
                                            the stream; regions must not overlap (arena sinks only)    */
+    void* caller_stream;                /* cudaStream_t on which the caller produced (stage-out) or
+                                           last used (stage-in, relay targets) the device buffers;
+                                           NULL = the legacy default stream.  Unless wait_event or
+                                           DR_STAGE_UNORDERED is given, the first copy waits for all
+                                           work enqueued on it before the call                        */
+    void* done_event;                   /* caller's cudaEvent_t recorded after the call's last copy
+                                           (already complete when the call returns), or NULL          */
 } dr_stage_desc;
 
 /* Buffer i of a stage call rests at host_arena + host_offset[i].  This is how training state crosses a
@@ -296,6 +323,9 @@ typedef struct dr_stage_desc {
  * rank stages its shard out to its place in one flat host image, every new rank stages its own,
  * differently cut, range back in (see dr_shard_range). */
 #define DR_STAGE_HOST_OFFSETS 1u
+/* The caller has ordered the device buffers itself (a synchronise, or its own events): the call neither
+ * records on nor waits for caller_stream. */
+#define DR_STAGE_UNORDERED 2u
 
 typedef struct dr_stage_stats {
     uint64_t bytes;                    /* bytes moved by this call                                    */
@@ -311,9 +341,11 @@ typedef struct dr_stage_stats {
 /*
  * dr_stage_out -- device -> host in bounded chunks (Sec. 3.3: the states are partitioned into
  * chunks and streamed through host-memory buffers, store and reload pipelined chunk by chunk).
- * Blocking pump on the calling thread; copies run on the plan's side stream so that a dr_reshard
- * enqueued before it overlaps (both only read the master buffer).  On return every delivered chunk
- * is complete and byte-exact.  Errors: DR_ERR_INVALID, DR_ERR_BUDGET, DR_ERR_SIZE (arena too small),
+ * Blocking pump on the calling thread; copies run on the plan's side stream.  Overlap recipe: record
+ * an event on the caller's stream once the state buffers are final, enqueue dr_reshard, then call
+ * dr_stage_out with wait_event = that event: the copies start while the repack runs (both only read
+ * the master buffer).  Without wait_event the first copy waits for all of caller_stream's pending
+ * work, the repack included.  On return every delivered chunk is complete and byte-exact.  Errors: DR_ERR_INVALID, DR_ERR_BUDGET, DR_ERR_SIZE (arena too small),
  * DR_ERR_NOMEM (pinned ring), DR_ERR_SINK, DR_ERR_TIMEOUT, DR_ERR_CUDA, DR_ERR_STATE.
  * Calls on one plan must not overlap in time (they share the ring).
  */
@@ -323,7 +355,9 @@ int dr_stage_out(dr_plan* plan, const dr_stage_desc* desc, dr_stage_stats* stats
  * dr_stage_in -- host -> device, buffers in desc->order so that the weights are resident first and
  * the optimizer state follows (Sec. 3.3: only the weights are loaded during the transition, the
  * optimizer states are deferred to the first step on the new topology).  stats->ready_ms[i] and
- * ready_events[i] tell when buffer i became usable.  Same pump, errors and threading as above.
+ * ready_events[i] tell when buffer i became usable.  The first copy is ordered after caller_stream's
+ * pending work (a zero-fill or an allocation reuse of the target buffers must not land after it).
+ * Same pump, errors and threading as above.
  */
 int dr_stage_in(dr_plan* plan, const dr_stage_desc* desc, dr_stage_stats* stats);
 
@@ -338,7 +372,7 @@ int dr_stage_in(dr_plan* plan, const dr_stage_desc* desc, dr_stage_stats* stats)
  * applied to the device side, and Sec. 3.3's overlap of operations that do not depend on one another).
  */
 typedef struct dr_stream_desc {
-    uint32_t struct_size, flags;  /* sizeof(dr_stream_desc), 0                                         */
+    uint32_t struct_size, flags;  /* sizeof(dr_stream_desc); 0 or DR_STREAM_UNORDERED                  */
     const void* host_src;         /* pinned host: the plan's source buffer (dr_plan_query: src_bytes)  */
     uint64_t host_src_bytes;
     void* dst_dev;                /* device: the rollout arena                                         */
@@ -350,7 +384,16 @@ typedef struct dr_stream_desc {
     uint64_t chunk_bytes;         /* multiple of 32; 0: window_bytes / 2 rounded down to 4096          */
     uint32_t timeout_ms;          /* bound on the final wait; 0 = 60 000                               */
     uint32_t pad;
+    void* caller_stream;          /* cudaStream_t on which the caller last touched dst_dev / window_dev
+                                     (e.g. filled or zeroed them); NULL = the legacy default stream.  All
+                                     work enqueued on it before the call completes before the first copy
+                                     or kernel of the call, unless wait_event or DR_STREAM_UNORDERED      */
+    void* wait_event;             /* cudaEvent_t to wait for instead of caller_stream's pending work      */
+    void* done_event;             /* caller's cudaEvent_t recorded after the last kernel and copy, or NULL */
 } dr_stream_desc;
+
+/* The caller has ordered dst_dev and window_dev itself: no record on / wait for caller_stream. */
+#define DR_STREAM_UNORDERED 1u
 
 typedef struct dr_stream_stats {
     uint64_t h2d_bytes, d2h_bytes, n_chunks, kernels;
@@ -361,9 +404,12 @@ typedef struct dr_stream_stats {
  * dr_reshard_stream -- the result in dst_dev (and host_dst) is exactly dr_reshard's on the same source.
  * Blocking: returns when every copy and kernel has completed (bounded poll, DR_ERR_TIMEOUT).  The first
  * call with a given chunk size compiles and uploads one small segment table per chunk (device memory
- * owned by the plan, re-used by later calls).  Errors: DR_ERR_INVALID, DR_ERR_SIZE (a buffer too small),
- * DR_ERR_ALIGN (pointers not 32-byte aligned), DR_ERR_BUDGET (window below two chunks), DR_ERR_STATE
- * (host-only plan), DR_ERR_NOMEM, DR_ERR_CUDA, DR_ERR_TIMEOUT.  Calls on one plan must not overlap.
+ * owned by the plan, re-used by later calls).  On a timeout or an enqueue error the call still waits
+ * (bounded, a generous fixed limit) for what it had already enqueued, so that nothing of it is in flight
+ * on return.  Errors: DR_ERR_INVALID (bad descriptor; chunk_bytes not a multiple of 32), DR_ERR_SIZE (a
+ * buffer too small), DR_ERR_ALIGN (pointers not 32-byte aligned), DR_ERR_BUDGET (window below two chunks),
+ * DR_ERR_STATE (host-only plan), DR_ERR_NOMEM, DR_ERR_CUDA, DR_ERR_TIMEOUT.  Calls on one plan must not
+ * overlap.
  */
 int dr_reshard_stream(dr_plan* plan, const dr_stream_desc* desc, dr_stream_stats* stats);
 

@@ -16,6 +16,8 @@ DR_DST_ROLLOUT_FUSED = 1
 DR_F32, DR_BF16, DR_FP8_E4M3_B128 = 1, 2, 3
 DR_MAX_STAGE_BUFS = 8
 DR_STAGE_HOST_OFFSETS = 1
+DR_STAGE_UNORDERED = 2
+DR_STREAM_UNORDERED = 1
 
 EXPORTS = ["dr_plan_create", "dr_plan_create_host", "dr_plan_window_host", "dr_plan_query", "dr_plan_tensor", "dr_plan_segment",
            "dr_reshard", "dr_reshard_inverse", "dr_plan_group", "dr_reshard_groups", "dr_reshard_static", "dr_reshard_stream", "dr_shard_range", "dr_stage_out", "dr_stage_in", "dr_plan_destroy", "dr_strerror",
@@ -68,7 +70,7 @@ class dr_stage_desc(C.Structure):
                 ("budget_bytes", u64), ("chunk_bytes", u64), ("host_arena", vp), ("host_arena_bytes", u64),
                 ("callback", dr_chunk_fn), ("user", vp), ("relay_dev", vp * 8), ("first_chunk", u64),
                 ("wait_event", vp), ("ready_events", vp * 8), ("timeout_ms", u32), ("flags", u32),
-                ("host_offset", u64 * 8)]
+                ("host_offset", u64 * 8), ("caller_stream", vp), ("done_event", vp)]
 
 
 class dr_stage_stats(C.Structure):
@@ -79,7 +81,8 @@ class dr_stage_stats(C.Structure):
 class dr_stream_desc(C.Structure):
     _fields_ = [("struct_size", u32), ("flags", u32), ("host_src", vp), ("host_src_bytes", u64), ("dst_dev", vp),
                 ("dst_bytes", u64), ("host_dst", vp), ("host_dst_bytes", u64), ("window_dev", vp), ("window_bytes", u64),
-                ("chunk_bytes", u64), ("timeout_ms", u32), ("pad", u32)]
+                ("chunk_bytes", u64), ("timeout_ms", u32), ("pad", u32), ("caller_stream", vp), ("wait_event", vp),
+                ("done_event", vp)]
 
 
 class dr_stream_stats(C.Structure):
@@ -160,9 +163,20 @@ def dst_layout(dtype=DR_BF16, arena_align_bytes=256, moe_tp=1, kv_replicate=Fals
                          moe_ep=moe_ep, moe_ep_rank=moe_ep_rank)
 
 
+def _current_stream(stream):
+    """cudaStream_t of `stream` (a torch stream, a raw handle, or None = torch's current stream)."""
+    if stream is None:
+        import torch
+        # without a CUDA device the descriptor can still be built (argument checks); NULL = legacy default stream
+        return torch.cuda.current_stream().cuda_stream if torch.cuda.is_available() else None
+    return getattr(stream, "cuda_stream", stream)
+
+
 def stage_desc(dev_ptrs, sizes, budget, chunk=0, order=None, host_arena=None, host_arena_bytes=0, callback=None,
                relay_dev=None, first_chunk=0, wait_event=None, ready_events=None, timeout_ms=0,
-               host_offsets=None) -> dr_stage_desc:
+               host_offsets=None, caller_stream=None, done_event=None, unordered=False) -> dr_stage_desc:
+    """Fill a dr_stage_desc.  caller_stream=None names torch's current stream: the call's first copy then waits
+    for whatever has been enqueued there (the fills or kernels that produced the device buffers)."""
     d = dr_stage_desc()
     d.struct_size = C.sizeof(dr_stage_desc)
     d.n_bufs = len(dev_ptrs)
@@ -184,6 +198,11 @@ def stage_desc(dev_ptrs, sizes, budget, chunk=0, order=None, host_arena=None, ho
         d.flags |= DR_STAGE_HOST_OFFSETS
         for i, o in enumerate(host_offsets):
             d.host_offset[i] = o
+    if unordered:
+        d.flags |= DR_STAGE_UNORDERED
+    else:
+        d.caller_stream = _current_stream(caller_stream)
+    d.done_event = done_event
     return d
 
 
@@ -255,10 +274,15 @@ def dr_stage_in(plan, desc):
 
 
 def stream_desc(host_src, host_src_bytes, dst_dev, dst_bytes, window_dev, window_bytes, chunk_bytes=0, host_dst=None,
-                host_dst_bytes=0, timeout_ms=0) -> dr_stream_desc:
-    return dr_stream_desc(struct_size=C.sizeof(dr_stream_desc), host_src=host_src, host_src_bytes=host_src_bytes,
+                host_dst_bytes=0, timeout_ms=0, caller_stream=None, wait_event=None, done_event=None,
+                unordered=False) -> dr_stream_desc:
+    """Fill a dr_stream_desc; caller_stream=None names torch's current stream (see stage_desc)."""
+    return dr_stream_desc(struct_size=C.sizeof(dr_stream_desc), flags=DR_STREAM_UNORDERED if unordered else 0,
+                          host_src=host_src, host_src_bytes=host_src_bytes,
                           dst_dev=dst_dev, dst_bytes=dst_bytes, host_dst=host_dst, host_dst_bytes=host_dst_bytes,
-                          window_dev=window_dev, window_bytes=window_bytes, chunk_bytes=chunk_bytes, timeout_ms=timeout_ms)
+                          window_dev=window_dev, window_bytes=window_bytes, chunk_bytes=chunk_bytes, timeout_ms=timeout_ms,
+                          caller_stream=None if unordered else _current_stream(caller_stream), wait_event=wait_event,
+                          done_event=done_event)
 
 
 def dr_reshard_stream(plan, desc):
@@ -360,12 +384,7 @@ class Plan:
             out.append(s)
         return out
 
-    @staticmethod
-    def _stream(stream):
-        if stream is None:
-            import torch
-            return torch.cuda.current_stream().cuda_stream
-        return getattr(stream, "cuda_stream", stream)
+    _stream = staticmethod(_current_stream)
 
     def reshard(self, src, dst, stream=None):
         """src: CUDA tensor holding the flat fp32 buffer; dst: CUDA tensor holding the rollout arena."""

@@ -30,6 +30,12 @@ __device__ __forceinline__ void ld256f(const void* p, float (&v)[8])
                  : "=f"(v[0]), "=f"(v[1]), "=f"(v[2]), "=f"(v[3]), "=f"(v[4]), "=f"(v[5]), "=f"(v[6]), "=f"(v[7])
                  : "l"(p));
 }
+__device__ __forceinline__ void ld128f(const void* p, float* v)
+{
+    asm volatile("ld.global.nc.L1::no_allocate.v4.f32 {%0,%1,%2,%3}, [%4];"
+                 : "=f"(v[0]), "=f"(v[1]), "=f"(v[2]), "=f"(v[3])
+                 : "l"(p));
+}
 __device__ __forceinline__ float ld32f(const void* p)
 {
     float v;
@@ -47,7 +53,7 @@ __device__ __forceinline__ uint32_t cvt_e4m3x2(float lo, float hi)
 __global__ void __launch_bounds__(kQThreads, DR_Q_MIN_BLOCKS)
     quant_kernel(const QTensor* __restrict__ tensors, uint32_t n_tensors, const QPart* __restrict__ parts,
                  const uint32_t* __restrict__ hints, uint32_t hint_shift, const char* __restrict__ flat,
-                 char* __restrict__ arena)
+                 char* __restrict__ arena, int allow256)
 {
     __shared__ uint64_t row_src[128];  // flat element offset of (row, first column of the tensor)
     __shared__ float warp_max[kQThreads / 32];
@@ -92,8 +98,13 @@ __global__ void __launch_bounds__(kQThreads, DR_Q_MIN_BLOCKS)
         for (int k = 0; k < 8; ++k) v[p][k] = 0.0f;
         if (row < nrows && col < T.cols) {
             const char* src = flat + (row_src[row] + col) * 4;
-            if (T.aligned) {
+            // T.aligned speaks of offsets from the flat base; the base itself is only promised to be 16-byte
+            // aligned, so the 256-bit form also needs a 32-byte aligned base (allow256)
+            if (T.aligned && allow256) {
                 ld256f(src, v[p]);
+            } else if (T.aligned) {
+                ld128f(src, &v[p][0]);
+                ld128f(src + 16, &v[p][4]);
             } else {
 #pragma unroll
                 for (int k = 0; k < 8; ++k)
@@ -159,7 +170,7 @@ int launch_quant(const dr_plan* p, const void* flat, void* arena, void* stream)
     }
     quant_kernel<<<(unsigned)blocks, kQThreads, 0, (cudaStream_t)stream>>>(
         p->d_qtensors, (uint32_t)p->qtensors.size(), p->d_qparts, p->d_qhints, p->qhint_shift, (const char*)flat,
-        (char*)arena);
+        (char*)arena, (((uintptr_t)flat | (uintptr_t)arena) & 31) == 0);
     cudaError_t e = cudaGetLastError();
     if (e != cudaSuccess) {
         set_error("quant kernel launch: %s", cudaGetErrorString(e));

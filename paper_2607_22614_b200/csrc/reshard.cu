@@ -266,7 +266,7 @@ __global__ void __launch_bounds__(kThreads, DR_MIN_BLOCKS)
             }
         } else {
             // Scalar path for runs that start or end off the vector grid (odd shapes, shard cuts):
-            // element e of the tile is handled by thread e % 256, so accesses stay coalesced.
+            // consecutive threads take consecutive elements of the tile, so accesses stay coalesced.
             const uint64_t e0 = (uint64_t)(tile - g.tile0) * kTileUnits * 8;
 #pragma unroll 1
             for (uint32_t k = threadIdx.x; k < kTileUnits * 8; k += kThreads) {
@@ -323,6 +323,10 @@ int launch_reshard(const dr_plan* p, bool inverse, const void* flat, void* arena
     const int allow256 = (((uintptr_t)f | (uintptr_t)a) & 31) == 0;
     uint64_t want = DR_GRID_MULT ? (uint64_t)p->grid : (n + DR_TILES_PER_CTA - 1) / DR_TILES_PER_CTA;
     uint64_t g64 = n < want ? n : want;
+    if (g64 > 0x7FFFFFFFull) {
+        set_error("%llu tiles exceed the largest grid", (unsigned long long)g64);
+        return DR_ERR_UNSUPPORTED;
+    }
     dim3 grid((unsigned)g64), block(kThreads);
     cudaStream_t s = (cudaStream_t)stream;
     const uint32_t n_segs = (uint32_t)p->dev_segs.size();
@@ -351,6 +355,10 @@ int launch_forward_tables(uint32_t elem_size, const DevSeg* d_segs, uint32_t n_s
     char* a = (char*)arena;
     const int allow256 = (((uintptr_t)f | (uintptr_t)a) & 31) == 0;
     const uint64_t want = (n_tiles + DR_TILES_PER_CTA - 1) / DR_TILES_PER_CTA;
+    if (want > 0x7FFFFFFFull) {
+        set_error("%llu tiles exceed the largest grid", (unsigned long long)want);
+        return DR_ERR_UNSUPPORTED;
+    }
     dim3 grid((unsigned)want), block(kThreads);
     cudaStream_t s = (cudaStream_t)stream;
     if (elem_size == 2)
@@ -460,6 +468,10 @@ extern "C" int dr_reshard_static(const dr_plan* plan, const void* src_dev, uint6
     if (rc) return rc;
     const uint64_t n_tiles = plan->info.n_tiles;
     if (n_tiles == 0) return DR_OK;
+    if (n_tiles > 0x7FFFFFFFull) {
+        set_error("%llu tiles exceed the largest grid", (unsigned long long)n_tiles);
+        return DR_ERR_UNSUPPORTED;
+    }
     cudaStream_t s = (cudaStream_t)cuda_stream;
     // The table is rewritten for every call, in stream order before the kernel that reads it.
     cudaError_t e = cudaMemcpyAsync(slot.table, plan->dev_segs.data(), n_segs * sizeof(DevSeg), cudaMemcpyHostToDevice, s);

@@ -30,6 +30,7 @@ struct Ring {
     uint64_t chunk = 0;
     uint32_t slots = 0;
     std::vector<cudaEvent_t> ev_copy, ev_relay;  // one per slot
+    cudaEvent_t ev_entry = nullptr;              // recorded on the caller's stream when a call begins
     std::unique_ptr<CopyPool> pool;
 };
 
@@ -40,6 +41,7 @@ void ring_destroy(Ring* r)
     if (r->s_relay) cudaStreamSynchronize(r->s_relay);
     for (auto e : r->ev_copy) cudaEventDestroy(e);
     for (auto e : r->ev_relay) cudaEventDestroy(e);
+    if (r->ev_entry) cudaEventDestroy(r->ev_entry);
     if (r->base) cudaFreeHost(r->base);
     if (r->s_copy) cudaStreamDestroy(r->s_copy);
     if (r->s_relay) cudaStreamDestroy(r->s_relay);
@@ -91,6 +93,7 @@ int ensure_ring(dr_plan* p, const Geometry& g, bool need_memory)
         p->ring = r;
         DR_CUDA(cudaStreamCreateWithFlags(&r->s_copy, cudaStreamNonBlocking));
         DR_CUDA(cudaStreamCreateWithFlags(&r->s_relay, cudaStreamNonBlocking));
+        DR_CUDA(cudaEventCreateWithFlags(&r->ev_entry, cudaEventDisableTiming));
         unsigned hw = std::thread::hardware_concurrency();
         r->pool.reset(new CopyPool(std::max(1u, std::min(16u, hw))));
     }
@@ -115,6 +118,21 @@ int ensure_ring(dr_plan* p, const Geometry& g, bool need_memory)
         r->chunk = g.chunk;
         r->slots = g.slots;
     }
+    return DR_OK;
+}
+
+// The plan's streams are non-blocking, so nothing orders them after the caller's work by itself: make them
+// wait for the caller's event, or for everything enqueued so far on the caller's stream.
+int order_after_caller(Ring* r, const dr_stage_desc* d)
+{
+    cudaEvent_t ev = (cudaEvent_t)d->wait_event;
+    if (!ev) {
+        if (d->flags & DR_STAGE_UNORDERED) return DR_OK;
+        DR_CUDA(cudaEventRecord(r->ev_entry, (cudaStream_t)d->caller_stream));
+        ev = r->ev_entry;
+    }
+    DR_CUDA(cudaStreamWaitEvent(r->s_copy, ev, 0));
+    DR_CUDA(cudaStreamWaitEvent(r->s_relay, ev, 0));
     return DR_OK;
 }
 
@@ -226,7 +244,7 @@ extern "C" int dr_stage_out(dr_plan* plan, const dr_stage_desc* d, dr_stage_stat
     st.n_chunks = g.n_chunks;
     st.chunks_done = std::min<uint64_t>(d->first_chunk, g.n_chunks);
     st.pinned_high_water_bytes = direct ? 0 : g.chunk * g.slots;
-    if (d->wait_event) DR_CUDA(cudaStreamWaitEvent(r->s_copy, (cudaEvent_t)d->wait_event, 0));
+    if ((rc = order_after_caller(r, d))) return rc;
 
     // ring slot of chunk k (unused when chunks are copied straight into a pinned arena)
     auto slot_ptr = [&](uint64_t k) -> char* { return r->base + (k % g.slots) * g.chunk; };
@@ -286,6 +304,7 @@ extern "C" int dr_stage_out(dr_plan* plan, const dr_stage_desc* d, dr_stage_stat
         if (rc == DR_OK && (rc = complete(next_done)) == DR_OK) st.chunks_done = ++next_done;
     }
     if (rc) drain(r);
+    if (d->done_event) cudaEventRecord((cudaEvent_t)d->done_event, relay ? r->s_relay : r->s_copy);
     st.elapsed_ms = ms_since(t0);
     st.link_gbs = st.elapsed_ms > 0 ? (double)st.bytes / st.elapsed_ms * 1e-6 : 0;
     if (stats) *stats = st;
@@ -335,7 +354,7 @@ extern "C" int dr_stage_in(dr_plan* plan, const dr_stage_desc* d, dr_stage_stats
     st.n_chunks = pieces.size();
     st.chunks_done = std::min<uint64_t>(d->first_chunk, pieces.size());
     st.pinned_high_water_bytes = direct ? 0 : g.chunk * g.slots;
-    if (d->wait_event) DR_CUDA(cudaStreamWaitEvent(r->s_copy, (cudaEvent_t)d->wait_event, 0));
+    if ((rc = order_after_caller(r, d))) return rc;
 
     auto issue = [&](uint64_t i) -> int {
         const Piece& pc = pieces[i];
@@ -376,6 +395,7 @@ extern "C" int dr_stage_in(dr_plan* plan, const dr_stage_desc* d, dr_stage_stats
         else if ((rc = complete(next_done)) == DR_OK) st.chunks_done = ++next_done;
     }
     if (rc) drain(r);
+    if (d->done_event) cudaEventRecord((cudaEvent_t)d->done_event, r->s_copy);
     st.elapsed_ms = ms_since(t0);
     st.link_gbs = st.elapsed_ms > 0 ? (double)st.bytes / st.elapsed_ms * 1e-6 : 0;
     if (stats) *stats = st;

@@ -142,9 +142,13 @@ extern "C" int dr_reshard_stream(dr_plan* plan, const dr_stream_desc* d, dr_stre
         return DR_ERR_ALIGN;
     }
     const uint64_t chunk = d->chunk_bytes ? d->chunk_bytes : d->window_bytes / 2 / 4096 * 4096;
-    if (chunk == 0 || chunk % 32 || d->window_bytes / chunk < 2) {
-        set_error("window of %llu bytes cannot hold two chunks of %llu (chunk must be a multiple of 32)",
-                  (unsigned long long)d->window_bytes, (unsigned long long)chunk);
+    if (chunk % 32) {
+        set_error("chunk_bytes %llu is not a multiple of 32", (unsigned long long)chunk);
+        return DR_ERR_INVALID;
+    }
+    if (chunk == 0 || d->window_bytes / chunk < 2) {
+        set_error("window of %llu bytes cannot hold two chunks of %llu", (unsigned long long)d->window_bytes,
+                  (unsigned long long)chunk);
         return DR_ERR_BUDGET;
     }
     int dev = -1;
@@ -162,10 +166,18 @@ extern "C" int dr_reshard_stream(dr_plan* plan, const dr_stream_desc* d, dr_stre
     st.n_chunks = s->chunks.size();
 
     // Everything is enqueued up front; a failure stops the enqueueing, and what was already enqueued is still
-    // waited for below, so that no copy or kernel of this call is in flight when it returns.
+    // waited for below.
     auto enqueue = [&]() -> int {
         uint64_t copied_below = 0;  // arena bytes already on their way to host_dst
-        DR_CUDA(cudaEventRecord(s->ev_first, s->s_h2d));
+        // The three streams are non-blocking: order them after the caller's event, or after everything the
+        // caller has enqueued so far on its stream (a fill of the arena or the window must not land later).
+        cudaEvent_t after = (cudaEvent_t)d->wait_event;
+        if (!after && !(d->flags & DR_STREAM_UNORDERED)) {
+            DR_CUDA(cudaEventRecord(s->ev_first, (cudaStream_t)d->caller_stream));
+            after = s->ev_first;
+        }
+        if (after)
+            for (cudaStream_t q : {s->s_h2d, s->s_kernel, s->s_d2h}) DR_CUDA(cudaStreamWaitEvent(q, after, 0));
         for (uint64_t k = 0; k < s->chunks.size(); ++k) {
             const ChunkTables& c = s->chunks[k];
             const uint32_t slot = (uint32_t)(k % slots);
@@ -189,12 +201,21 @@ extern "C" int dr_reshard_stream(dr_plan* plan, const dr_stream_desc* d, dr_stre
                 copied_below = c.final_below;
             }
         }
+        if (d->done_event) {  // after the last kernel (s_kernel) and the last copy back (s_d2h)
+            DR_CUDA(cudaEventRecord(s->ev_last_kernel, s->s_kernel));
+            DR_CUDA(cudaStreamWaitEvent(s->s_d2h, s->ev_last_kernel, 0));
+            DR_CUDA(cudaEventRecord((cudaEvent_t)d->done_event, s->s_d2h));
+        }
         return DR_OK;
     };
     rc = enqueue();
-    // one bounded wait for the tail of each stream
+    // One bounded wait for the tail of each stream.  When the caller's bound runs out (or enqueueing failed half
+    // way) the work already enqueued cannot be cancelled: it is waited for under a generous fixed bound, so that
+    // no copy or kernel of this call still targets the caller's buffers when the call returns.
     const auto limit = std::chrono::milliseconds(d->timeout_ms ? d->timeout_ms : 60000);
-    const auto deadline = std::chrono::steady_clock::now() + limit;
+    auto deadline = std::chrono::steady_clock::now() + limit;
+    bool draining = rc != DR_OK;
+    if (draining) deadline = std::chrono::steady_clock::now() + std::chrono::seconds(20);
     for (cudaStream_t q : {s->s_h2d, s->s_kernel, s->s_d2h}) {
         for (;;) {
             cudaError_t e = cudaStreamQuery(q);
@@ -204,9 +225,12 @@ extern "C" int dr_reshard_stream(dr_plan* plan, const dr_stream_desc* d, dr_stre
                 return DR_ERR_CUDA;
             }
             if (std::chrono::steady_clock::now() > deadline) {
+                if (draining) break;  // gave up on the drain as well: report the first error
                 set_error("streamed repack wait timed out");
-                rc = rc ? rc : DR_ERR_TIMEOUT;
-                break;
+                rc = DR_ERR_TIMEOUT;
+                draining = true;
+                deadline = std::chrono::steady_clock::now() + std::chrono::seconds(20);
+                continue;
             }
             std::this_thread::sleep_for(std::chrono::microseconds(50));
         }

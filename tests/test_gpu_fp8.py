@@ -60,6 +60,34 @@ def test_fp8_special_blocks():
     plan.close()
 
 
+@pytest.mark.parametrize("misalign", [16, 48])
+def test_fp8_sixteen_byte_aligned_bases_take_the_narrow_path(misalign):
+    """Bases that are 16- but not 32-byte aligned are legal: the quantisation kernel then reads with 128-bit
+    loads instead of 256-bit ones and produces the same bytes."""
+    spec = MID[0]["spec"]
+    om = oracle.Model(spec, tp=2, tp_rank=1)
+    total, _ = om.fp8_layout()
+    src = make_source(om.flat_elems, 71)
+    want = np.full(total, SENT8, dtype=np.uint8)
+    om.forward_fp8(src, want)
+    plan = dr.Plan(spec, tp=2, tp_rank=1, dtype=dr.DR_FP8_E4M3_B128)
+    pad = misalign // 4
+    s_buf = torch.zeros(src.size + pad, dtype=torch.int32, device=dev())
+    s_dev = s_buf[pad:]
+    s_dev.copy_(torch.from_numpy(src.view(np.int32)))
+    a_buf = torch.full((256 + misalign + total + 256,), SENT8, dtype=torch.uint8, device=dev())
+    a_dev = a_buf[256 + misalign:256 + misalign + total]
+    assert s_dev.data_ptr() % 32 == 16 and a_dev.data_ptr() % 32 == 16
+    plan.reshard(s_dev, a_dev)
+    torch.cuda.synchronize()
+    assert first_diff(a_dev.cpu().numpy(), want) is None
+    assert (a_buf[:256 + misalign] == SENT8).all() and (a_buf[256 + misalign + total:] == SENT8).all()
+    # a base that is not even 16-byte aligned is refused on the host, before any launch
+    s = torch.cuda.current_stream().cuda_stream
+    assert dr.dr_reshard(plan.handle, s_dev.data_ptr() + 4, 4 * src.size, a_dev.data_ptr(), total, s) == B.DR_ERR_ALIGN
+    plan.close()
+
+
 def test_fp8_unsupported_calls():
     spec = MID[2]["spec"]
     plan = dr.Plan(spec, dtype=dr.DR_FP8_E4M3_B128)

@@ -285,3 +285,59 @@ def test_pinned_ring_allocation_failure_is_reported_and_the_plan_stays_usable(pl
     p2.reshard(src, arena)
     torch.cuda.synchronize()
     p2.close()
+
+
+def test_stage_in_and_out_are_ordered_after_pending_work_on_the_callers_stream(plan):
+    """The pump copies on the plan's own non-blocking streams.  On entry it makes them wait for what the caller
+    has already enqueued on caller_stream, so a fill of the target buffer that is still running cannot land
+    after the first host-to-device copy, and a stage-out cannot read a buffer that is still being produced.
+    The queue of fills is long enough to be still running when the calls are made (checked with an event)."""
+    n = 1 << 22                                          # 4 Mi words of state at the head of a 1 GiB buffer
+    host = synth.fill_f32(31, synth.BUF_ADAM_M, 0, n)
+    pinned = torch.from_numpy(host.view(np.int32)).pin_memory()
+    side = torch.cuda.Stream()
+    big = torch.empty(1 << 28, dtype=torch.int32, device=dev())
+    torch.cuda.synchronize()
+    with torch.cuda.stream(side):
+        for i in range(80):
+            big.fill_(i)
+        queued = torch.cuda.Event()
+        queued.record()
+        d = dr.stage_desc([big.data_ptr()], [4 * n], budget=8 * MiB, chunk=1 * MiB, host_arena=pinned.data_ptr(),
+                          host_arena_bytes=4 * n)       # caller_stream defaults to the current stream: side
+        pending_in = not queued.query()
+        plan.stage_in(d)
+    assert pending_in, "the fills finished before the call: the test did not exercise the ordering"
+    got = big[:n].cpu().numpy().view(np.uint32)
+    assert np.array_equal(got, host)
+    assert int(big[n]) == 79                             # the rest of the buffer holds the last fill
+    # stage-out: the buffer is produced by the tail of a long queue; the image must hold the final values
+    out = torch.zeros(4 * n, dtype=torch.uint8).pin_memory()
+    with torch.cuda.stream(side):
+        for i in range(80):
+            big.fill_(i)
+        synth.cuda_fill_f32(big[:n], 37, synth.BUF_ADAM_V, stream=side)
+        queued = torch.cuda.Event()
+        queued.record()
+        d = dr.stage_desc([big.data_ptr()], [4 * n], budget=8 * MiB, chunk=1 * MiB, host_arena=out.data_ptr(),
+                          host_arena_bytes=4 * n, caller_stream=side)
+        pending_out = not queued.query()
+        plan.stage_out(d)
+    assert pending_out
+    assert np.array_equal(out.numpy().view(np.uint32), synth.fill_f32(37, synth.BUF_ADAM_V, 0, n))
+
+
+def test_done_event_and_unordered_flag(plan):
+    """done_event is recorded after the last copy; DR_STAGE_UNORDERED skips the entry ordering (the caller has
+    synchronised)."""
+    n = 300_000
+    host, devs = _state(n, 41, bufs=(1,))
+    torch.cuda.synchronize()
+    image = np.zeros(4 * n, dtype=np.uint8)
+    done = torch.cuda.Event()
+    d = dr.stage_desc([devs[0].data_ptr()], [4 * n], budget=1 * MiB, host_arena=image.ctypes.data, host_arena_bytes=4 * n,
+                      unordered=True, done_event=done.cuda_event)
+    assert d.flags & B.DR_STAGE_UNORDERED and not d.caller_stream
+    plan.stage_out(d)
+    assert done.query()                                   # the call blocks until its copies are complete
+    assert np.array_equal(image.view(np.uint32), host[0])

@@ -68,9 +68,43 @@ def test_streamed_repack_without_host_copy_and_argument_errors():
     assert st.d2h_bytes == 0 and st.n_chunks == -(-src.nbytes // (2 << 20))
     assert first_diff(arena.cpu().numpy(), want) is None
     assert dr.dr_reshard_stream(plan.handle, mk(chunk_bytes=3 << 20))[0] == B.DR_ERR_BUDGET
-    assert dr.dr_reshard_stream(plan.handle, mk(chunk_bytes=1000))[0] == B.DR_ERR_BUDGET        # not a multiple of 32
+    assert dr.dr_reshard_stream(plan.handle, mk(chunk_bytes=1000))[0] == B.DR_ERR_INVALID       # not a multiple of 32
     assert dr.dr_reshard_stream(plan.handle, mk(host_src_bytes=src.nbytes - 4))[0] == B.DR_ERR_SIZE
     assert dr.dr_reshard_stream(plan.handle, mk(window_dev=window.data_ptr() + 8))[0] == B.DR_ERR_ALIGN
     host_plan = dr.Plan(spec, tp=2, tp_rank=1, host_only=True)
     assert dr.dr_reshard_stream(host_plan.handle, mk())[0] == B.DR_ERR_STATE
+    plan.close()
+
+
+def test_streamed_repack_is_ordered_after_pending_work_on_the_callers_stream():
+    """The call's own streams are non-blocking, so the library orders them after the caller's stream on entry.
+    A long queue of arena and window fills is still running on a side stream when the call begins; without the
+    ordering the first repacked chunks would be overwritten by the late fills.  With a timing event recorded
+    after the call returns we also check that the fills really were still pending when the call was made."""
+    spec = MID[0]["spec"]
+    plan = dr.Plan(spec)
+    om = oracle.Model(spec)
+    src = make_source(om.flat_elems, 9)
+    want = np.full(om.arena_bytes, SENT8, dtype=np.uint8)
+    om.forward(src, want)
+    h_src = torch.from_numpy(src.view(np.int32)).pin_memory()
+    chunk, slots = 1 << 20, 4
+    side = torch.cuda.Stream()
+    big = torch.empty(1 << 30, dtype=torch.uint8, device=dev())
+    arena = big[:om.arena_bytes]
+    window = torch.empty(chunk * slots, dtype=torch.uint8, device=dev())
+    torch.cuda.synchronize()
+    with torch.cuda.stream(side):
+        for i in range(60):            # about 60 x 1 GiB of fills: tens of milliseconds of queued work
+            big.fill_(i)
+            window.fill_(i)
+        big.fill_(SENT8)
+        queued = torch.cuda.Event()
+        queued.record()
+        d = dr.stream_desc(h_src.data_ptr(), src.nbytes, arena.data_ptr(), om.arena_bytes, window.data_ptr(), chunk * slots,
+                           chunk_bytes=chunk)   # caller_stream = torch's current stream = side
+        still_pending = not queued.query()
+        plan.reshard_stream(d)
+    assert still_pending, "the fills finished before the call: the test did not exercise the ordering"
+    assert first_diff(arena.cpu().numpy(), want) is None
     plan.close()
