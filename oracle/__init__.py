@@ -1,7 +1,7 @@
 """TEST INFRASTRUCTURE -- not part of the product path.
 
 ctypes wrapper around ``dr_oracle.c``, the plain CPU statement of the role-switch state transform
-(layout map D1-D4, bf16 round-to-nearest-even cast D5, chunked staging D6).  Only ``tests/``,
+(layout map D1-D4, bf16 round-to-nearest-even cast D5, chunked staging D6, fp8 block scaling D7).  Only ``tests/``,
 ``__graft_entry__.smoke()`` and the bench's CPU-baseline / ``--impl reference`` legs may import this.
 It shares no code with the CUDA library and never imports it.
 """
@@ -84,6 +84,8 @@ def _l():
         lib.orc_fp8_layout.argtypes = [p, u64, ctypes.POINTER(ctypes.c_int), ctypes.POINTER(u64), ctypes.POINTER(u64)]
         lib.orc_forward_fp8.restype = ctypes.c_int
         lib.orc_forward_fp8.argtypes = [p, p, p, i64]
+        lib.orc_inverse_fp8.restype = ctypes.c_int
+        lib.orc_inverse_fp8.argtypes = [p, p, p]
         lib.orc_restage_out.restype = None
         lib.orc_restage_out.argtypes = [p, u64, u64, u64, p]
         lib.orc_restage_in.restype = None
@@ -207,6 +209,12 @@ class Model:
         assert src_u32.dtype == np.uint32 and src_u32.flags.c_contiguous and src_u32.size >= self.flat_elems
         assert arena_u8.dtype == np.uint8 and arena_u8.size >= self.fp8_layout()[0]
         _l().orc_forward_fp8(self._h, src_u32.ctypes.data, arena_u8.ctypes.data, only)
+
+    def inverse_fp8(self, arena_u8: np.ndarray, flat_u32: np.ndarray) -> None:
+        """Inverse of D7: codes times block scales (and widened bf16 tensors) back to their flat positions."""
+        assert flat_u32.dtype == np.uint32 and flat_u32.flags.c_contiguous and flat_u32.size >= self.flat_elems
+        assert arena_u8.dtype == np.uint8 and arena_u8.flags.c_contiguous and arena_u8.size >= self.fp8_layout()[0]
+        _l().orc_inverse_fp8(self._h, arena_u8.ctypes.data, flat_u32.ctypes.data)
 
     def inverse(self, arena_u8: np.ndarray, flat_u32: np.ndarray, *, gathered: bool = True, rank: int = 0) -> None:
         assert flat_u32.dtype == np.uint32 and flat_u32.flags.c_contiguous

@@ -24,6 +24,7 @@
  * source with world W, rank r, per-parameter alignment A; rollout layout at
  * tensor-parallel degree T, rank t.  All matrices are [out, in] row-major.
  */
+#include <float.h>
 #include <math.h>
 #include <stdint.h>
 #include <stdio.h>
@@ -634,17 +635,18 @@ void orc_restage_in(const uint32_t *image, uint64_t N, uint64_t W_new, uint64_t 
 /* ---- D7: fp8 (e4m3) rollout weights with one fp32 scale per 128 x 128 block ----------------------
  * A reading for rollout engines that serve block-quantised weights (the paper is silent).  The linear
  * weights (qkv, o, gate_up, down, w13, w2) are quantised; embeddings, lm_head, router and norms stay
- * bf16.  For a quantised rollout tensor X[rows, cols]:
+ * bf16.  The definition is the plain one of scaled quantisation: the stored code is the e4m3 rounding
+ * of x / scale, where scale is the number a consumer multiplies the code by to get x back.  For a
+ * quantised rollout tensor X[rows, cols]:
  *   block (bi, bj) = rows [128 bi, 128 bi + 128) x cols [128 bj, 128 bj + 128), clipped to the tensor;
- *   amax  = max |x| over the block, NaNs skipped, starting from 0;
- *   scale = amax / 448 in fp32 (round to nearest), the number a consumer multiplies by to dequantise;
- *   r     = 448 / amax in fp32 (round to nearest), the number the quantiser multiplies by;
- *           an all-zero block (amax = 0) takes scale = r = 1;
- *   q     = e4m3( x * r ), one fp32 multiplication (round to nearest), then round to nearest even onto
+ *   amax  = max |x| over the block, NaNs skipped (infinities count), starting from 0;
+ *   scale = amax / 448 in fp32 (one division, round to nearest), then clamped to
+ *           [2^-126, FLT_MAX]: the smallest normal fp32 for blocks whose amax / 448 would be zero or
+ *           subnormal (the all-zero block among them), so that x / scale and code * scale stay finite
+ *           and zeros stay zeros; the largest finite fp32 for a block holding an infinity;
+ *   q     = e4m3( x / scale ): one fp32 division (round to nearest), then round to nearest even onto
  *           the e4m3 grid (3 mantissa bits, bias 7, subnormal step 2^-9), magnitudes above 448 saturate
  *           to 448 (code 0x7E), NaN becomes 0x7F.
- * (The multiply-by-reciprocal form is the one public block-quantisation references use; per element it
- * costs one multiplication instead of a division.)
  * Arena: payload rows*cols bytes at arena_off, then the scales [ceil(rows/128), ceil(cols/128)] fp32,
  * row-major, at the next multiple of arena_align.
  */
@@ -778,7 +780,7 @@ int orc_forward_fp8(const orc_model *m, const uint32_t *src, uint8_t *arena, int
                 for (bj = 0; bj < nbc; ++bj) {
                     uint64_t r1 = bi * 128 + 128 < d->rows ? bi * 128 + 128 : d->rows;
                     uint64_t c1 = bj * 128 + 128 < d->cols ? bj * 128 + 128 : d->cols;
-                    float amax = 0.0f, scale, recip;
+                    float amax = 0.0f, scale;
                     for (r = bi * 128; r < r1; ++r)
                         for (c = bj * 128; c < c1; ++c) {
                             uint32_t mag = x[r * d->cols + c] & 0x7FFFFFFFu;
@@ -788,8 +790,8 @@ int orc_forward_fp8(const orc_model *m, const uint32_t *src, uint8_t *arena, int
                             if (a > amax) amax = a;
                         }
                     scale = amax / 448.0f;
-                    recip = 448.0f / amax;
-                    if (amax == 0.0f) scale = recip = 1.0f;
+                    if (scale < FLT_MIN) scale = FLT_MIN; /* 2^-126 */
+                    if (scale > FLT_MAX) scale = FLT_MAX; /* amax was an infinity */
                     memcpy(arena + soff + (bi * nbc + bj) * 4, &scale, 4);
                     for (r = bi * 128; r < r1; ++r)
                         for (c = bj * 128; c < c1; ++c) {
@@ -797,13 +799,53 @@ int orc_forward_fp8(const orc_model *m, const uint32_t *src, uint8_t *arena, int
                             uint32_t qb;
                             if (!has[r]) continue;
                             memcpy(&v, &x[r * d->cols + c], 4);
-                            qv = v * recip;
+                            qv = v / scale;
                             memcpy(&qb, &qv, 4);
                             arena[off + r * d->cols + c] = orc_cast_e4m3(qb);
                         }
                 }
             free(x);
             free(has);
+        }
+    }
+    return 0;
+}
+
+/* Inverse of D7: Rollout -> Training from an fp8 arena.  A bf16 rollout tensor is widened exactly, as in
+ * the base definition.  An element of a quantised tensor becomes value(code) * scale of its block: the
+ * exact e4m3 value, one fp32 multiplication (round to nearest); a NaN code, or a NaN product (a scale
+ * that is itself NaN, or 0 * Inf), becomes the quiet NaN 0x7FC00000.  Positions no rollout element maps
+ * to keep their words. */
+int orc_inverse_fp8(const orc_model *m, const uint8_t *arena, uint32_t *flat)
+{
+    uint64_t i, p, r, c;
+    for (i = 0; i < m->n_dst; ++i) {
+        const orc_dst *d = &m->dst[i];
+        int qz;
+        uint64_t off, soff, nbc = (d->cols + 127) / 128;
+        if (d->alias_of >= 0) continue;
+        orc_fp8_layout(m, i, &qz, &off, &soff);
+        for (p = 0; p < d->n_parts; ++p) {
+            const orc_part *q = &d->parts[p];
+            const orc_src *s = &m->src[q->src];
+            for (r = 0; r < q->rows; ++r)
+                for (c = 0; c < d->cols; ++c) {
+                    uint64_t f = s->flat_off + (q->src_row0 + r) * s->cols + (q->src_col0 + c);
+                    uint64_t row = q->dst_row0 + r;
+                    if (!qz) {
+                        uint16_t b;
+                        memcpy(&b, arena + off + (row * d->cols + c) * 2, 2);
+                        flat[f] = orc_widen_bf16(b);
+                    } else {
+                        float scale, y;
+                        uint32_t bits;
+                        memcpy(&scale, arena + soff + ((row / 128) * nbc + c / 128) * 4, 4);
+                        y = orc_e4m3_value(arena[off + row * d->cols + c]) * scale;
+                        memcpy(&bits, &y, 4);
+                        if ((bits & 0x7FFFFFFFu) > 0x7F800000u) bits = 0x7FC00000u;
+                        flat[f] = bits;
+                    }
+                }
         }
     }
     return 0;
