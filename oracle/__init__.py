@@ -75,7 +75,7 @@ def _l():
         lib.orc_stage_out.restype = i64
         lib.orc_stage_out.argtypes = [p, p, u64, u64, u64, u64, p, p]
         lib.orc_stage_in.restype = i64
-        lib.orc_stage_in.argtypes = [p, p, u64, p, u64, u64, p, p]
+        lib.orc_stage_in.argtypes = [p, p, u64, p, u64, u64, p, p, p]
         lib.orc_cast_e4m3.restype = ctypes.c_uint8
         lib.orc_cast_e4m3.argtypes = [ctypes.c_uint32]
         lib.orc_e4m3_value.restype = ctypes.c_float
@@ -244,14 +244,20 @@ def stage_out(bufs: list[np.ndarray], budget: int, chunk: int = 0, first_chunk: 
     return sink, sizes[:n]
 
 
-def stage_in(bufs: list[np.ndarray], source: np.ndarray, budget: int, chunk: int = 0, order=None):
-    """D6 stage-in into bufs (in place), buffers restored in ``order``; returns (pieces, completion order)."""
+def stage_in(bufs: list[np.ndarray], source: np.ndarray, budget: int, chunk: int = 0, order=None, pieces=False):
+    """D6 stage-in into bufs (in place), buffers restored in ``order``; returns (piece count, completion
+    order), plus the walk itself as a list of (buffer, position, bytes) when ``pieces`` is set."""
     arr, nb = _ptr_array(bufs)
     o = (ctypes.c_uint32 * len(bufs))(*(order if order is not None else range(len(bufs))))
     done = (ctypes.c_uint32 * len(bufs))()
-    n = _l().orc_stage_in(arr, nb, len(bufs), o, budget, chunk, source.ctypes.data, done)
+    c = chunk or budget // 2 // 4096 * 4096
+    cap = sum(-(-b.nbytes // c) for b in bufs) if c else 0
+    walk = np.zeros((max(cap, 1), 3), dtype=np.uint64)
+    n = _l().orc_stage_in(arr, nb, len(bufs), o, budget, chunk, source.ctypes.data, done, walk.ctypes.data)
     if n < 0:
         raise ValueError("oracle: budget cannot hold two slots")
+    if pieces:
+        return int(n), list(done), [tuple(int(x) for x in row) for row in walk[:n]]
     return int(n), list(done)
 
 

@@ -578,12 +578,17 @@ int64_t orc_stage_out(const uint8_t *const *bufs, const uint64_t *bytes, uint64_
     return (int64_t)n_chunks;
 }
 
-/* Stage-in: buffers are restored in `order` (weights first); within a buffer, bytes arrive in
- * ring-sized pieces of C bytes.  completed[i] receives the position at which order[i] finished. */
+/* Stage-in (Sec. 3.3: weights at the transition, optimizer state deferred): buffers are restored one
+ * after the other in `order` (weights first), and each buffer on its own is cut into pieces of at most C
+ * bytes, so a piece never holds bytes of two buffers and buffer order[0] is whole before the first byte
+ * of order[1] moves.  Piece number i goes through ring slot i mod slots.  The walk is recorded:
+ * piece_list receives (buffer, position inside the buffer, bytes) for every piece in the order taken,
+ * completed[o] the buffer that became whole o-th.  Returns the number of pieces. */
 int64_t orc_stage_in(uint8_t *const *bufs, const uint64_t *bytes, uint64_t n_bufs, const uint32_t *order,
-                     uint64_t budget, uint64_t chunk, const uint8_t *source, uint32_t *completed)
+                     uint64_t budget, uint64_t chunk, const uint8_t *source, uint32_t *completed,
+                     uint64_t *piece_list)
 {
-    uint64_t b, o, slots, pieces = 0, i;
+    uint64_t b, o, slots, pieces = 0, i, n_completed = 0;
     uint8_t *ring;
     if (chunk == 0) chunk = budget / 2 / 4096 * 4096;
     if (chunk == 0) return -1;
@@ -599,9 +604,15 @@ int64_t orc_stage_in(uint8_t *const *bufs, const uint64_t *bytes, uint64_t n_buf
             uint8_t *slot = ring + (pieces % slots) * chunk;
             for (i = 0; i < n; ++i) slot[i] = source[base + pos + i];          /* source -> ring slot */
             for (i = 0; i < n; ++i) stream_put(bufs, bytes, n_bufs, base + pos + i, slot[i]); /* -> device */
+            if (piece_list) {
+                piece_list[3 * pieces] = b;
+                piece_list[3 * pieces + 1] = pos;
+                piece_list[3 * pieces + 2] = n;
+            }
             pieces++;
         }
-        if (completed) completed[o] = (uint32_t)b;
+        if (completed) completed[n_completed] = (uint32_t)b; /* every byte of b has now been put */
+        n_completed++;
     }
     free(ring);
     return (int64_t)pieces;

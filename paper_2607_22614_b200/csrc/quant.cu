@@ -3,9 +3,16 @@
 // One CTA per block: 512 threads hold the block's 16 384 values in registers (four 256-bit loads in
 // flight per thread, three CTAs per SM, each row of the block one contiguous 512 B request), reduce |x| to the block
 // maximum with shuffles and one shared-memory step, then
-// multiply by the block's reciprocal scale, convert two values per cvt.rn.satfinite.e4m3x2.f32 and store
+// divide by the block's scale, convert two values per cvt.rn.satfinite.e4m3x2.f32 and store
 // each row as one contiguous 128 B request.  The bound is HBM: 4 B read + 1 B written per element (+ 4 B
 // per 16 384 elements for the scale).
+//
+// The definition is code = e4m3(fl32(x / scale)).  A correctly rounded fp32 division costs about twenty
+// instructions, which would make the kernel issue-bound, so the quotient is taken as t = x * fl32(1 / scale)
+// wherever that provably gives the same code: t and the true quotient differ by at most 2 ulp, so they can
+// round to different e4m3 codes only if t lies within a few ulp of a midpoint between two codes (its 20 dropped
+// mantissa bits within 4 of 0x80000) or below 2^-6, where the e4m3 grid is no longer 3 mantissa bits wide.
+// Those elements (about one in 10^4 for weight-like data) take the exact division.
 #include <cuda_runtime.h>
 
 #include "dr_internal.h"
@@ -50,6 +57,15 @@ __device__ __forceinline__ uint32_t cvt_e4m3x2(float lo, float hi)
     asm("cvt.rn.satfinite.e4m3x2.f32 %0, %1, %2;" : "=h"(d) : "f"(hi), "f"(lo));
     return d;
 }
+// x / scale as far as the e4m3 code is concerned: the product with the reciprocal, or the correctly rounded
+// division where the product could round to a different code (see the header of this file).
+__device__ __forceinline__ float quotient(float x, float scale, float recip, float exact_below)
+{
+    float t = __fmul_rn(x, recip);
+    const uint32_t low = __float_as_uint(t) & 0xFFFFFu;
+    if (low - (0x80000u - 4u) <= 8u || fabsf(t) < exact_below) t = __fdiv_rn(x, scale);
+    return t;
+}
 __global__ void __launch_bounds__(kQThreads, DR_Q_MIN_BLOCKS)
     quant_kernel(const QTensor* __restrict__ tensors, uint32_t n_tensors, const QPart* __restrict__ parts,
                  const uint32_t* __restrict__ hints, uint32_t hint_shift, const char* __restrict__ flat,
@@ -57,7 +73,7 @@ __global__ void __launch_bounds__(kQThreads, DR_Q_MIN_BLOCKS)
 {
     __shared__ uint64_t row_src[128];  // flat element offset of (row, first column of the tensor)
     __shared__ float warp_max[kQThreads / 32];
-    __shared__ float s_recip;
+    __shared__ float s_scale;
 
     const uint64_t b = blockIdx.x;
     // block -> tensor: hint plus a short walk (all threads, same addresses: broadcast loads)
@@ -124,13 +140,18 @@ __global__ void __launch_bounds__(kQThreads, DR_Q_MIN_BLOCKS)
         float m = warp_max[0];
 #pragma unroll
         for (int w = 1; w < kQThreads / 32; ++w) m = fmaxf(m, warp_max[w]);
-        float scale = __fdiv_rn(m, 448.0f), recip = __fdiv_rn(448.0f, m);
-        if (m == 0.0f) scale = recip = 1.0f;
-        s_recip = recip;
+        // amax / 448, held inside the normal fp32 range: 2^-126 for blocks whose amax / 448 underflows (the
+        // all-zero block among them), FLT_MAX for a block holding an infinity
+        float scale = fminf(fmaxf(__fdiv_rn(m, 448.0f), 1.17549435e-38f), 3.40282347e+38f);
+        s_scale = scale;
         *(float*)(arena + T.scale_off + ((uint64_t)bi * T.nbc + bj) * 4) = scale;
     }
     __syncthreads();
-    const float recip = s_recip;
+    const float scale = s_scale;
+    const float recip = __frcp_rn(scale);
+    // the product form needs a normal reciprocal (scale <= 2^126: always, except for the infinity block);
+    // otherwise every element takes the exact division
+    const float exact_below = recip >= 1.17549435e-38f ? 0.015625f : __int_as_float(0x7F800000);
 
 #pragma unroll
     for (int p = 0; p < kPasses; ++p) {
@@ -139,7 +160,8 @@ __global__ void __launch_bounds__(kQThreads, DR_Q_MIN_BLOCKS)
         uint32_t q[8];
 #pragma unroll
         for (int k = 0; k < 8; k += 2) {
-            const float a = __fmul_rn(v[p][k], recip), c = __fmul_rn(v[p][k + 1], recip);
+            const float a = quotient(v[p][k], scale, recip, exact_below);
+            const float c = quotient(v[p][k + 1], scale, recip, exact_below);
             const uint32_t two = cvt_e4m3x2(a, c);
             q[k] = two & 0xFF;
             q[k + 1] = two >> 8;

@@ -120,9 +120,11 @@ def test_random_staging_geometries(c):
                 assert (image.numpy()[offsets[i] + h.size:offsets[i] + h.size + 64] == 0x5A).all()
     assert st_out.n_chunks == st_out.chunks_done == len(csz) and st_out.bytes == total
     back = [torch.zeros_like(t) for t in devs]
+    asked = []
     if c["sink"] == "callback":
         @dr.dr_chunk_fn
         def source(user, k, off, ptr, n):
+            asked.append((k, off, n))
             C.memmove(ptr, want.ctypes.data + off, n)
             return 0
         st_in = plan.stage_in(dr.stage_desc([t.data_ptr() for t in back], c["sizes"], callback=source, order=c["order"], **kw))
@@ -130,8 +132,14 @@ def test_random_staging_geometries(c):
         st_in = plan.stage_in(dr.stage_desc([t.data_ptr() for t in back], c["sizes"], host_arena=image.data_ptr(),
                                             host_arena_bytes=image.numel(), host_offsets=offsets, order=c["order"], **kw))
     ob = [np.zeros(n, dtype=np.uint8) for n in c["sizes"]]
-    pieces, done = oracle.stage_in(ob, want, c["budget"], c["chunk"], c["order"])
+    pieces, done, walk = oracle.stage_in(ob, want, c["budget"], c["chunk"], c["order"], pieces=True)
     assert st_in.chunks_done == st_in.n_chunks == pieces and done == c["order"]
+    if c["sink"] == "callback":  # the pieces the engine asked for are the oracle's walk, in its order
+        prefix = np.concatenate([[0], np.cumsum(c["sizes"])])
+        assert asked == [(i, int(prefix[b]) + pos, nb) for i, (b, pos, nb) in enumerate(walk)]
+    # buffers became resident in the asked order (empty buffers never report a time)
+    ready = [st_in.ready_ms[b] for b in c["order"] if c["sizes"][b]]
+    assert all(x > 0 for x in ready) and ready == sorted(ready)
     for b, h, o in zip(back, host, ob):
         assert np.array_equal(b.cpu().numpy()[:h.size], h) and np.array_equal(o, h)
     plan.close()

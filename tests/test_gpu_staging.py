@@ -104,17 +104,27 @@ def test_callback_sink_failure_and_resume(plan):
     assert [c[2] for c in calls] == [int(x) for x in sizes_k]
     assert np.array_equal(got, want)
 
-    # stage-in from a callback source
+    # stage-in from a callback source: the pieces asked for, in order, are the oracle's walk (buffer 2 first,
+    # every buffer cut on its own, no piece straddling two buffers)
+    asked = []
+
     @dr.dr_chunk_fn
     def source(user, k, off, ptr, n):
+        asked.append((k, off, n))
         C.memmove(ptr, want.ctypes.data + off, n)
         return 0
 
     back = [torch.zeros_like(t) for t in devs]
     d = dr.stage_desc([t.data_ptr() for t in back], sizes, budget=64 * 1024, chunk=16 * 1024, callback=source,
                       order=[2, 0, 1])
-    plan.stage_in(d)
+    st = plan.stage_in(d)
     assert all(torch.equal(a, b) for a, b in zip(back, devs))
+    ob = [np.zeros(n, dtype=np.uint8) for n in sizes]
+    n_pieces, done, walk = oracle.stage_in(ob, want, 64 * 1024, 16 * 1024, order=[2, 0, 1], pieces=True)
+    prefix = np.concatenate([[0], np.cumsum(sizes)])
+    assert asked == [(i, int(prefix[b]) + pos, nb) for i, (b, pos, nb) in enumerate(walk)]
+    assert st.n_chunks == n_pieces and done == [2, 0, 1]
+    assert [b for b, _, _ in walk][:16] == [2] * 16      # 250 001 bytes of buffer 2 = 16 pieces, before anything else
 
 
 def test_relay_sink_moves_state_to_other_device_buffers(plan):

@@ -44,6 +44,56 @@ def test_tiny_workload_chunking_matches_the_quoted_figures():
     assert np.array_equal(sink, np.concatenate(bufs))
 
 
+def test_stage_in_walks_buffers_in_order_in_pieces_that_never_straddle_hand_written():
+    """The walk of stage-in, written out by hand.  Tiny workload: Adam m and v of 3 951 616 bytes each
+    (7 x 524 288 + 281 600), 1 MiB budget, v asked for first: eight pieces of v, then eight of m."""
+    shard_bytes = 987_904 * 4
+    assert shard_bytes == 7 * 524_288 + 281_600
+    bufs = _bufs((shard_bytes, shard_bytes), 2)
+    back = [np.zeros_like(b) for b in bufs]
+    n, done, walk = oracle.stage_in(back, np.concatenate(bufs), 1 << 20, order=[1, 0], pieces=True)
+    expected = [
+        (1, 0, 524_288), (1, 524_288, 524_288), (1, 1_048_576, 524_288), (1, 1_572_864, 524_288),
+        (1, 2_097_152, 524_288), (1, 2_621_440, 524_288), (1, 3_145_728, 524_288), (1, 3_670_016, 281_600),
+        (0, 0, 524_288), (0, 524_288, 524_288), (0, 1_048_576, 524_288), (0, 1_572_864, 524_288),
+        (0, 2_097_152, 524_288), (0, 2_621_440, 524_288), (0, 3_145_728, 524_288), (0, 3_670_016, 281_600),
+    ]
+    assert n == 16 and walk == expected and done == [1, 0]
+    assert all(np.array_equal(a, b) for a, b in zip(back, bufs))
+    # three buffers of 5, 0 and 3 bytes, pieces of 2 bytes, order 2, 0, 1: the empty buffer has no piece
+    bufs = _bufs((5, 0, 3), 4)
+    back = [np.zeros_like(b) for b in bufs]
+    n, done, walk = oracle.stage_in(back, np.concatenate(bufs), 4, 2, order=[2, 0, 1], pieces=True)
+    assert walk == [(2, 0, 2), (2, 2, 1), (0, 0, 2), (0, 2, 2), (0, 4, 1)] and n == 5 and done == [2, 0, 1]
+    assert all(np.array_equal(a, b) for a, b in zip(back, bufs))
+
+
+def test_stage_in_walk_properties_on_random_geometries():
+    """Whatever the sizes: pieces of one buffer are consecutive and cover it from 0 upwards without gaps,
+    none is longer than the chunk, buffers appear in the asked order, nothing straddles."""
+    rng = np.random.default_rng(8)
+    for _ in range(40):
+        k = int(rng.integers(1, 5))
+        sizes = [int(rng.integers(0, 5000)) for _ in range(k)]
+        chunk = int(rng.integers(1, 1500))
+        order = [int(x) for x in rng.permutation(k)]
+        bufs = _bufs(sizes, 5)
+        back = [np.zeros_like(b) for b in bufs]
+        n, done, walk = oracle.stage_in(back, np.concatenate(bufs) if sum(sizes) else np.zeros(1, np.uint8), 3 * chunk, chunk,
+                                        order=order, pieces=True)
+        assert done == order
+        seen_order, cursor = [], {}
+        for b, pos, nb in walk:
+            if not seen_order or seen_order[-1] != b:
+                assert b not in seen_order          # a buffer's pieces are consecutive
+                seen_order.append(b)
+            assert pos == cursor.get(b, 0) and 0 < nb <= chunk and pos + nb <= sizes[b]
+            cursor[b] = pos + nb
+        assert seen_order == [b for b in order if sizes[b]]
+        assert all(cursor.get(b, 0) == sizes[b] for b in range(k))
+        assert all(np.array_equal(a, b) for a, b in zip(back, bufs))
+
+
 def test_resume_from_a_failed_chunk_gives_the_same_bytes():
     bufs = _bufs((9000, 7000), 3)
     full, csz = oracle.stage_out(bufs, 4096, 1024)
