@@ -240,6 +240,45 @@ int dr_reshard_groups(const dr_plan* plan, uint32_t first, uint32_t count, const
                       void* dst_dev, uint64_t dst_bytes, void* cuda_stream);
 
 /*
+ * Exchange after the local repack (Sec. 3.2: the weight synchronisation between roles that follows a
+ * switch).  With gathered = 0 every FSDP rank repacks only the rollout elements whose sources lie in its
+ * own shard; a rollout rank then needs the pieces of all W training ranks.  The pieces are already cast
+ * to bf16, so they cross the links at half the bytes of gathering fp32 first.
+ *
+ * dr_plan_ranges -- the arena byte ranges [off, off + bytes) that dr_reshard on this plan writes,
+ * ascending and coalesced (touching ranges merged).  Host arithmetic only.  Over the W shard-local plans
+ * of one (tp, rank) these ranges are pairwise disjoint and their union is the range set of the gathered
+ * plan: they are the send / receive lists of an all-gather of the repacked pieces.  Writes at most
+ * max_ranges entries to out (out may be NULL when max_ranges is 0) and always the full count to
+ * *n_ranges.  Not for fp8 plans (DR_ERR_UNSUPPORTED).
+ */
+typedef struct dr_range {
+    uint64_t off, bytes;
+} dr_range;
+int dr_plan_ranges(const dr_plan* plan, uint64_t max_ranges, dr_range* out, uint64_t* n_ranges);
+
+/*
+ * dr_reshard_push -- dr_reshard fused with the exchange: the same gather / cast kernel stores every
+ * element it produces into n_dst rollout arenas instead of one, so that a training rank repacks its
+ * shard and delivers the pieces to the rollout ranks in one pass over its master shard, with no packed
+ * send buffer and no second kernel.  dst_dev[i] are device pointers this GPU can store to: its own
+ * memory, or peers' arenas mapped into this process (CUDA IPC or any other peer mapping, peer access
+ * enabled by the caller); plain peer stores over NVLink, no multicast of any kind.  Every arena gets
+ * exactly the bytes dr_reshard would write (the plan's dr_plan_ranges); all else keeps its bytes.
+ *   n_dst   : 1 .. DR_MAX_PUSH_DST
+ *   dst_dev : n_dst arena base pointers, each 16-byte aligned and dst_bytes large
+ * The kernel waits on nothing and signals nothing: a consumer on another GPU may read its arena only
+ * after the pushing rank's stream has reached the point after this call (an event shared between the
+ * processes, or a host-side barrier after a stream synchronise), which is the caller's to arrange.
+ * Once all W ranks of one (tp, rank) have pushed, every arena holds the gathered plan's result.
+ * Asynchronous on cuda_stream; errors as dr_reshard, plus DR_ERR_INVALID for a bad n_dst or a NULL
+ * entry and DR_ERR_UNSUPPORTED for fp8 plans.
+ */
+#define DR_MAX_PUSH_DST 8u
+int dr_reshard_push(const dr_plan* plan, const void* src_dev, uint64_t src_bytes, void* const* dst_dev, uint32_t n_dst,
+                    uint64_t dst_bytes, void* cuda_stream);
+
+/*
  * dr_reshard_static -- dr_reshard for callers that must not allocate device memory.  (The paper has
  * no counterpart; this is a deployment aid.)
  *
@@ -449,6 +488,29 @@ int dr_ctl_observe(dr_ctl* ctl, double t_rollout, double t_train, int32_t* move,
  * infinity when the step did not get faster. */
 int dr_ctl_break_even(double resize_cost_s, double step_before_s, double step_after_s, double* steps);
 int dr_ctl_destroy(dr_ctl* ctl);
+
+/*
+ * dr_probe_stream -- measurement aid (the paper has no counterpart): a trivial contiguous streaming
+ * kernel in the repack kernel's launch shape, so that a benchmark can measure, in the same run as the
+ * repack, what this GPU sustains for the repack's read : write mix.  n_bytes counts the wider side and
+ * must be a multiple of 49 152 (one CTA's tile); both buffers 32-byte aligned.
+ *   DR_PROBE_READ   reads n_bytes of a_dev                       (b_dev unused, may be NULL)
+ *   DR_PROBE_WRITE  writes n_bytes to b_dev                      (a_dev unused, may be NULL)
+ *   DR_PROBE_COPY   copies n_bytes a_dev -> b_dev                (1 : 1)
+ *   DR_PROBE_NARROW reads n_bytes of fp32, writes n_bytes / 2 of bf16 (2 : 1, the forward repack's mix)
+ *   DR_PROBE_WIDEN  reads n_bytes / 2 of bf16, writes n_bytes of fp32 (1 : 2, the inverse map's mix)
+ * Asynchronous on cuda_stream.  Errors: DR_ERR_INVALID, DR_ERR_ALIGN, DR_ERR_UNSUPPORTED, DR_ERR_CUDA.
+ */
+enum { DR_PROBE_READ = 0, DR_PROBE_WRITE = 1, DR_PROBE_COPY = 2, DR_PROBE_NARROW = 3, DR_PROBE_WIDEN = 4 };
+int dr_probe_stream(uint32_t mode, const void* a_dev, void* b_dev, uint64_t n_bytes, void* cuda_stream);
+
+/*
+ * dr_host_copy -- measurement aid (the paper has no counterpart): the multi-threaded host copy that the
+ * staging engine uses between its pinned ring and a pageable arena, run on its own, so that a benchmark
+ * can state what the host's cores sustain without the link (the CPU baseline of staging through pageable
+ * memory).  threads = 0 takes the engine's own count (at most 16).  Blocking.  DR_ERR_INVALID on NULL.
+ */
+int dr_host_copy(void* dst_host, const void* src_host, uint64_t n_bytes, uint32_t threads);
 
 /* Synchronises the plan's own streams, frees its ring, table and streams.  NULL is accepted. */
 int dr_plan_destroy(dr_plan* plan);

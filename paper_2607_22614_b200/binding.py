@@ -20,8 +20,8 @@ DR_STAGE_UNORDERED = 2
 DR_STREAM_UNORDERED = 1
 
 EXPORTS = ["dr_plan_create", "dr_plan_create_host", "dr_plan_window_host", "dr_plan_query", "dr_plan_tensor", "dr_plan_segment",
-           "dr_reshard", "dr_reshard_inverse", "dr_plan_group", "dr_reshard_groups", "dr_reshard_static", "dr_reshard_stream", "dr_shard_range", "dr_stage_out", "dr_stage_in", "dr_plan_destroy", "dr_strerror",
-           "dr_last_error", "dr_ctl_create", "dr_ctl_observe", "dr_ctl_break_even", "dr_ctl_destroy"]
+           "dr_reshard", "dr_reshard_inverse", "dr_plan_group", "dr_reshard_groups", "dr_reshard_static", "dr_plan_ranges", "dr_reshard_push", "dr_reshard_stream", "dr_shard_range", "dr_stage_out", "dr_stage_in", "dr_plan_destroy", "dr_strerror",
+           "dr_last_error", "dr_probe_stream", "dr_host_copy", "dr_ctl_create", "dr_ctl_observe", "dr_ctl_break_even", "dr_ctl_destroy"]
 
 u8, u32, u64, i64, vp = C.c_uint8, C.c_uint32, C.c_uint64, C.c_int64, C.c_void_p
 
@@ -50,6 +50,10 @@ class dr_plan_info(C.Structure):
 
 class dr_group_desc(C.Structure):
     _fields_ = [("first_tensor", u32), ("n_tensors", u32), ("elems", u64), ("bytes_moved", u64)]
+
+
+class dr_range(C.Structure):
+    _fields_ = [("off", u64), ("bytes", u64)]
 
 
 class dr_tensor_desc(C.Structure):
@@ -121,6 +125,8 @@ def lib() -> C.CDLL:
         L.dr_reshard.argtypes = [vp, vp, u64, vp, u64, vp]
         L.dr_reshard_inverse.argtypes = [vp, vp, u64, vp, u64, vp]
         L.dr_reshard_static.argtypes = [vp, vp, u64, vp, u64, vp]
+        L.dr_plan_ranges.argtypes = [vp, u64, P(dr_range), P(u64)]
+        L.dr_reshard_push.argtypes = [vp, vp, u64, P(vp), u32, u64, vp]
         L.dr_plan_group.argtypes = [vp, u32, P(dr_group_desc)]
         L.dr_reshard_groups.argtypes = [vp, u32, u32, vp, u64, vp, u64, vp]
         L.dr_stage_out.argtypes = [vp, P(dr_stage_desc), P(dr_stage_stats)]
@@ -128,6 +134,8 @@ def lib() -> C.CDLL:
         L.dr_reshard_stream.argtypes = [vp, P(dr_stream_desc), P(dr_stream_stats)]
         L.dr_plan_destroy.argtypes = [vp]
         L.dr_shard_range.argtypes = [u64, u32, u32, P(u64), P(u64), P(u64)]
+        L.dr_probe_stream.argtypes = [u32, vp, vp, u64, vp]
+        L.dr_host_copy.argtypes = [vp, vp, u64, u32]
         L.dr_ctl_create.argtypes = [P(dr_ctl_config), P(vp)]
         L.dr_ctl_observe.argtypes = [vp, C.c_double, C.c_double, P(C.c_int32), P(u32)]
         L.dr_ctl_break_even.argtypes = [C.c_double, C.c_double, C.c_double, P(C.c_double)]
@@ -256,6 +264,22 @@ def dr_reshard_groups(plan, first, count, src_dev, src_bytes, dst_dev, dst_bytes
     return lib().dr_reshard_groups(plan, first, count, src_dev, src_bytes, dst_dev, dst_bytes, cuda_stream)
 
 
+def dr_plan_ranges(plan):
+    """(status, [(off, bytes), ...]): the coalesced arena byte ranges the plan's repack writes."""
+    n = u64()
+    rc = lib().dr_plan_ranges(plan, 0, None, C.byref(n))
+    if rc:
+        return rc, []
+    arr = (dr_range * max(n.value, 1))()
+    rc = lib().dr_plan_ranges(plan, n.value, arr, C.byref(n))
+    return rc, [(arr[i].off, arr[i].bytes) for i in range(n.value)]
+
+
+def dr_reshard_push(plan, src_dev, src_bytes, dst_devs, dst_bytes, cuda_stream):
+    arr = (vp * len(dst_devs))(*dst_devs)
+    return lib().dr_reshard_push(plan, src_dev, src_bytes, arr, len(dst_devs), dst_bytes, cuda_stream)
+
+
 def dr_reshard_static(plan, src_dev, src_bytes, dst_dev, dst_bytes, cuda_stream):
     """dr_reshard without any device allocation: the segment table goes into the library's fixed
     1 MiB table (at most 16 384 segments).  For workers whose memory pool owns the whole GPU, or whose
@@ -288,6 +312,17 @@ def stream_desc(host_src, host_src_bytes, dst_dev, dst_bytes, window_dev, window
 def dr_reshard_stream(plan, desc):
     st = dr_stream_stats()
     return lib().dr_reshard_stream(plan, C.byref(desc), C.byref(st)), st
+
+
+DR_PROBE_READ, DR_PROBE_WRITE, DR_PROBE_COPY, DR_PROBE_NARROW, DR_PROBE_WIDEN = range(5)
+
+
+def dr_probe_stream(mode, a_dev, b_dev, n_bytes, cuda_stream):
+    return lib().dr_probe_stream(mode, a_dev, b_dev, n_bytes, cuda_stream)
+
+
+def dr_host_copy(dst_host, src_host, n_bytes, threads=0):
+    return lib().dr_host_copy(dst_host, src_host, n_bytes, threads)
 
 
 def dr_shard_range(flat_elems, world, rank):
@@ -392,6 +427,22 @@ class Plan:
                         dst.numel() * dst.element_size(), self._stream(stream))
         if rc:
             raise DrError(rc, "dr_reshard")
+
+    def ranges(self):
+        rc, out = dr_plan_ranges(self.handle)
+        if rc:
+            raise DrError(rc, "dr_plan_ranges")
+        return out
+
+    def reshard_push(self, src, dsts, stream=None):
+        """Repack src and store the result into every arena of dsts (CUDA tensors, or raw device pointers with
+        the plan's dst_bytes behind them)."""
+        ptrs = [d.data_ptr() if hasattr(d, "data_ptr") else int(d) for d in dsts]
+        nbytes = min([d.numel() * d.element_size() for d in dsts if hasattr(d, "numel")] or [self.info.dst_bytes])
+        rc = dr_reshard_push(self.handle, src.data_ptr(), src.numel() * src.element_size(), ptrs, nbytes,
+                             self._stream(stream))
+        if rc:
+            raise DrError(rc, "dr_reshard_push")
 
     def reshard_groups(self, first, count, src, dst, stream=None):
         """Repack only groups [first, first + count) (0: embed, l + 1: layer l, last: final norm and lm_head)."""

@@ -9,7 +9,7 @@ _DIR = os.path.dirname(os.path.abspath(__file__))
 _ROOT = os.path.dirname(_DIR)
 CSRC = os.path.join(_DIR, "csrc")
 LIB = os.path.join(_DIR, "libdynaresize.so")
-SOURCES = ["api.cu", "planner.cpp", "copy_pool.cpp", "reshard.cu", "staging.cu", "stream.cu", "quant.cu", "controller.cpp"]
+SOURCES = ["api.cu", "planner.cpp", "copy_pool.cpp", "reshard.cu", "staging.cu", "stream.cu", "quant.cu", "probe.cu", "controller.cpp"]
 NVCC_FLAGS = ["-gencode", "arch=compute_100a,code=sm_100a", "-lineinfo", "-O3", "-std=c++17",
               "-Xcompiler", "-fPIC,-Wall,-pthread"]
 

@@ -335,6 +335,45 @@ int dr_reshard_groups(const dr_plan* plan, uint32_t first, uint32_t count, const
     return launch_reshard(plan, false, src_dev, dst_dev, nullptr, cuda_stream, lo, hi);
 }
 
+int dr_plan_ranges(const dr_plan* plan, uint64_t max_ranges, dr_range* out, uint64_t* n_ranges)
+{
+    if (!plan || !n_ranges || (max_ranges && !out)) {
+        set_error("NULL argument");
+        return DR_ERR_INVALID;
+    }
+    if (plan->fp8) {
+        set_error("fp8 plans have no exchange ranges: a block is scaled from all of its elements");
+        return DR_ERR_UNSUPPORTED;
+    }
+    try {
+        std::vector<dr_range> v = plan_ranges(plan);
+        *n_ranges = v.size();
+        for (uint64_t i = 0; i < v.size() && i < max_ranges; ++i) out[i] = v[i];
+    } catch (const std::bad_alloc&) {
+        return DR_ERR_NOMEM;
+    }
+    return DR_OK;
+}
+
+int dr_reshard_push(const dr_plan* plan, const void* src_dev, uint64_t src_bytes, void* const* dst_dev, uint32_t n_dst,
+                    uint64_t dst_bytes, void* cuda_stream)
+{
+    if (!dst_dev || n_dst == 0 || n_dst > DR_MAX_PUSH_DST) {
+        set_error("n_dst must be 1..%u and dst_dev non-NULL", DR_MAX_PUSH_DST);
+        return DR_ERR_INVALID;
+    }
+    for (uint32_t i = 0; i < n_dst; ++i) {
+        int rc = check_call(plan, src_dev, src_bytes, plan ? plan->info.src_bytes : 0, dst_dev[i], dst_bytes,
+                            plan ? plan->info.dst_bytes : 0);
+        if (rc) return rc;
+    }
+    if (plan->fp8) {
+        set_error("fp8 plans cannot be pushed shard by shard");
+        return DR_ERR_UNSUPPORTED;
+    }
+    return launch_push(plan, src_dev, dst_dev, n_dst, cuda_stream);
+}
+
 int dr_reshard_inverse(const dr_plan* plan, const void* rollout_dev, uint64_t rollout_bytes, void* flat_dev,
                        uint64_t flat_bytes, void* cuda_stream)
 {

@@ -119,4 +119,57 @@ void CopyPool::loop(unsigned i)
     }
 }
 
+Drainer::Drainer(CopyPool* pool) : pool_(pool), th_([this] { loop(); }) {}
+
+Drainer::~Drainer()
+{
+    {
+        std::lock_guard<std::mutex> l(mu_);
+        stop_ = true;
+    }
+    work_.notify_all();
+    th_.join();
+}
+
+void Drainer::submit(const Part* parts, unsigned n_parts)
+{
+    {
+        std::lock_guard<std::mutex> l(mu_);
+        q_.emplace_back(parts, parts + n_parts);
+    }
+    work_.notify_one();
+}
+
+uint64_t Drainer::completed()
+{
+    std::lock_guard<std::mutex> l(mu_);
+    return completed_;
+}
+
+bool Drainer::wait_completed(uint64_t count, std::chrono::steady_clock::time_point deadline)
+{
+    std::unique_lock<std::mutex> l(mu_);
+    return done_.wait_until(l, deadline, [&] { return completed_ >= count; });
+}
+
+void Drainer::loop()
+{
+    for (;;) {
+        std::vector<Part> job;
+        {
+            std::unique_lock<std::mutex> l(mu_);
+            work_.wait(l, [&] { return stop_ || !q_.empty(); });
+            if (q_.empty()) return;  // stop requested and nothing left to copy
+            job.swap(q_.front());
+            q_.pop_front();
+        }
+        for (const Part& p : job) pool_->copy(p.dst, p.src, p.n);
+        {
+            std::lock_guard<std::mutex> l(mu_);
+            ++completed_;
+        }
+        done_.notify_all();
+    }
+}
+
 }  // namespace dr

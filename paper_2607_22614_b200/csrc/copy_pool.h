@@ -1,7 +1,9 @@
 // Host-side parallel copy between the pinned staging ring and a pageable host arena.
 #pragma once
+#include <chrono>
 #include <condition_variable>
 #include <cstdint>
+#include <deque>
 #include <mutex>
 #include <thread>
 #include <vector>
@@ -30,6 +32,34 @@ private:
     char* dst_ = nullptr;
     const char* src_ = nullptr;
     uint64_t len_ = 0;
+};
+
+// Copies finished chunks from the pinned ring to a pageable arena on a thread of its own (which in turn
+// drives the CopyPool), so that the pump thread is free to issue the next device-to-host copies while a
+// chunk is still being copied out.  Chunks are copied in submission order.
+class Drainer {
+public:
+    struct Part {
+        char* dst;
+        const char* src;
+        uint64_t n;
+    };
+    explicit Drainer(CopyPool* pool);
+    ~Drainer();
+    void submit(const Part* parts, unsigned n_parts);  // one chunk: up to one part per state buffer it touches
+    uint64_t completed();                               // chunks copied out since construction
+    // Blocks until `count` chunks have been copied out, or the deadline passes (returns false).
+    bool wait_completed(uint64_t count, std::chrono::steady_clock::time_point deadline);
+
+private:
+    void loop();
+    CopyPool* pool_;
+    std::thread th_;
+    std::mutex mu_;
+    std::condition_variable work_, done_;
+    std::deque<std::vector<Part>> q_;
+    uint64_t completed_ = 0;
+    bool stop_ = false;
 };
 
 }  // namespace dr

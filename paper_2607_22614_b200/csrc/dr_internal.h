@@ -150,6 +150,9 @@ int compile_plan(dr_plan* p);  // planner.cpp: fills tensors, segs, dev_segs, in
 // Tiles [tile_lo, min(tile_hi, all)) of the plan.
 int launch_reshard(const dr_plan* p, bool inverse, const void* flat, void* arena_or_flat_out, const void* arena_in,
                    void* stream, uint64_t tile_lo = 0, uint64_t tile_hi = ~0ull);
+// Forward repack into several arenas at once (the fused exchange).
+int launch_push(const dr_plan* p, const void* flat, void* const* arenas, uint32_t n_dst, void* stream);
+std::vector<dr_range> plan_ranges(const dr_plan* p);  // planner.cpp: coalesced arena byte ranges the plan writes
 int choose_grid(int device, uint32_t elem_size);  // resident CTAs of the reshard kernel on the whole GPU
 int launch_quant(const dr_plan* p, const void* flat, void* arena, void* stream);
 void ring_destroy(Ring* r);

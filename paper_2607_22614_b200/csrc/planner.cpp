@@ -307,6 +307,28 @@ std::vector<HostSeg> window_segments(const std::vector<HostSeg>& segs, uint64_t 
     return v;
 }
 
+// Arena byte ranges the plan writes, ascending, touching ranges merged.
+std::vector<dr_range> plan_ranges(const dr_plan* p)
+{
+    const uint64_t es = p->elem_size;
+    std::vector<dr_range> v;
+    for (const HostSeg& g : p->segs) {
+        if (g.rows == 1 || g.dst_stride == g.row_len) {  // rows are adjacent in the arena: one range
+            v.push_back(dr_range{g.dst_off, g.rows * g.row_len * es});
+        } else {
+            for (uint64_t i = 0; i < g.rows; ++i) v.push_back(dr_range{g.dst_off + i * g.dst_stride * es, g.row_len * es});
+        }
+    }
+    std::sort(v.begin(), v.end(), [](const dr_range& a, const dr_range& b) { return a.off < b.off; });
+    std::vector<dr_range> out;
+    for (const dr_range& r : v) {
+        if (r.bytes == 0) continue;
+        if (!out.empty() && out.back().off + out.back().bytes == r.off) out.back().bytes += r.bytes;
+        else out.push_back(r);
+    }
+    return out;
+}
+
 int compile_plan(dr_plan* p)
 {
     const dr_model_spec& s = p->spec;

@@ -1,6 +1,6 @@
 // fp32 -> fp8 e4m3 with one fp32 scale per 128 x 128 block of the rollout tensor (sm_100a).
 //
-// One CTA per block: 512 threads hold the block's 16 384 values in registers (four 256-bit loads in
+// One CTA per block: 256 threads hold the block's 16 384 values in registers (eight 256-bit loads in
 // flight per thread, three CTAs per SM, each row of the block one contiguous 512 B request), reduce |x| to the block
 // maximum with shuffles and one shared-memory step, then
 // divide by the block's scale, convert two values per cvt.rn.satfinite.e4m3x2.f32 and store
@@ -12,7 +12,8 @@
 // wherever that provably gives the same code: t and the true quotient differ by at most 2 ulp, so they can
 // round to different e4m3 codes only if t lies within a few ulp of a midpoint between two codes (its 20 dropped
 // mantissa bits within 4 of 0x80000) or below 2^-6, where the e4m3 grid is no longer 3 mantissa bits wide.
-// Those elements (about one in 10^4 for weight-like data) take the exact division.
+// A thread's eight values take the exact division together when any of them is in doubt (about one group in
+// 10^3 for weight-like data).
 #include <cuda_runtime.h>
 
 #include "dr_internal.h"
@@ -21,7 +22,7 @@ namespace dr {
 namespace {
 
 #ifndef DR_Q_THREADS
-#define DR_Q_THREADS 512
+#define DR_Q_THREADS 256
 #endif
 #ifndef DR_Q_MIN_BLOCKS
 #define DR_Q_MIN_BLOCKS 3
@@ -57,14 +58,49 @@ __device__ __forceinline__ uint32_t cvt_e4m3x2(float lo, float hi)
     asm("cvt.rn.satfinite.e4m3x2.f32 %0, %1, %2;" : "=h"(d) : "f"(hi), "f"(lo));
     return d;
 }
-// x / scale as far as the e4m3 code is concerned: the product with the reciprocal, or the correctly rounded
-// division where the product could round to a different code (see the header of this file).
-__device__ __forceinline__ float quotient(float x, float scale, float recip, float exact_below)
+// x[k] / scale for a group of one thread's values, as far as the e4m3 codes are concerned: the products with the
+// reciprocal, unless one of them could round to a different code than the true quotient (see the header of
+// this file), in which case the whole group is divided exactly.  The midpoint test is one multiply-add and one
+// compare: shifting the 20 dropped mantissa bits to the top and subtracting (0x80000 - 4) << 12 leaves a
+// value <= 8 << 12 exactly when the bits lie within 4 of 0x80000.
+#ifndef DR_Q_GROUP
+#define DR_Q_GROUP 8  // values sharing one "in doubt" branch
+#endif
+#ifndef DR_Q_TREE
+#define DR_Q_TREE 1  // 1: reduce the group's tests with min trees (short dependency chains); 0: chained predicates
+#endif
+__device__ __forceinline__ void quotients(const float* x, float* t, float scale, float recip, float exact_below)
 {
-    float t = __fmul_rn(x, recip);
-    const uint32_t low = __float_as_uint(t) & 0xFFFFFu;
-    if (low - (0x80000u - 4u) <= 8u || fabsf(t) < exact_below) t = __fdiv_rn(x, scale);
-    return t;
+    bool near = false;
+#if DR_Q_TREE
+    uint32_t d[DR_Q_GROUP];
+    float a[DR_Q_GROUP];
+#pragma unroll
+    for (int k = 0; k < DR_Q_GROUP; ++k) {
+        t[k] = __fmul_rn(x[k], recip);
+        d[k] = __float_as_uint(t[k]) * 4096u - 0x7FFFC000u;
+        a[k] = fabsf(t[k]);
+    }
+#pragma unroll
+    for (int w = DR_Q_GROUP / 2; w >= 1; w /= 2)
+#pragma unroll
+        for (int k = 0; k < w; ++k) {
+            d[k] = min(d[k], d[k + w]);
+            a[k] = fminf(a[k], a[k + w]);  // a NaN operand is dropped: a NaN needs no exact division
+        }
+    near = (d[0] <= 0x8000u) | (a[0] < exact_below);
+#else
+#pragma unroll
+    for (int k = 0; k < DR_Q_GROUP; ++k) {
+        t[k] = __fmul_rn(x[k], recip);
+        const uint32_t d = __float_as_uint(t[k]) * 4096u - 0x7FFFC000u;
+        near |= (d <= 0x8000u) | (fabsf(t[k]) < exact_below);
+    }
+#endif
+    if (near) {
+#pragma unroll
+        for (int k = 0; k < DR_Q_GROUP; ++k) t[k] = __fdiv_rn(x[k], scale);
+    }
 }
 __global__ void __launch_bounds__(kQThreads, DR_Q_MIN_BLOCKS)
     quant_kernel(const QTensor* __restrict__ tensors, uint32_t n_tensors, const QPart* __restrict__ parts,
@@ -158,11 +194,12 @@ __global__ void __launch_bounds__(kQThreads, DR_Q_MIN_BLOCKS)
         const uint32_t row = p * kRowsPerPass + rb;
         if (row >= nrows || col >= T.cols) continue;
         uint32_t q[8];
+        float t[8];
+#pragma unroll
+        for (int k = 0; k < 8; k += DR_Q_GROUP) quotients(&v[p][k], &t[k], scale, recip, exact_below);
 #pragma unroll
         for (int k = 0; k < 8; k += 2) {
-            const float a = quotient(v[p][k], scale, recip, exact_below);
-            const float c = quotient(v[p][k + 1], scale, recip, exact_below);
-            const uint32_t two = cvt_e4m3x2(a, c);
+            const uint32_t two = cvt_e4m3x2(t[k], t[k + 1]);
             q[k] = two & 0xFF;
             q[k + 1] = two >> 8;
         }

@@ -180,13 +180,21 @@ __device__ __forceinline__ uint32_t find_segment(const DevSeg* __restrict__ segs
     return lo;
 }
 
+// Further arenas that receive every element the forward kernel produces (the fused exchange): own memory or
+// peers' memory reached by plain stores.  The kernel's `arena` argument is destination 0; these are 1..n.
+struct Peers {
+    char* a[DR_MAX_PUSH_DST - 1];
+    uint32_t n;
+};
+
 // ES: rollout element size (2 = bf16, 4 = fp32).  INV: false = flat -> arena, true = arena -> flat.
 // BLOCKED: each CTA takes one contiguous range of tiles; otherwise tiles are dealt round-robin.
-template <int ES, bool INV, bool BLOCKED>
+// PUSH: forward only; every store is repeated into peers.a[0 .. peers.n).
+template <int ES, bool INV, bool BLOCKED, bool PUSH = false>
 __global__ void __launch_bounds__(kThreads, DR_MIN_BLOCKS)
     reshard_kernel(const DevSeg* __restrict__ segs, uint32_t n_segs, const uint32_t* __restrict__ hints,
                    uint32_t hint_shift, uint64_t tile_begin, uint64_t n_tiles, char* __restrict__ flat,
-                   char* __restrict__ arena, int allow256)
+                   char* __restrict__ arena, int allow256, Peers peers = Peers{})
 {
     // this launch covers tiles [tile_begin, n_tiles)
     uint64_t tile, last, step;
@@ -244,8 +252,22 @@ __global__ void __launch_bounds__(kThreads, DR_MIN_BLOCKS)
 #pragma unroll
                 for (int j = 0; j < kUnroll; ++j) {
                     if (!ok[j]) continue;
-                    if (ES == 2) st128(abase + ao[j] * 2, narrow(v[j]));
-                    else store_flat(abase + ao[j] * 4, v[j], allow256);
+                    if (ES == 2) {
+                        const V4 o = narrow(v[j]);
+                        st128(abase + ao[j] * 2, o);
+                        if (PUSH) {  // fully unrolled: a run-time index would force the pointer array into local memory
+#pragma unroll
+                            for (uint32_t q = 0; q < DR_MAX_PUSH_DST - 1; ++q)
+                                if (q < peers.n) st128(peers.a[q] + g.dst_off + ao[j] * 2, o);
+                        }
+                    } else {
+                        store_flat(abase + ao[j] * 4, v[j], allow256);
+                        if (PUSH) {
+#pragma unroll
+                            for (uint32_t q = 0; q < DR_MAX_PUSH_DST - 1; ++q)
+                                if (q < peers.n) store_flat(peers.a[q] + g.dst_off + ao[j] * 4, v[j], allow256);
+                        }
+                    }
                 }
             } else if (ES == 2) {
                 V4 v[kUnroll];
@@ -286,6 +308,14 @@ __global__ void __launch_bounds__(kThreads, DR_MIN_BLOCKS)
                 if (!INV) {
                     uint32_t x = ld32(fp);
                     if (ES == 2) st16(ap, cvt_one(x)); else st32(ap, x);
+                    if (PUSH) {
+                        const uint64_t off = g.dst_off + (row * g.dst_stride + col) * ES;
+#pragma unroll
+                        for (uint32_t q = 0; q < DR_MAX_PUSH_DST - 1; ++q) {
+                            if (q >= peers.n) continue;
+                            if (ES == 2) st16(peers.a[q] + off, cvt_one(x)); else st32(peers.a[q] + off, x);
+                        }
+                    }
                 } else {
                     uint32_t x = ES == 2 ? (uint32_t)ld16(ap) << 16 : ld32(ap);
                     st32((char*)fp, x);
@@ -342,6 +372,43 @@ int launch_reshard(const dr_plan* p, bool inverse, const void* flat, void* arena
     cudaError_t e = cudaGetLastError();
     if (e != cudaSuccess) {
         set_error("reshard kernel launch: %s", cudaGetErrorString(e));
+        return DR_ERR_CUDA;
+    }
+    return DR_OK;
+}
+
+int launch_push(const dr_plan* p, const void* flat, void* const* arenas, uint32_t n_dst, void* stream)
+{
+    const uint64_t n = p->info.n_tiles;
+    if (n == 0) return DR_OK;
+    if (DR_GRID_MULT || DR_TILES_PER_CTA != 1) {
+        set_error("the fused exchange is built for the one-tile-per-CTA launch only");
+        return DR_ERR_UNSUPPORTED;
+    }
+    if (n > 0x7FFFFFFFull) {
+        set_error("%llu tiles exceed the largest grid", (unsigned long long)n);
+        return DR_ERR_UNSUPPORTED;
+    }
+    Peers peers{};
+    uintptr_t all = (uintptr_t)flat;
+    for (uint32_t i = 0; i < n_dst; ++i) {
+        all |= (uintptr_t)arenas[i];
+        if (i) peers.a[i - 1] = (char*)arenas[i];
+    }
+    peers.n = n_dst - 1;
+    const int allow256 = (all & 31) == 0;  // one flag for all destinations
+    dim3 grid((unsigned)n), block(kThreads);
+    cudaStream_t s = (cudaStream_t)stream;
+    const uint32_t n_segs = (uint32_t)p->dev_segs.size();
+    if (p->elem_size == 2)
+        reshard_kernel<2, false, DR_BLOCKED, true><<<grid, block, DR_OCC_SMEM, s>>>(
+            p->d_segs, n_segs, p->d_hints, p->hint_shift, 0, n, (char*)flat, (char*)arenas[0], allow256, peers);
+    else
+        reshard_kernel<4, false, DR_BLOCKED, true><<<grid, block, DR_OCC_SMEM, s>>>(
+            p->d_segs, n_segs, p->d_hints, p->hint_shift, 0, n, (char*)flat, (char*)arenas[0], allow256, peers);
+    cudaError_t e = cudaGetLastError();
+    if (e != cudaSuccess) {
+        set_error("push kernel launch: %s", cudaGetErrorString(e));
         return DR_ERR_CUDA;
     }
     return DR_OK;

@@ -8,6 +8,7 @@
 #include <chrono>
 #include <condition_variable>
 #include <cstring>
+#include <exception>
 #include <functional>
 #include <thread>
 
@@ -22,6 +23,13 @@ using Clock = std::chrono::steady_clock;
 
 double ms_since(Clock::time_point t0) { return std::chrono::duration<double, std::milli>(Clock::now() - t0).count(); }
 
+// A single core cannot keep up with the host link; beyond 16 threads the copy is bound by memory, not cores.
+unsigned default_copy_threads()
+{
+    unsigned hw = std::thread::hardware_concurrency();
+    return std::max(1u, std::min(16u, hw));
+}
+
 }  // namespace
 
 struct Ring {
@@ -32,6 +40,7 @@ struct Ring {
     std::vector<cudaEvent_t> ev_copy, ev_relay;  // one per slot
     cudaEvent_t ev_entry = nullptr;              // recorded on the caller's stream when a call begins
     std::unique_ptr<CopyPool> pool;
+    std::unique_ptr<Drainer> drainer;  // started by the first stage-out into a pageable arena
 };
 
 void ring_destroy(Ring* r)
@@ -39,6 +48,7 @@ void ring_destroy(Ring* r)
     if (!r) return;
     if (r->s_copy) cudaStreamSynchronize(r->s_copy);
     if (r->s_relay) cudaStreamSynchronize(r->s_relay);
+    r->drainer.reset();  // joins its thread; nothing is queued once a stage call has returned
     for (auto e : r->ev_copy) cudaEventDestroy(e);
     for (auto e : r->ev_relay) cudaEventDestroy(e);
     if (r->ev_entry) cudaEventDestroy(r->ev_entry);
@@ -94,8 +104,12 @@ int ensure_ring(dr_plan* p, const Geometry& g, bool need_memory)
         DR_CUDA(cudaStreamCreateWithFlags(&r->s_copy, cudaStreamNonBlocking));
         DR_CUDA(cudaStreamCreateWithFlags(&r->s_relay, cudaStreamNonBlocking));
         DR_CUDA(cudaEventCreateWithFlags(&r->ev_entry, cudaEventDisableTiming));
-        unsigned hw = std::thread::hardware_concurrency();
-        r->pool.reset(new CopyPool(std::max(1u, std::min(16u, hw))));
+        try {
+            r->pool.reset(new CopyPool(default_copy_threads()));
+        } catch (const std::exception& e) {
+            set_error("cannot start the host copy threads: %s", e.what());
+            return DR_ERR_NOMEM;
+        }
     }
     Ring* r = p->ring;
     while (r->ev_copy.size() < g.slots) {
@@ -277,6 +291,20 @@ extern "C" int dr_stage_out(dr_plan* plan, const dr_stage_desc* d, dr_stage_stat
         }
         return DR_OK;
     };
+    // A pageable arena is filled by the drainer thread: the pump hands it a chunk as soon as the chunk has
+    // arrived in its ring slot and goes on issuing copies; the slot is free again once the chunk is copied out.
+    const bool via_drainer = !d->callback && !relay && !direct;
+    if (via_drainer && !r->drainer) {
+        try {
+            r->drainer.reset(new Drainer(r->pool.get()));
+        } catch (const std::exception& e) {
+            set_error("cannot start the host copy thread: %s", e.what());
+            return DR_ERR_NOMEM;
+        }
+    }
+    const uint64_t drained0 = via_drainer ? r->drainer->completed() : 0;
+    uint64_t handed = 0;  // chunks given to the drainer by this call
+
     // wait for chunk k and hand it to the sink
     auto complete = [&](uint64_t k) -> int {
         uint64_t lo = k * g.chunk, n = std::min(lo + g.chunk, g.total) - lo;
@@ -288,20 +316,54 @@ extern "C" int dr_stage_out(dr_plan* plan, const dr_stage_desc* d, dr_stage_stat
                 set_error("chunk callback failed at chunk %llu", (unsigned long long)k);
                 return DR_ERR_SINK;
             }
-        } else if (!relay && !direct) {
+        } else if (via_drainer) {
+            Drainer::Part parts[DR_MAX_STAGE_BUFS];
+            unsigned np = 0;
             for (uint32_t b = 0; b < d->n_bufs; ++b) {  // one copy per buffer the chunk touches
                 uint64_t a = std::max(lo, g.prefix[b]), e = std::min(lo + n, g.prefix[b + 1]);
-                if (a < e) r->pool->copy((char*)d->host_arena + g.host_at[b] + (a - g.prefix[b]), slot_ptr(k) + (a - lo), e - a);
+                if (a < e)
+                    parts[np++] = Drainer::Part{(char*)d->host_arena + g.host_at[b] + (a - g.prefix[b]), slot_ptr(k) + (a - lo),
+                                                e - a};
             }
+            r->drainer->submit(parts, np);
+            ++handed;
+            return DR_OK;  // counted as done once the drainer has copied it out
         }
         st.bytes += n;
         return DR_OK;
     };
+    auto chunk_bytes_of = [&](uint64_t k) { return std::min((k + 1) * g.chunk, g.total) - k * g.chunk; };
 
-    uint64_t next_issue = st.chunks_done, next_done = st.chunks_done;
-    while (rc == DR_OK && next_done < g.n_chunks) {
-        while (rc == DR_OK && next_issue < g.n_chunks && next_issue - next_done < g.slots) rc = issue(next_issue++);
-        if (rc == DR_OK && (rc = complete(next_done)) == DR_OK) st.chunks_done = ++next_done;
+    const uint64_t first = st.chunks_done;
+    uint64_t next_issue = first, next_done = first;  // next_done: next chunk whose device-to-host copy is awaited
+    if (!via_drainer) {
+        while (rc == DR_OK && next_done < g.n_chunks) {
+            while (rc == DR_OK && next_issue < g.n_chunks && next_issue - next_done < g.slots) rc = issue(next_issue++);
+            if (rc == DR_OK && (rc = complete(next_done)) == DR_OK) st.chunks_done = ++next_done;
+        }
+    } else {
+        uint64_t out = first;  // chunks below this index rest in the arena; their slots are free
+        auto refresh = [&] {
+            const uint64_t now = first + (r->drainer->completed() - drained0);
+            for (; out < now; ++out) st.bytes += chunk_bytes_of(out);
+            st.chunks_done = out;
+        };
+        while (rc == DR_OK && out < g.n_chunks) {
+            refresh();
+            while (rc == DR_OK && next_issue < g.n_chunks && next_issue - out < g.slots) rc = issue(next_issue++);
+            if (rc != DR_OK) break;
+            if (next_done < next_issue) {
+                if ((rc = complete(next_done)) == DR_OK) ++next_done;
+            } else if (out < g.n_chunks) {  // every issued chunk is with the drainer: wait for a slot to come back
+                if (!r->drainer->wait_completed(drained0 + (out - first) + 1, Clock::now() + limit)) {
+                    set_error("staging wait timed out (host copy)");
+                    rc = DR_ERR_TIMEOUT;
+                }
+            }
+        }
+        // whatever happened, no host copy of this call may still be running when it returns
+        r->drainer->wait_completed(drained0 + handed, Clock::now() + std::chrono::seconds(60));
+        refresh();
     }
     if (rc) drain(r);
     if (d->done_event) cudaEventRecord((cudaEvent_t)d->done_event, relay ? r->s_relay : r->s_copy);
@@ -400,4 +462,20 @@ extern "C" int dr_stage_in(dr_plan* plan, const dr_stage_desc* d, dr_stage_stats
     st.link_gbs = st.elapsed_ms > 0 ? (double)st.bytes / st.elapsed_ms * 1e-6 : 0;
     if (stats) *stats = st;
     return rc;
+}
+
+extern "C" int dr_host_copy(void* dst_host, const void* src_host, uint64_t n_bytes, uint32_t threads)
+{
+    if (!dst_host || !src_host) {
+        set_error("NULL host pointer");
+        return DR_ERR_INVALID;
+    }
+    try {
+        CopyPool pool(threads ? threads : default_copy_threads());
+        pool.copy(dst_host, src_host, n_bytes);
+    } catch (const std::exception& e) {
+        set_error("cannot start the host copy threads: %s", e.what());
+        return DR_ERR_NOMEM;
+    }
+    return DR_OK;
 }
