@@ -455,25 +455,47 @@ def main():
             ok &= torch.equal(arena.view(torch.bfloat16)[lo:lo + w], master.view(torch.float32)[lo:lo + w].to(torch.bfloat16))
         line["config"]["output_equals_torch_cast_on_windows"] = bool(ok)
 
-    # context: what torch's own streaming kernels reach on this GPU in this run (the measured-peak file is a
-    # torch copy too); 1 Gi-element buffers, best of 5
-    if halves == 1 and n_src >= (1 << 30):
-        a16, b16 = master.view(torch.bfloat16)[:1 << 30], arena.view(torch.bfloat16)[:1 << 30] if info.dst_bytes >= (2 << 30) else None
-        def best(fn, nbytes):
+    # Ceilings measured in this run: trivial contiguous streaming kernels in the repack's own launch shape
+    # (dr_probe_stream), one per read : write mix.  The forward repack is a 2 : 1 stream (4 B read, 2 B written),
+    # the inverse map a 1 : 2 stream; torch's own copy and reduction are given for context.
+    TILE = 49152
+    if halves == 1 and n_src >= (1 << 28):
+        nb = min(info.src_bytes, info.dst_bytes, 8 << 30) // TILE * TILE   # bytes of the wider side
+        s0 = torch.cuda.current_stream().cuda_stream
+
+        def best(fn, nbytes, reps=7):
             ts = []
-            for _ in range(5):
+            for i in range(reps + 2):
                 e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
                 e0.record(); fn(); e1.record(); torch.cuda.synchronize()
-                ts.append(e0.elapsed_time(e1))
+                if i >= 2:
+                    ts.append(e0.elapsed_time(e1))
             return nbytes / min(ts) / 1e6
-        ctx_peaks = {"torch_read_sum_gbs": best(lambda: master.view(torch.float32)[:1 << 30].sum(), 4 << 30)}
-        if b16 is not None:
-            saved = b16.clone()
-            ctx_peaks["torch_copy_gbs"] = best(lambda: b16.copy_(a16), 4 << 30)
-            ctx_peaks["torch_fill_gbs"] = best(lambda: b16.zero_(), 2 << 30)
-            b16.copy_(saved)
-            del saved
-        line["context_ceilings"] = ctx_peaks
+
+        def probe(mode, a, b, n):
+            rc = dr.dr_probe_stream(mode, a, b, n, s0)
+            if rc:
+                raise dr.DrError(rc, "dr_probe_stream")
+
+        mp, ap = master.data_ptr(), arena.data_ptr()
+        ceil = {"bytes_wider_side": int(nb),
+                "read_gbs": best(lambda: probe(dr.binding.DR_PROBE_READ, mp, None, nb), nb),
+                "write_gbs": best(lambda: probe(dr.binding.DR_PROBE_WRITE, None, ap, nb), nb),
+                "copy_1to1_gbs": best(lambda: probe(dr.binding.DR_PROBE_COPY, mp, ap, nb), 2 * nb),
+                "narrow_2to1_gbs": best(lambda: probe(dr.binding.DR_PROBE_NARROW, mp, ap, nb), nb * 3 // 2)}
+        if flat_back is not None:
+            ceil["widen_1to2_gbs"] = best(lambda: probe(dr.binding.DR_PROBE_WIDEN, ap, flat_back.data_ptr(), nb), nb * 3 // 2)
+        w = min(n_src, 1 << 30)
+        ceil["torch_read_sum_gbs"] = best(lambda: master.view(torch.float32)[:w].sum(), 4 * w, reps=3)
+        if info.dst_bytes >= 2 * w:
+            ceil["torch_copy_gbs"] = best(lambda: arena.view(torch.bfloat16)[:w].copy_(master.view(torch.bfloat16)[:w]), 4 * w, reps=3)
+        line["context_ceilings"] = ceil
+        line["roofline"]["same_run_ceiling_for_this_mix"] = ceil["narrow_2to1_gbs"]
+        line["roofline"]["frac_of_same_run_ceiling"] = ach / ceil["narrow_2to1_gbs"]
+        if inv_ms and "widen_1to2_gbs" in ceil:
+            line["inverse"]["same_run_ceiling_for_this_mix"] = ceil["widen_1to2_gbs"]
+            line["inverse"]["frac_of_same_run_ceiling"] = line["inverse"]["gbs_avg"] / ceil["widen_1to2_gbs"]
+    line["roofline"]["frac_of_nominal_8000"] = ach / 8000.0
 
     del flat_back
     torch.cuda.empty_cache()
@@ -643,16 +665,42 @@ def staging_sections(args, cfg, plan, master, arena, seed, base, dev, world, lin
                              "all_state_resident_deferred": st_in.elapsed_ms},
     }
 
-    # re-shard across a changed training world size (Sec. 3.3): the image above is the flat state; a new rank 1 of a
-    # world of 4 stages its own range of master, m, v in (weights first), then the old cut is put back
+    # Re-shard across a changed training world size (Sec. 3.3; the paper's 6 -> 4 training GPUs): the device buffers
+    # stand for the flat state; every old rank r of 6 stages its shard of master, m, v out to its place in the flat
+    # host image (ranks one after the other on this GPU), then a new rank 1 of 4 stages its own, differently cut,
+    # range back in, weights first.  Windows of the image are scribbled on first so that the check means something.
     if len(bufs) == 3 and cfg["gathered"]:
-        rc, lo, hi, s4 = dr.dr_shard_range(n, 4, 1)
+        W_OLD, W_NEW = 6, 4
+        spots = []
+        for r in range(W_OLD):
+            rc, lo, hi, _ = dr.dr_shard_range(n, W_OLD, r)
+            for k in range(3):
+                for off in (lo, max(lo, hi - 4096)):
+                    img[k * n + off:k * n + off + 4096] = 0xDEADBEEF
+                    spots.append((k, off))
+        outs6 = []
+        for r in range(W_OLD):
+            rc, lo, hi, _ = dr.dr_shard_range(n, W_OLD, r)
+            d6 = dr.stage_desc([p + 4 * lo for p in ptrs], [4 * (hi - lo)] * 3, budget=budget, host_arena=image.data_ptr(),
+                               host_arena_bytes=image.numel(), host_offsets=[4 * (k * n + lo) for k in range(3)])
+            outs6.append(plan.stage_out(d6))
+        ok6 = all(np.array_equal(img[k * n + off:k * n + off + 4096], synth.fill_f32(seed, ids[k], base + off, 4096))
+                  for k, off in spots)
+        for b in bufs:
+            b.zero_()
+        rc, lo, hi, s4 = dr.dr_shard_range(n, W_NEW, 1)
         d4 = dr.stage_desc(ptrs, [4 * (hi - lo)] * 3, budget=budget, host_arena=image.data_ptr(),
                            host_arena_bytes=image.numel(), host_offsets=[4 * (k * n + lo) for k in range(3)], order=[0, 1, 2])
         r4 = [plan.stage_in(d4) for _ in range(2)]
         ok4 = all(synth.cuda_mismatch_f32(b[:hi - lo], seed, bid, start=base + lo) == 0 for b, bid in zip(bufs, ids))
         best = max(r4, key=lambda x: x.link_gbs)
-        out["restage"] = {"what": "new rank 1 of world 4 stages its range of master, m, v in from the flat host image",
+        out["restage"] = {"what": f"{W_OLD} old ranks stage their shards of master, m, v out to one flat host image; new rank 1 "
+                                  f"of {W_NEW} stages its range back in, weights first",
+                          "stage_out_bytes_per_old_rank": int(outs6[1].bytes),
+                          "stage_out_gbs_per_old_rank": [x.link_gbs for x in outs6],
+                          "stage_out_frac_of_link": max(x.link_gbs for x in outs6) / link_d2h,
+                          "stage_out_ms_all_old_ranks": sum(x.elapsed_ms for x in outs6),
+                          "image_matches_generator": bool(ok6),
                           "bytes": int(best.bytes), "stage_in_gbs": best.link_gbs, "frac_of_link": best.link_gbs / link_h2d,
                           "weights_resident_ms": best.ready_ms[0], "all_state_resident_ms": best.elapsed_ms,
                           "matches_generator": bool(ok4)}
@@ -662,25 +710,89 @@ def staging_sections(args, cfg, plan, master, arena, seed, base, dev, world, lin
     if mem_available_bytes() > 4 * n * 1.5:
         pageable = torch.empty(4 * n, dtype=torch.uint8)
         pageable.fill_(0)  # commit the pages before timing
-        r_out = [plan.stage_out(desc(ptrs[:1], pageable)) for _ in range(2)]
         w = min(n, 1 << 20)
-        ok = bool(np.array_equal(pageable.numpy().view(np.uint32)[:w], img[:w]))
-        bufs[0].zero_()
-        r_in = [plan.stage_in(desc(ptrs[:1], pageable, order=[0])) for _ in range(2)]
-        ok &= synth.cuda_mismatch_f32(bufs[0], seed, ids[0], start=base) == 0
-        small = dr.stage_desc(ptrs[:1], sizes[:1], budget=256 << 20, chunk=64 << 20, host_arena=pageable.data_ptr(),
-                              host_arena_bytes=pageable.numel())
-        s_out = max(plan.stage_out(small).link_gbs for _ in range(2))
-        s_in = max(plan.stage_in(small).link_gbs for _ in range(2))
-        ok &= synth.cuda_mismatch_f32(bufs[0], seed, ids[0], start=base) == 0
+
+        def ring(budget_b, chunk_b):
+            dd = dr.stage_desc(ptrs[:1], sizes[:1], budget=budget_b, chunk=chunk_b, host_arena=pageable.data_ptr(),
+                               host_arena_bytes=pageable.numel())
+            ro = [plan.stage_out(dd) for _ in range(2)]
+            good = bool(np.array_equal(pageable.numpy().view(np.uint32)[:w], img[:w]))
+            bufs[0].zero_()
+            ri = [plan.stage_in(dd) for _ in range(2)]
+            good &= synth.cuda_mismatch_f32(bufs[0], seed, ids[0], start=base) == 0
+            o, i = max(x.link_gbs for x in ro), max(x.link_gbs for x in ri)
+            return {"budget_bytes": int(budget_b), "chunk_bytes": int(chunk_b), "slots": int(budget_b // chunk_b),
+                    "pinned_high_water_bytes": int(ro[0].pinned_high_water_bytes), "stage_out_gbs": o, "stage_in_gbs": i,
+                    "stage_out_frac_of_link": o / link_d2h, "stage_in_frac_of_link": i / link_h2d, "bytes_match": good}
+
+        eight = ring(budget, budget // 8 // 4096 * 4096)          # the workload's budget as eight slots
+        two = ring(budget, budget // 2 // 4096 * 4096)            # ... and as two
+        small = ring(256 << 20, 16 << 20) if 4 * n >= (1 << 30) else None
+        # CPU baseline of this path: the engine's multi-threaded host copy on its own, and the same copy while the
+        # link moves data in the same direction beside it (what the ring path has to share the host's memory with)
+        hb = min(4 * n, GiB)
+        p1 = torch.empty(hb, dtype=torch.uint8, pin_memory=True)
+        p2 = torch.empty(hb, dtype=torch.uint8, pin_memory=True)
+        p1.fill_(1)
+        scratch = torch.empty(hb, dtype=torch.uint8, device=dev)
+        pg = pageable[:hb]
+
+        def host_copy(dst, src, reps=3):
+            best = 1e30
+            for _ in range(reps):
+                t0 = time.perf_counter()
+                rc = dr.dr_host_copy(dst.data_ptr(), src.data_ptr(), hb, 0)
+                best = min(best, time.perf_counter() - t0)
+                if rc:
+                    raise dr.DrError(rc, "dr_host_copy")
+            return hb / best / 1e9
+
+        def beside_dma(dst, src, d2h):
+            stop, copied = threading.Event(), [0, 0.0]
+
+            def worker():
+                t0 = time.perf_counter()
+                while not stop.is_set():
+                    dr.dr_host_copy(dst.data_ptr(), src.data_ptr(), hb, 0)
+                    copied[0] += hb
+                copied[1] = time.perf_counter() - t0
+
+            th = threading.Thread(target=worker)
+            e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            th.start()
+            time.sleep(0.05)
+            e0.record()
+            reps = 24
+            for _ in range(reps):
+                if d2h:
+                    p2.copy_(scratch, non_blocking=True)
+                else:
+                    scratch.copy_(p2, non_blocking=True)
+            e1.record()
+            torch.cuda.synchronize()
+            stop.set()
+            th.join()
+            return copied[0] / copied[1] / 1e9, reps * hb / e0.elapsed_time(e1) / 1e6
+
+        alone_out, alone_in = host_copy(pg, p1), host_copy(p1, pg)
+        c_out, dma_out = beside_dma(pg, p1, True)
+        c_in, dma_in = beside_dma(p1, pg, False)
+        del p1, p2, scratch
         out["staging"]["through_ring_to_pageable"] = {
-            "with_256MiB_budget_64MiB_chunks": {"stage_out_gbs": s_out, "stage_in_gbs": s_in,
-                                                "stage_out_frac_of_link": s_out / link_d2h,
-                                                "stage_in_frac_of_link": s_in / link_h2d},
-            "bytes": int(4 * n), "pinned_high_water_bytes": int(r_out[0].pinned_high_water_bytes),
-            "stage_out_gbs": max(x.link_gbs for x in r_out), "stage_in_gbs": max(x.link_gbs for x in r_in),
-            "stage_out_frac_of_link": max(x.link_gbs for x in r_out) / link_d2h,
-            "stage_in_frac_of_link": max(x.link_gbs for x in r_in) / link_h2d, "bytes_match": ok}
+            "bytes": int(4 * n), "eight_slots": eight, "two_slots": two, "with_256MiB_budget_16MiB_chunks": small,
+            "stage_out_gbs": max(eight["stage_out_gbs"], two["stage_out_gbs"]),
+            "stage_in_gbs": max(eight["stage_in_gbs"], two["stage_in_gbs"]),
+            "stage_out_frac_of_link": max(eight["stage_out_frac_of_link"], two["stage_out_frac_of_link"]),
+            "stage_in_frac_of_link": max(eight["stage_in_frac_of_link"], two["stage_in_frac_of_link"]),
+            "bytes_match": bool(eight["bytes_match"] and two["bytes_match"]),
+            "cpu_baseline_host_copy": {
+                "what": "dr_host_copy, the engine's multi-threaded copy (non-temporal stores), 1 GiB, this box's host cores",
+                "threads": min(16, os.cpu_count() or 1),
+                "pinned_to_pageable_alone_gbs": alone_out, "pageable_to_pinned_alone_gbs": alone_in,
+                "pinned_to_pageable_beside_d2h_gbs": c_out, "d2h_beside_host_copy_gbs": dma_out,
+                "pageable_to_pinned_beside_h2d_gbs": c_in, "h2d_beside_host_copy_gbs": dma_in,
+                "note": "every byte staged through the ring crosses host memory three times (link write, copy read, "
+                        "copy write); the beside-the-link rates are what the host sustains for that mix"}}
         del pageable
     for b in bufs[1:]:
         del b

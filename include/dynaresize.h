@@ -116,13 +116,18 @@ typedef struct dr_dst_layout {
  * dtype DR_FP8_E4M3_B128 (a rollout-engine layout, no counterpart in the paper): the linear weights
  * (qkv, o, gate_up, down, w13, w2) are written as fp8 e4m3 with one fp32 scale per 128 x 128 block of
  * the rollout tensor; embed, lm_head, router and the norms stay bf16.  Per block: amax = max |x| (NaNs
- * skipped), stored scale = amax / 448 in fp32, q = e4m3(x * (448 / amax)) with the reciprocal and the
- * product each rounded once in fp32 (an all-zero block takes scale 1), round to nearest even,
- * magnitudes above 448 saturating to 448, NaN -> 0x7F.  A quantised tensor
- * occupies rows * cols bytes at arena_off, then its scales, row-major, at scale_off (the next multiple
- * of arena_align_bytes).  Needs the whole flat buffer (gathered = 1 or world = 1): a block cannot be
- * scaled from part of its elements.  dr_reshard only; the inverse, static and streamed calls return
- * DR_ERR_UNSUPPORTED for such a plan.
+ * skipped), stored scale = amax / 448 in fp32, held inside [2^-126, FLT_MAX] (so a block whose
+ * amax / 448 underflows, the all-zero block included, keeps zeros as zeros and yields no NaN, and a block
+ * holding an infinity keeps a finite scale); code = e4m3(x / scale): one fp32 division rounded to
+ * nearest, then round to nearest even onto the e4m3 grid, magnitudes above 448 saturating to 448,
+ * NaN -> 0x7F.  A consumer dequantises with code * scale.  A quantised tensor occupies rows * cols
+ * bytes at arena_off, then its scales, row-major, at scale_off (the next multiple of
+ * arena_align_bytes).  Needs the whole flat buffer (gathered = 1 or world = 1): a block cannot be
+ * scaled from part of its elements.
+ * Supported on such a plan: dr_reshard, dr_reshard_groups, and dr_reshard_inverse, which writes
+ * value(code) * scale (one fp32 multiplication; any NaN becomes 0x7FC00000) to the flat positions of
+ * the quantised tensors and widens the bf16 ones.  dr_reshard_static, dr_reshard_stream,
+ * dr_reshard_push, dr_plan_ranges and dr_plan_window_host return DR_ERR_UNSUPPORTED.
  */
 typedef struct dr_plan dr_plan;
 
@@ -213,8 +218,9 @@ int dr_reshard(const dr_plan* plan, const void* src_dev, uint64_t src_bytes, voi
  * dr_reshard_inverse -- Rollout -> Training (Sec. 3.3: bringing back the state the new topology
  * needs)..  Scatters the rollout arena back to the flat positions it was taken from, widening
  * bf16 to fp32 exactly (bits << 16).  Only positions covered by this TP rank (and, for gathered = 0,
- * lying in this shard) are written; padding and everything else keep their bytes.  Asynchronous on
- * cuda_stream; same errors as dr_reshard.
+ * lying in this shard) are written; padding and everything else keep their bytes.  On an fp8 plan the
+ * quantised tensors come back as value(code) * scale.  Asynchronous on cuda_stream; same errors as
+ * dr_reshard.
  */
 int dr_reshard_inverse(const dr_plan* plan, const void* rollout_dev, uint64_t rollout_bytes, void* flat_dev,
                        uint64_t flat_bytes, void* cuda_stream);
@@ -234,7 +240,8 @@ int dr_plan_group(const dr_plan* plan, uint32_t g, dr_group_desc* out); /* DR_ER
  * other GPUs) can overlap the repack of the next ones; this is the switch split into the fine-grained,
  * overlappable operations Sec. 3.1 and 3.3 argue for.  Elements of other groups keep their bytes;
  * running every group once, in any order, gives exactly dr_reshard's result.  Same arguments and errors
- * as dr_reshard, plus DR_ERR_INVALID for a range outside the groups and DR_ERR_UNSUPPORTED for fp8 plans.
+ * as dr_reshard, plus DR_ERR_INVALID for a range outside the groups.  fp8 plans: a group's quantised tensors
+ * are block-scaled by the same call.
  */
 int dr_reshard_groups(const dr_plan* plan, uint32_t first, uint32_t count, const void* src_dev, uint64_t src_bytes,
                       void* dst_dev, uint64_t dst_bytes, void* cuda_stream);
@@ -317,12 +324,17 @@ typedef int (*dr_chunk_fn)(void* user, uint64_t chunk_idx, uint64_t stream_off, 
  * k.  Stage-in restores the buffers in `order` (weights first); each buffer is cut into pieces of at
  * most chunk_bytes, numbered consecutively in that order.
  * At most budget_bytes of pinned ring memory are held: slots = floor(budget / chunk) >= 2.
- * Where the bytes rest (exactly one of):
- *   callback   != NULL : every chunk goes to / comes from the callback
- *   relay_dev[0] != NULL (stage-out only): every chunk is copied straight on to relay_dev[i], the
- *                        old-rank -> new-rank pipeline of Sec. 3.3, never resting on the host
- *   host_arena != NULL : arena[0, B) is the stream image; a pinned arena is copied to directly
- *                        (still chunk by chunk), a pageable one through the ring by worker threads
+ * Where the bytes rest:
+ *   callback   != NULL : every chunk goes to / comes from the callback (excludes the other two)
+ *   relay_dev[i] != NULL (stage-out only): buffer i is copied straight on to relay_dev[i] through the
+ *                        ring, the old-rank -> new-rank pipeline of Sec. 3.3, never resting on the host
+ *   host_arena != NULL : every buffer without a relay target rests in the arena (arena[0, B) is the
+ *                        stream image, or host_offset[i] with DR_STAGE_HOST_OFFSETS); a pinned arena is
+ *                        copied to directly (still chunk by chunk), a pageable one through the ring by
+ *                        worker threads
+ * One stage-out call may mix relay and arena buffers: a rank that keeps training under a new world size
+ * relays the part of its new shard it already holds and rests the remainder of its old shard on the
+ * host in the same pass.  A non-empty buffer with neither place to go is DR_ERR_INVALID.
  */
 typedef struct dr_stage_desc {
     uint32_t struct_size, n_bufs;       /* sizeof(dr_stage_desc); 1..DR_MAX_STAGE_BUFS                */

@@ -303,8 +303,8 @@ int dr_plan_group(const dr_plan* plan, uint32_t g, dr_group_desc* out)
     const Group& G = plan->groups[g];
     out->first_tensor = G.first_tensor;
     out->n_tensors = G.n_tensors;
-    out->elems = G.elems;
-    out->bytes_moved = G.elems * (4 + plan->elem_size);
+    out->elems = G.elems + G.qelems;
+    out->bytes_moved = G.elems * (4 + plan->elem_size) + G.qelems * 5 + (G.qblock_hi - G.qblock_lo) * 4;
     return DR_OK;
 }
 
@@ -314,25 +314,26 @@ int dr_reshard_groups(const dr_plan* plan, uint32_t first, uint32_t count, const
     int rc = check_call(plan, src_dev, src_bytes, plan ? plan->info.src_bytes : 0, dst_dev, dst_bytes,
                         plan ? plan->info.dst_bytes : 0);
     if (rc) return rc;
-    if (plan->fp8) {
-        set_error("fp8 plans are repacked whole");
-        return DR_ERR_UNSUPPORTED;
-    }
     if (count == 0 || first >= plan->groups.size() || count > plan->groups.size() - first) {
         set_error("group range outside the plan's %zu groups", plan->groups.size());
         return DR_ERR_INVALID;
     }
     // groups own consecutive tile ranges: the union of the non-empty ones is one range
-    uint64_t lo = ~0ull, hi = 0;
+    uint64_t lo = ~0ull, hi = 0, qlo = ~0ull, qhi = 0;
     for (uint32_t g = first; g < first + count; ++g) {
         const Group& G = plan->groups[g];
         if (G.tile_hi > G.tile_lo) {
             lo = G.tile_lo < lo ? G.tile_lo : lo;
             hi = G.tile_hi > hi ? G.tile_hi : hi;
         }
+        if (G.qblock_hi > G.qblock_lo) {  // fp8 plans: the groups' quantisation blocks, consecutive as well
+            qlo = G.qblock_lo < qlo ? G.qblock_lo : qlo;
+            qhi = G.qblock_hi > qhi ? G.qblock_hi : qhi;
+        }
     }
-    if (hi == 0) return DR_OK;  // nothing of these groups lies in this shard
-    return launch_reshard(plan, false, src_dev, dst_dev, nullptr, cuda_stream, lo, hi);
+    if (hi != 0) rc = launch_reshard(plan, false, src_dev, dst_dev, nullptr, cuda_stream, lo, hi);
+    if (rc == DR_OK && qhi != 0) rc = launch_quant(plan, src_dev, dst_dev, cuda_stream, qlo, qhi);
+    return rc;  // nothing launched when none of these groups lies in this shard
 }
 
 int dr_plan_ranges(const dr_plan* plan, uint64_t max_ranges, dr_range* out, uint64_t* n_ranges)
@@ -380,11 +381,9 @@ int dr_reshard_inverse(const dr_plan* plan, const void* rollout_dev, uint64_t ro
     int rc = check_call(plan, rollout_dev, rollout_bytes, plan ? plan->info.dst_bytes : 0, flat_dev, flat_bytes,
                         plan ? plan->info.src_bytes : 0);
     if (rc) return rc;
-    if (plan->fp8) {
-        set_error("fp8 plans have no inverse map");
-        return DR_ERR_UNSUPPORTED;
-    }
-    return launch_reshard(plan, true, nullptr, flat_dev, rollout_dev, cuda_stream);
+    rc = launch_reshard(plan, true, nullptr, flat_dev, rollout_dev, cuda_stream);
+    if (rc == DR_OK && plan->fp8) rc = launch_dequant(plan, rollout_dev, flat_dev, cuda_stream);
+    return rc;
 }
 
 int dr_shard_range(uint64_t flat_elems, uint32_t world, uint32_t rank, uint64_t* begin, uint64_t* end,

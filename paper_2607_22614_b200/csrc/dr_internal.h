@@ -70,6 +70,7 @@ struct HostSeg {
 // A group of rollout tensors that can be repacked on its own (tiles [tile_lo, tile_hi) of the plan).
 struct Group {
     uint64_t tile_lo = 0, tile_hi = 0, elems = 0;
+    uint64_t qblock_lo = 0, qblock_hi = 0, qelems = 0;  // fp8 plans: the group's quantisation blocks
     uint32_t first_tensor = 0, n_tensors = 0;
 };
 
@@ -154,7 +155,10 @@ int launch_reshard(const dr_plan* p, bool inverse, const void* flat, void* arena
 int launch_push(const dr_plan* p, const void* flat, void* const* arenas, uint32_t n_dst, void* stream);
 std::vector<dr_range> plan_ranges(const dr_plan* p);  // planner.cpp: coalesced arena byte ranges the plan writes
 int choose_grid(int device, uint32_t elem_size);  // resident CTAs of the reshard kernel on the whole GPU
-int launch_quant(const dr_plan* p, const void* flat, void* arena, void* stream);
+// Blocks [block_lo, min(block_hi, all)) of the plan's quantised tensors.
+int launch_quant(const dr_plan* p, const void* flat, void* arena, void* stream, uint64_t block_lo = 0,
+                 uint64_t block_hi = ~0ull);
+int launch_dequant(const dr_plan* p, const void* arena, void* flat, void* stream);
 void ring_destroy(Ring* r);
 void stream_destroy(Stream* s);
 int build_tables(const std::vector<HostSeg>& segs, Tables* out);

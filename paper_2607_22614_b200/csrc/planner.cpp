@@ -476,10 +476,19 @@ int compile_plan(dr_plan* p)
 
     // fp8: block prefix per quantised tensor and a block -> tensor hint table
     uint64_t qblocks = 0, qelems = 0;
-    for (QTensor& q : p->qtensors) {
-        q.block0 = qblocks;
-        qblocks += (uint64_t)((q.rows + 127) / 128) * q.nbc;
-        qelems += (uint64_t)q.rows * q.cols;
+    {
+        size_t qi = 0;  // quantised tensors appear in p->qtensors in tensor order
+        for (const Tensor& t : p->tensors) {
+            if (!t.quant || t.alias_of >= 0) continue;
+            QTensor& q = p->qtensors[qi++];
+            Group& G = p->groups[t.group];
+            q.block0 = qblocks;
+            if (G.qblock_hi == G.qblock_lo) G.qblock_lo = qblocks;
+            qblocks += (uint64_t)((q.rows + 127) / 128) * q.nbc;
+            G.qblock_hi = qblocks;
+            G.qelems += (uint64_t)q.rows * q.cols;
+            qelems += (uint64_t)q.rows * q.cols;
+        }
     }
     if (p->fp8) {
         p->qhint_shift = 0;
@@ -504,7 +513,7 @@ int compile_plan(dr_plan* p)
     I.n_tiles = tiles;
     I.elems_moved = moved + qelems;
     I.bytes_moved_fwd = moved * (4 + es) + qelems * 5 + qblocks * 4;
-    I.bytes_moved_inv = moved * (4 + es);
+    I.bytes_moved_inv = moved * (4 + es) + qelems * 5 + qblocks * 4;
     I.n_groups = p->groups.size();
     I.quant_elems = qelems;
     I.quant_blocks = qblocks;

@@ -105,13 +105,13 @@ __device__ __forceinline__ void quotients(const float* x, float* t, float scale,
 __global__ void __launch_bounds__(kQThreads, DR_Q_MIN_BLOCKS)
     quant_kernel(const QTensor* __restrict__ tensors, uint32_t n_tensors, const QPart* __restrict__ parts,
                  const uint32_t* __restrict__ hints, uint32_t hint_shift, const char* __restrict__ flat,
-                 char* __restrict__ arena, int allow256)
+                 char* __restrict__ arena, int allow256, uint64_t block_begin)
 {
     __shared__ uint64_t row_src[128];  // flat element offset of (row, first column of the tensor)
     __shared__ float warp_max[kQThreads / 32];
     __shared__ float s_scale;
 
-    const uint64_t b = blockIdx.x;
+    const uint64_t b = block_begin + blockIdx.x;
     // block -> tensor: hint plus a short walk (all threads, same addresses: broadcast loads)
     uint32_t ti = hints[b >> hint_shift];
     while (ti + 1 < n_tensors && tensors[ti + 1].block0 <= b) ++ti;
@@ -217,9 +217,125 @@ __global__ void __launch_bounds__(kQThreads, DR_Q_MIN_BLOCKS)
     }
 }
 
+
+// ---- the inverse: e4m3 codes times the block's scale, back to the flat fp32 positions ----------------------
+// Same decomposition (one CTA per 128 x 128 block, 16 threads per block row, eight values per thread and row),
+// no reduction: 1 B read + 4 B written per element.  value(code) is exact in fp16 (cvt.rn.f16x2.e4m3x2), the
+// product with the scale is one fp32 multiplication, and any NaN (a NaN code, a NaN scale, 0 * Inf) becomes the
+// quiet NaN 0x7FC00000.
+__device__ __forceinline__ void e4m3x2_to_f32(uint32_t two, float& lo, float& hi)
+{
+    uint32_t h2;
+    asm("cvt.rn.f16x2.e4m3x2 %0, %1;" : "=r"(h2) : "h"((uint16_t)two));
+    asm("cvt.f32.f16 %0, %1;" : "=f"(lo) : "h"((uint16_t)(h2 & 0xFFFF)));
+    asm("cvt.f32.f16 %0, %1;" : "=f"(hi) : "h"((uint16_t)(h2 >> 16)));
+}
+__global__ void __launch_bounds__(kQThreads)
+    dequant_kernel(const QTensor* __restrict__ tensors, uint32_t n_tensors, const QPart* __restrict__ parts,
+                   const uint32_t* __restrict__ hints, uint32_t hint_shift, const char* __restrict__ arena,
+                   char* __restrict__ flat, int allow256)
+{
+    __shared__ uint64_t row_src[128];
+    const uint64_t b = blockIdx.x;
+    uint32_t ti = hints[b >> hint_shift];
+    while (ti + 1 < n_tensors && tensors[ti + 1].block0 <= b) ++ti;
+    const QTensor T = tensors[ti];
+    const uint32_t lb = (uint32_t)(b - T.block0);
+    const uint32_t bi = lb / T.nbc, bj = lb - bi * T.nbc;
+    const uint32_t r0 = bi * 128, c0 = bj * 128;
+    const uint32_t nrows = min(128u, T.rows - r0);
+    if (threadIdx.x < 128) {
+        uint64_t off = 0;
+        const uint32_t r = r0 + threadIdx.x;
+        if (threadIdx.x < nrows) {
+            uint32_t lo = T.part0, hi = T.part0 + T.n_parts;
+            while (hi - lo > 1) {
+                uint32_t mid = lo + (hi - lo) / 2;
+                if (parts[mid].dst_row0 <= r) lo = mid; else hi = mid;
+            }
+            const QPart P = parts[lo];
+            off = P.src_off + (uint64_t)(r - P.dst_row0) * P.src_stride;
+        }
+        row_src[threadIdx.x] = off;
+    }
+    const float scale = *(const float*)(arena + T.scale_off + ((uint64_t)bi * T.nbc + bj) * 4);
+    __syncthreads();
+
+    const uint32_t cu = threadIdx.x & 15, rb = threadIdx.x >> 4;
+    const uint32_t col = c0 + cu * 8;
+    uint32_t q[kPasses][2];
+#pragma unroll
+    for (int p = 0; p < kPasses; ++p) {
+        const uint32_t row = p * kRowsPerPass + rb;
+        q[p][0] = q[p][1] = 0;
+        if (row < nrows && col < T.cols) {
+            const char* src = arena + T.payload_off + (uint64_t)(r0 + row) * T.cols + col;
+            if (T.aligned) {
+                asm volatile("ld.global.nc.L1::no_allocate.v2.b32 {%0,%1}, [%2];" : "=r"(q[p][0]), "=r"(q[p][1]) : "l"(src));
+            } else {
+#pragma unroll
+                for (int k = 0; k < 8; ++k)
+                    if (col + k < T.cols) q[p][k >> 2] |= (uint32_t)(uint8_t)src[k] << (8 * (k & 3));
+            }
+        }
+    }
+#pragma unroll
+    for (int p = 0; p < kPasses; ++p) {
+        const uint32_t row = p * kRowsPerPass + rb;
+        if (row >= nrows || col >= T.cols) continue;
+        uint32_t y[8];
+#pragma unroll
+        for (int k = 0; k < 8; k += 2) {
+            float lo, hi;
+            e4m3x2_to_f32((q[p][k >> 2] >> (8 * (k & 3))) & 0xFFFF, lo, hi);
+            lo = __fmul_rn(lo, scale);
+            hi = __fmul_rn(hi, scale);
+            y[k] = lo != lo ? 0x7FC00000u : __float_as_uint(lo);
+            y[k + 1] = hi != hi ? 0x7FC00000u : __float_as_uint(hi);
+        }
+        char* dst = flat + (row_src[row] + col) * 4;
+        if (T.aligned && allow256) {
+            asm volatile("st.global.L1::no_allocate.v8.b32 [%0], {%1,%2,%3,%4,%5,%6,%7,%8};" ::"l"(dst), "r"(y[0]), "r"(y[1]),
+                         "r"(y[2]), "r"(y[3]), "r"(y[4]), "r"(y[5]), "r"(y[6]), "r"(y[7])
+                         : "memory");
+        } else if (T.aligned) {
+            asm volatile("st.global.L1::no_allocate.v4.b32 [%0], {%1,%2,%3,%4};" ::"l"(dst), "r"(y[0]), "r"(y[1]), "r"(y[2]),
+                         "r"(y[3])
+                         : "memory");
+            asm volatile("st.global.L1::no_allocate.v4.b32 [%0], {%1,%2,%3,%4};" ::"l"(dst + 16), "r"(y[4]), "r"(y[5]),
+                         "r"(y[6]), "r"(y[7])
+                         : "memory");
+        } else {
+#pragma unroll
+            for (int k = 0; k < 8; ++k)
+                if (col + k < T.cols) *(uint32_t*)(dst + 4 * k) = y[k];
+        }
+    }
+}
+
 }  // namespace
 
-int launch_quant(const dr_plan* p, const void* flat, void* arena, void* stream)
+int launch_quant(const dr_plan* p, const void* flat, void* arena, void* stream, uint64_t block_lo, uint64_t block_hi)
+{
+    if (block_hi > p->info.quant_blocks) block_hi = p->info.quant_blocks;
+    if (block_lo >= block_hi) return DR_OK;
+    const uint64_t blocks = block_hi - block_lo;
+    if (blocks > 0x7FFFFFFFull) {
+        set_error("too many quantisation blocks");
+        return DR_ERR_UNSUPPORTED;
+    }
+    quant_kernel<<<(unsigned)blocks, kQThreads, 0, (cudaStream_t)stream>>>(
+        p->d_qtensors, (uint32_t)p->qtensors.size(), p->d_qparts, p->d_qhints, p->qhint_shift, (const char*)flat,
+        (char*)arena, (((uintptr_t)flat | (uintptr_t)arena) & 31) == 0, block_lo);
+    cudaError_t e = cudaGetLastError();
+    if (e != cudaSuccess) {
+        set_error("quant kernel launch: %s", cudaGetErrorString(e));
+        return DR_ERR_CUDA;
+    }
+    return DR_OK;
+}
+
+int launch_dequant(const dr_plan* p, const void* arena, void* flat, void* stream)
 {
     const uint64_t blocks = p->info.quant_blocks;
     if (blocks == 0) return DR_OK;
@@ -227,12 +343,12 @@ int launch_quant(const dr_plan* p, const void* flat, void* arena, void* stream)
         set_error("too many quantisation blocks");
         return DR_ERR_UNSUPPORTED;
     }
-    quant_kernel<<<(unsigned)blocks, kQThreads, 0, (cudaStream_t)stream>>>(
-        p->d_qtensors, (uint32_t)p->qtensors.size(), p->d_qparts, p->d_qhints, p->qhint_shift, (const char*)flat,
-        (char*)arena, (((uintptr_t)flat | (uintptr_t)arena) & 31) == 0);
+    dequant_kernel<<<(unsigned)blocks, kQThreads, 0, (cudaStream_t)stream>>>(
+        p->d_qtensors, (uint32_t)p->qtensors.size(), p->d_qparts, p->d_qhints, p->qhint_shift, (const char*)arena,
+        (char*)flat, (((uintptr_t)flat | (uintptr_t)arena) & 31) == 0);
     cudaError_t e = cudaGetLastError();
     if (e != cudaSuccess) {
-        set_error("quant kernel launch: %s", cudaGetErrorString(e));
+        set_error("dequant kernel launch: %s", cudaGetErrorString(e));
         return DR_ERR_CUDA;
     }
     return DR_OK;

@@ -196,9 +196,16 @@ int check_common(dr_plan* p, const dr_stage_desc* d, const Geometry& g, bool out
         set_error("host-only plan cannot stage");
         return DR_ERR_STATE;
     }
-    int n_sinks = (d->callback != nullptr) + (d->host_arena != nullptr) + (out && d->relay_dev[0] != nullptr);
-    if (n_sinks != 1) {
-        set_error("exactly one of callback, relay_dev, host_arena must be given");
+    // a callback takes everything and excludes the rest; otherwise every non-empty buffer needs a place to go:
+    // its relay target (stage-out only) or the host arena
+    bool any_relay = false, any_unplaced = false;
+    for (uint32_t i = 0; i < d->n_bufs; ++i) {
+        if (out && d->relay_dev[i]) any_relay = true;
+        else if (d->bytes[i] && !d->host_arena) any_unplaced = true;
+    }
+    if (d->callback ? (d->host_arena != nullptr || any_relay) : any_unplaced) {
+        set_error(d->callback ? "a callback excludes host_arena and relay_dev"
+                              : "a buffer has neither a relay target nor a host arena to go to");
         return DR_ERR_INVALID;
     }
     if (g.scattered && !d->host_arena) {
@@ -211,14 +218,15 @@ int check_common(dr_plan* p, const dr_stage_desc* d, const Geometry& g, bool out
         return DR_ERR_SIZE;
     }
     if (g.scattered) {
+        auto rests_on_host = [&](uint32_t i) { return d->bytes[i] && !(out && d->relay_dev[i]); };
         for (uint32_t i = 0; i < d->n_bufs; ++i) {
+            if (!rests_on_host(i)) continue;
             if (g.host_at[i] + d->bytes[i] > d->host_arena_bytes) {
                 set_error("buffer %u does not fit the host arena at its offset", i);
                 return DR_ERR_SIZE;
             }
             for (uint32_t j = 0; j < i; ++j)
-                if (d->bytes[i] && d->bytes[j] && g.host_at[i] < g.host_at[j] + d->bytes[j] &&
-                    g.host_at[j] < g.host_at[i] + d->bytes[i]) {
+                if (rests_on_host(j) && g.host_at[i] < g.host_at[j] + d->bytes[j] && g.host_at[j] < g.host_at[i] + d->bytes[i]) {
                     set_error("host regions of buffers %u and %u overlap", j, i);
                     return DR_ERR_INVALID;
                 }
@@ -248,42 +256,52 @@ extern "C" int dr_stage_out(dr_plan* plan, const dr_stage_desc* d, dr_stage_stat
     if (rc) return rc;
     if ((rc = check_common(plan, d, g, true))) return rc;
     std::lock_guard<std::mutex> lock(plan->stage_mu);
-    const bool relay = !d->callback && d->relay_dev[0];
-    const bool direct = !d->callback && !relay && is_pinned_host(d->host_arena);  // DMA straight into the arena
-    if ((rc = ensure_ring(plan, g, !direct))) return rc;
+    // Where each buffer goes: to its relay target (device -> ring slot -> device), or to the host arena (straight
+    // into a pinned arena, through the ring and the host copy threads into a pageable one); or everything to the
+    // callback.  A call may mix relay and arena buffers: a rank whose new shard is partly on this GPU already
+    // relays that part and rests the remainder on the host in one pass.
+    bool to_relay[DR_MAX_STAGE_BUFS] = {false};
+    bool any_relay = false, any_host = false;
+    for (uint32_t b = 0; b < d->n_bufs && !d->callback; ++b) {
+        to_relay[b] = d->relay_dev[b] != nullptr;
+        if (d->bytes[b] == 0) continue;
+        any_relay |= to_relay[b];
+        any_host |= !to_relay[b];
+    }
+    const bool pinned_arena = any_host && is_pinned_host(d->host_arena);  // DMA straight into the arena
+    const bool via_drainer = any_host && !pinned_arena;                   // pageable arena: drainer thread copies out
+    const bool need_ring = d->callback || any_relay || via_drainer;
+    if ((rc = ensure_ring(plan, g, need_ring))) return rc;
     Ring* r = plan->ring;
     const auto t0 = Clock::now();
     const auto limit = std::chrono::milliseconds(d->timeout_ms ? d->timeout_ms : 60000);
     dr_stage_stats st{};
     st.n_chunks = g.n_chunks;
     st.chunks_done = std::min<uint64_t>(d->first_chunk, g.n_chunks);
-    st.pinned_high_water_bytes = direct ? 0 : g.chunk * g.slots;
+    st.pinned_high_water_bytes = need_ring ? g.chunk * g.slots : 0;
     if ((rc = order_after_caller(r, d))) return rc;
 
-    // ring slot of chunk k (unused when chunks are copied straight into a pinned arena)
+    // ring slot of chunk k (unused when every chunk is copied straight into a pinned arena)
     auto slot_ptr = [&](uint64_t k) -> char* { return r->base + (k % g.slots) * g.chunk; };
     // enqueue the copies of chunk k: one per buffer it touches
     auto issue = [&](uint64_t k) -> int {
         uint64_t lo = k * g.chunk, hi = std::min(lo + g.chunk, g.total);
         uint32_t s = (uint32_t)(k % g.slots);
-        char* host = direct ? nullptr : slot_ptr(k);
+        char* host = need_ring ? slot_ptr(k) : nullptr;
         for (uint32_t b = 0; b < d->n_bufs; ++b) {
             uint64_t a = std::max(lo, g.prefix[b]), e = std::min(hi, g.prefix[b + 1]);
             if (a >= e) continue;
-            char* to = direct ? (char*)d->host_arena + g.host_at[b] + (a - g.prefix[b]) : host + (a - lo);
+            const bool straight = !d->callback && !to_relay[b] && pinned_arena;
+            char* to = straight ? (char*)d->host_arena + g.host_at[b] + (a - g.prefix[b]) : host + (a - lo);
             DR_CUDA(cudaMemcpyAsync(to, (const char*)d->dev_ptr[b] + (a - g.prefix[b]), e - a, cudaMemcpyDeviceToHost,
                                     r->s_copy));
         }
         DR_CUDA(cudaEventRecord(r->ev_copy[s], r->s_copy));
-        if (relay) {
+        if (any_relay) {
             DR_CUDA(cudaStreamWaitEvent(r->s_relay, r->ev_copy[s], 0));
             for (uint32_t b = 0; b < d->n_bufs; ++b) {
                 uint64_t a = std::max(lo, g.prefix[b]), e = std::min(hi, g.prefix[b + 1]);
-                if (a >= e) continue;
-                if (!d->relay_dev[b]) {
-                    set_error("relay_dev[%u] is NULL", b);
-                    return DR_ERR_INVALID;
-                }
+                if (a >= e || !to_relay[b]) continue;
                 DR_CUDA(cudaMemcpyAsync((char*)d->relay_dev[b] + (a - g.prefix[b]), host + (a - lo), e - a,
                                         cudaMemcpyHostToDevice, r->s_relay));
             }
@@ -293,7 +311,6 @@ extern "C" int dr_stage_out(dr_plan* plan, const dr_stage_desc* d, dr_stage_stat
     };
     // A pageable arena is filled by the drainer thread: the pump hands it a chunk as soon as the chunk has
     // arrived in its ring slot and goes on issuing copies; the slot is free again once the chunk is copied out.
-    const bool via_drainer = !d->callback && !relay && !direct;
     if (via_drainer && !r->drainer) {
         try {
             r->drainer.reset(new Drainer(r->pool.get()));
@@ -309,7 +326,8 @@ extern "C" int dr_stage_out(dr_plan* plan, const dr_stage_desc* d, dr_stage_stat
     auto complete = [&](uint64_t k) -> int {
         uint64_t lo = k * g.chunk, n = std::min(lo + g.chunk, g.total) - lo;
         uint32_t s = (uint32_t)(k % g.slots);
-        int w = wait_event(relay ? r->ev_relay[s] : r->ev_copy[s], Clock::now() + limit);
+        int w = wait_event(r->ev_copy[s], Clock::now() + limit);
+        if (w == DR_OK && any_relay) w = wait_event(r->ev_relay[s], Clock::now() + limit);
         if (w) return w;
         if (d->callback) {
             if (d->callback(d->user, k, lo, slot_ptr(k), n)) {
@@ -319,13 +337,13 @@ extern "C" int dr_stage_out(dr_plan* plan, const dr_stage_desc* d, dr_stage_stat
         } else if (via_drainer) {
             Drainer::Part parts[DR_MAX_STAGE_BUFS];
             unsigned np = 0;
-            for (uint32_t b = 0; b < d->n_bufs; ++b) {  // one copy per buffer the chunk touches
+            for (uint32_t b = 0; b < d->n_bufs; ++b) {  // one copy per arena-bound buffer the chunk touches
                 uint64_t a = std::max(lo, g.prefix[b]), e = std::min(lo + n, g.prefix[b + 1]);
-                if (a < e)
+                if (a < e && !to_relay[b])
                     parts[np++] = Drainer::Part{(char*)d->host_arena + g.host_at[b] + (a - g.prefix[b]), slot_ptr(k) + (a - lo),
                                                 e - a};
             }
-            r->drainer->submit(parts, np);
+            r->drainer->submit(parts, np);  // possibly empty (a chunk of relay bytes only): keeps the count in step
             ++handed;
             return DR_OK;  // counted as done once the drainer has copied it out
         }
@@ -366,7 +384,7 @@ extern "C" int dr_stage_out(dr_plan* plan, const dr_stage_desc* d, dr_stage_stat
         refresh();
     }
     if (rc) drain(r);
-    if (d->done_event) cudaEventRecord((cudaEvent_t)d->done_event, relay ? r->s_relay : r->s_copy);
+    if (d->done_event) cudaEventRecord((cudaEvent_t)d->done_event, any_relay ? r->s_relay : r->s_copy);
     st.elapsed_ms = ms_since(t0);
     st.link_gbs = st.elapsed_ms > 0 ? (double)st.bytes / st.elapsed_ms * 1e-6 : 0;
     if (stats) *stats = st;

@@ -94,8 +94,100 @@ def test_fp8_unsupported_calls():
     src = torch.zeros(plan.info.src_bytes // 4, dtype=torch.int32, device=dev())
     arena = torch.zeros(plan.info.dst_bytes, dtype=torch.uint8, device=dev())
     s = torch.cuda.current_stream().cuda_stream
-    assert dr.dr_reshard_inverse(plan.handle, arena.data_ptr(), plan.info.dst_bytes, src.data_ptr(), plan.info.src_bytes, s) == B.DR_ERR_UNSUPPORTED
     assert dr.dr_reshard_static(plan.handle, src.data_ptr(), plan.info.src_bytes, arena.data_ptr(), plan.info.dst_bytes, s) == B.DR_ERR_UNSUPPORTED
+    plan.close()
+
+
+INV_CASES = [(MID[2]["spec"], 2, 1, {}, 0), (MID[1]["spec"], 4, 3, dict(vocab_pad=64), 0), (dict(BRUTE[0]["spec"], ffn=12), 2, 0, {}, 0),
+             (MID[0]["spec"], 2, 0, {}, 16), (MID[2]["spec"], 4, 1, dict(moe_tp=4, moe_ep=2, moe_ep_rank=1), 0)]
+
+
+@pytest.mark.parametrize("spec,T,t,opts,misalign", INV_CASES, ids=[f"i{i}" for i in range(len(INV_CASES))])
+def test_fp8_inverse_matches_oracle(spec, T, t, opts, misalign):
+    """Rollout -> Training from an fp8 arena: codes times block scales (one fp32 multiplication) and widened bf16
+    tensors at their flat positions, every other word untouched.  The arena holds every code (NaN codes too)
+    and scales over a wide range, including a NaN, an infinity and a zero scale."""
+    om = oracle.Model(spec, tp=T, tp_rank=t, **opts)
+    total, lay = om.fp8_layout()
+    rng = np.random.default_rng(17)
+    arena = rng.integers(0, 256, size=total, dtype=np.uint64).astype(np.uint8)
+    k = 0
+    for d, (qz, off, soff) in zip(om.dst_tensors(), lay):
+        if qz and d.alias_of < 0:
+            nb = (-(-d.rows // 128)) * (-(-d.cols // 128))
+            sc = np.exp(rng.uniform(-40, 20, nb)).astype(np.float32)
+            for special in (np.nan, np.inf, 0.0, 2.0 ** -140):
+                sc[k % nb] = special
+                k += 7
+            arena[soff:soff + 4 * nb] = sc.view(np.uint8)
+    want = np.full(om.flat_elems, 0xDEADBEEF, dtype=np.uint32)
+    om.inverse_fp8(arena, want)
+    plan = dr.Plan(spec, tp=T, tp_rank=t, dtype=dr.DR_FP8_E4M3_B128, **opts)
+    assert plan.info.dst_bytes == total and plan.info.src_bytes == 4 * om.flat_elems
+    pad = misalign // 4
+    f_buf = torch.full((om.flat_elems + pad + 64,), 0xDEADBEEF - (1 << 32), dtype=torch.int32, device=dev())
+    flat = f_buf[pad:pad + om.flat_elems]
+    a_buf = torch.zeros(total + misalign, dtype=torch.uint8, device=dev())
+    a_dev = a_buf[misalign:]
+    a_dev.copy_(torch.from_numpy(arena))
+    plan.reshard_inverse(a_dev, flat)
+    torch.cuda.synchronize()
+    assert first_diff(flat.cpu().numpy().view(np.uint32), want) is None
+    assert (f_buf[:pad] == 0xDEADBEEF - (1 << 32)).all() and (f_buf[pad + om.flat_elems:] == 0xDEADBEEF - (1 << 32)).all()
+    plan.close()
+
+
+def test_fp8_forward_then_inverse_is_within_half_a_code_step_of_the_weights():
+    """Dequantised weights: |code * scale - x| <= |x| / 16 (half an e4m3 step) or half a subnormal step."""
+    spec = MID[0]["spec"]
+    om = oracle.Model(spec)
+    src = synth.fill_f32(5, synth.BUF_MASTER, 0, om.flat_elems)
+    plan = dr.Plan(spec, dtype=dr.DR_FP8_E4M3_B128)
+    arena = torch.zeros(plan.info.dst_bytes, dtype=torch.uint8, device=dev())
+    back = torch.zeros(om.flat_elems, dtype=torch.float32, device=dev())
+    plan.reshard(to_dev_u32(src), arena)
+    plan.reshard_inverse(arena, back)
+    torch.cuda.synchronize()
+    x, y = src.view(np.float32).astype(np.float64), back.cpu().numpy().astype(np.float64)
+    lin = np.zeros(om.flat_elems, dtype=bool)
+    for s_ in om.src_tensors():
+        if s_.name.split(".")[-1] in ("q", "k", "v", "o", "gate", "up", "down"):
+            lin[s_.flat_off:s_.flat_off + s_.rows * s_.cols] = True
+    amax = np.abs(x[lin]).max()
+    assert (np.abs(y[lin] - x[lin]) <= np.maximum(np.abs(x[lin]) / 16, amax / 448 * 2.0 ** -10) * (1 + 1e-6)).all()
+    assert (np.abs(y[~lin] - x[~lin]) <= np.abs(x[~lin]) * 2.0 ** -8).all()     # bf16 tensors: half a bf16 step
+    plan.close()
+
+
+def test_fp8_groups_give_the_whole_plan_result():
+    spec = MID[2]["spec"]
+    om = oracle.Model(spec, tp=2, tp_rank=1)
+    total, _ = om.fp8_layout()
+    src = make_source(om.flat_elems, 19)
+    want = np.full(total, SENT8, dtype=np.uint8)
+    om.forward_fp8(src, want)
+    plan = dr.Plan(spec, tp=2, tp_rank=1, dtype=dr.DR_FP8_E4M3_B128)
+    s_dev = to_dev_u32(src)
+    arena = torch.full((total,), SENT8, dtype=torch.uint8, device=dev())
+    n_groups = plan.info.n_groups
+    moved = 0
+    for g in reversed(range(n_groups)):            # any order
+        plan.reshard_groups(g, 1, s_dev, arena)
+        rc, gd = dr.dr_plan_group(plan.handle, g)
+        moved += gd.bytes_moved
+    torch.cuda.synchronize()
+    assert first_diff(arena.cpu().numpy(), want) is None and moved == plan.info.bytes_moved_fwd
+    # one layer alone writes only that layer's tensors
+    arena.fill_(SENT8)
+    plan.reshard_groups(1, 1, s_dev, arena)
+    torch.cuda.synchronize()
+    got = arena.cpu().numpy()
+    tens = plan.tensors()
+    rc, gd = dr.dr_plan_group(plan.handle, 1)
+    lo = tens[gd.first_tensor].arena_off
+    hi = tens[gd.first_tensor + gd.n_tensors].arena_off
+    assert (got[:lo] == SENT8).all() and (got[hi:] == SENT8).all()
+    assert first_diff(got[lo:hi], want[lo:hi]) is None
     plan.close()
 
 

@@ -265,6 +265,65 @@ def test_part_of_the_new_shard_already_on_this_gpu_moves_through_the_relay(plan)
     assert (got[:lo - nlo] == 0).all() and (got[hi - nlo:] == 0).all()
 
 
+def _cut(begin, end, lo, hi):
+    """[begin, end) cut at the overlap [lo, hi) it contains: (a, e, inside the overlap) pieces, empty ones dropped."""
+    if hi <= lo:
+        return [(begin, end, False)] if end > begin else []
+    return [(a, e, inside) for a, e, inside in ((begin, lo, False), (lo, hi, True), (hi, end, False)) if e > a]
+
+
+@pytest.mark.parametrize("n,w_old,w_new,pinned", [(2_400_001, 6, 4, False), (2_400_001, 6, 4, True), (1_000_003, 4, 6, False)])
+def test_ranks_that_stay_relay_what_they_hold_and_rest_the_remainder_in_one_call(plan, n, w_old, w_new, pinned):
+    """A change of the training world size in which GPU i is old rank i and (if i < w_new) new rank i.  Each GPU
+    makes ONE stage-out call over master, m and v: the part of its old shard that lies inside its new range is
+    relayed into the new buffers, the rest goes to its place in the flat host image.  One stage-in call then
+    fetches what the new range still lacks.  The new shards must be the oracle's re-sharding (padding zero)."""
+    kinds = (synth.BUF_MASTER, synth.BUF_ADAM_M, synth.BUF_ADAM_V)
+    flats = [synth.fill_f32(53, k, 0, n) for k in kinds]
+    want = [oracle.restage(_split(f, w_old), n, w_new) for f in flats]
+    image = torch.zeros(3 * 4 * n, dtype=torch.uint8)
+    if pinned:
+        image = image.pin_memory()
+    new_bufs = {}
+    for i in range(w_old):                                   # every old rank, one after the other on this GPU
+        _, olo, ohi, _ = dr.dr_shard_range(n, w_old, i)
+        old = [to_dev_u32(_split(f, w_old)[i]) for f in flats]
+        ptrs, sizes, relay, offs = [], [], [], []
+        if i < w_new:
+            _, nlo, nhi, s_new = dr.dr_shard_range(n, w_new, i)
+            new_bufs[i] = [torch.zeros(s_new, dtype=torch.int32, device=dev()) for _ in kinds]
+            lo, hi = max(olo, nlo), min(ohi, nhi)
+        else:
+            lo = hi = nlo = 0
+        for k in range(3):                                   # up to three pieces of the old shard per state buffer
+            for a, e, keep in _cut(olo, ohi, lo, hi):
+                ptrs.append(old[k].data_ptr() + 4 * (a - olo))
+                sizes.append(4 * (e - a))
+                relay.append(new_bufs[i][k].data_ptr() + 4 * (a - nlo) if keep else None)
+                offs.append(4 * (k * n + a))
+        assert len(ptrs) <= dr.DR_MAX_STAGE_BUFS
+        d = dr.stage_desc(ptrs, sizes, budget=1 * MiB, chunk=128 * 1024, host_arena=image.data_ptr(),
+                          host_arena_bytes=image.numel(), host_offsets=offs, relay_dev=relay)
+        st = plan.stage_out(d)
+        assert st.bytes == 12 * (ohi - olo) and st.chunks_done == st.n_chunks
+    for i in range(w_new):                                   # each new rank fetches what it does not hold yet
+        _, olo, ohi, _ = dr.dr_shard_range(n, w_old, i)
+        _, nlo, nhi, s_new = dr.dr_shard_range(n, w_new, i)
+        lo, hi = max(olo, nlo), min(ohi, nhi)
+        ptrs, sizes, offs = [], [], []
+        for k in range(3):
+            for a, e, held in _cut(nlo, nhi, lo, hi):
+                if not held:
+                    ptrs.append(new_bufs[i][k].data_ptr() + 4 * (a - nlo))
+                    sizes.append(4 * (e - a))
+                    offs.append(4 * (k * n + a))
+        if ptrs:
+            plan.stage_in(dr.stage_desc(ptrs, sizes, budget=1 * MiB, chunk=128 * 1024, host_arena=image.data_ptr(),
+                                        host_arena_bytes=image.numel(), host_offsets=offs))
+        for k in range(3):
+            assert np.array_equal(new_bufs[i][k].cpu().numpy().view(np.uint32), want[k][i]), (i, k)
+
+
 def test_host_offset_errors(plan):
     t = torch.zeros(2048, dtype=torch.int32, device=dev())
     host = np.zeros(16384, dtype=np.uint8)
