@@ -266,7 +266,7 @@ def run_all(args):
     """The per-workload table: each workload in a process of its own (device memory is returned in between)."""
     for i in range(5):
         cmd = [sys.executable, os.path.abspath(__file__), "--cfg", str(i), "--steps", str(args.steps), "--warmup",
-               str(args.warmup), "--no-cpu"] + (["--no-staging"] if args.no_staging or i == 4 else [])
+               str(args.warmup), "--no-cpu", "--no-others"] + (["--no-staging"] if args.no_staging or i == 4 else [])
         r = subprocess.run(cmd, capture_output=True, text=True)
         lines = [l for l in r.stdout.splitlines() if l.startswith("{")]
         if r.returncode or not lines:
@@ -285,6 +285,72 @@ def run_all(args):
 # ------------------------------------------------------------------------------------------------
 # CUDA path
 # ------------------------------------------------------------------------------------------------
+def quick_transform(i, dev, peak, steps=10, warmup=3):
+    """Device-resident forward (and, where a second flat buffer fits, inverse) transform of workload i, timed per
+    launch with CUDA events: the per-workload figures that accompany the default workload's line."""
+    import torch
+
+    import paper_2607_22614_b200 as dr
+    import synth
+    from synth.configs import CONFIGS
+
+    cfg = dict(CONFIGS[i], index=i)
+    seed = synth.SEED_BASE + i
+    kw = dict(tp=cfg["tp"], tp_rank=cfg["tp_rank"])
+    free_b, _ = torch.cuda.mem_get_info()
+    probe = dr.Plan(cfg["spec"], world=cfg["world"], rank=cfg["rank"], gathered=cfg["gathered"], host_only=True, **kw)
+    halves = 2 if cfg["gathered"] and probe.info.src_bytes + probe.info.dst_bytes > free_b * 0.92 else 1
+    probe.close()
+    if halves == 2:  # does not fit beside its arena: two shard-local halves, back to back, into the same arena
+        plans = [dr.Plan(cfg["spec"], world=2, rank=r, gathered=False, **kw) for r in (0, 1)]
+    else:
+        plans = [dr.Plan(cfg["spec"], world=cfg["world"], rank=cfg["rank"], gathered=cfg["gathered"], **kw)]
+    info = plans[0].info
+    n_src = info.src_bytes // 4
+    base = cfg["rank"] * info.shard_elems if not cfg["gathered"] else 0
+    master = torch.empty(n_src, dtype=torch.int32, device=dev)
+    synth.cuda_fill_f32(master, seed, synth.BUF_MASTER, start=base)
+    arena = torch.empty(info.dst_bytes, dtype=torch.uint8, device=dev)
+    synth.cuda_fill_bf16(arena.view(torch.int16), seed, synth.BUF_ROLLOUT)
+    do_inverse = halves == 1 and free_b > (2 * info.src_bytes + info.dst_bytes) * 1.05
+    flat_back = torch.empty(n_src, dtype=torch.int32, device=dev) if do_inverse else None
+    fwd, inv = [], []
+    for it in range(warmup + steps):
+        ev = []
+        for h, p in enumerate(plans):
+            if halves == 2:
+                synth.cuda_fill_f32(master, seed, synth.BUF_MASTER, start=h * info.shard_elems)
+            ev.append(torch.cuda.Event(enable_timing=True)); ev[-1].record()
+            p.reshard(master, arena)
+            ev.append(torch.cuda.Event(enable_timing=True)); ev[-1].record()
+        if do_inverse:
+            plans[0].reshard_inverse(arena, flat_back)
+            ev.append(torch.cuda.Event(enable_timing=True)); ev[-1].record()
+        torch.cuda.synchronize()
+        if it >= warmup:
+            fwd.append(sum(ev[2 * h].elapsed_time(ev[2 * h + 1]) for h in range(halves)))
+            if do_inverse:
+                inv.append(ev[-2].elapsed_time(ev[-1]))
+    b_fwd = sum(p.info.bytes_moved_fwd for p in plans)
+    b_inv = plans[0].info.bytes_moved_inv
+    f_ms = sum(fwd) / len(fwd)
+    out = {"cfg": i, "workload": workload_name(cfg), "elements": int(sum(p.info.elems_moved for p in plans)),
+           "passes": halves, "segments": int(sum(p.info.n_segments for p in plans)), "steps": steps,
+           "forward_gbs": b_fwd / f_ms / 1e6, "forward_ms": f_ms, "forward_ms_best": min(fwd),
+           "forward_frac_of_measured_peak": b_fwd / f_ms / 1e6 / peak, "forward_frac_of_nominal_8000": b_fwd / f_ms / 1e6 / 8000.0}
+    if inv:
+        i_ms = sum(inv) / len(inv)
+        out.update({"inverse_gbs": b_inv / i_ms / 1e6, "inverse_ms": i_ms,
+                    "inverse_frac_of_measured_peak": b_inv / i_ms / 1e6 / peak})
+    if info.src_bytes < (64 << 20):
+        out["note"] = "working set fits L2: a latency figure, not a bandwidth one"
+    for p in plans:
+        p.close()
+    del master, arena, flat_back
+    torch.cuda.empty_cache()
+    return out
+
+
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
@@ -295,6 +361,7 @@ def main():
     ap.add_argument("--no-staging", action="store_true", help="skip the host-link sections")
     ap.add_argument("--no-cpu", action="store_true", help="skip the CPU oracle baseline")
     ap.add_argument("--no-fp8", action="store_true", help="skip the fp8 block-quantised variant")
+    ap.add_argument("--no-others", action="store_true", help="skip the short device-only runs of the other workloads")
     ap.add_argument("--cpu-seconds", type=float, default=12.0)
     ap.add_argument("--layers", type=int, default=0, help="profiling aid: override the layer count (smaller case)")
     ap.add_argument("--vocab", type=int, default=0, help="profiling aid: override the vocabulary size")
@@ -533,6 +600,21 @@ def main():
         except Exception as exc:  # e.g. the box cannot pin this much host memory: keep the device-side line
             line.setdefault("staging", {})["error"] = f"{type(exc).__name__}: {exc}"[:300]
             line.setdefault("e2e", {"value": None, "unit": "GB/s", "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0})
+
+    # the other four workloads, device-resident transform only (a few seconds each), so that one run reports all five
+    if world == 1 and not args.no_others and not (args.layers or args.vocab):
+        del master, arena
+        torch.cuda.empty_cache()
+        others = []
+        for i in range(5):
+            if i == args.cfg:
+                continue
+            try:
+                others.append(quick_transform(i, dev, peak))
+            except Exception as exc:
+                others.append({"cfg": i, "error": f"{type(exc).__name__}: {exc}"[:200]})
+                torch.cuda.empty_cache()
+        line["other_workloads"] = others
 
     if rank == 0 and not args.no_cpu and world == 1:
         gbs, elems, spent, desc = oracle_sample(cfg, args.cpu_seconds)

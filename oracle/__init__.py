@@ -159,8 +159,8 @@ class Model:
         self.n_dst = int(lib.orc_n_dst(self._h))
 
     def __del__(self):
-        if getattr(self, "_h", None):
-            _l().orc_model_destroy(self._h)
+        if getattr(self, "_h", None) and _lib is not None:  # at interpreter exit the module may be gone already
+            _lib.orc_model_destroy(self._h)
             self._h = None
 
     def src_tensors(self) -> list[SrcTensor]:

@@ -56,6 +56,10 @@ out = {"rank": rank, "equal_to_gathered_oracle": bool(np.array_equal(arena, want
        "mapped_bytes": int(mapped.sum())}
 for p in plans:
     p.close()
+gathered = [None] * world
+dist.all_gather_object(gathered, out)
 dist.barrier()
 dist.destroy_process_group()
-print(json.dumps(out), flush=True)
+if rank == 0:  # one writer: lines of two processes could interleave
+    for o in gathered:
+        print(json.dumps(o), flush=True)
