@@ -589,6 +589,27 @@ def main():
                                "gbs_best": qb / min(qms) / 1e6, "ms_avg": qavg, "ms_best": min(qms),
                                "frac_of_measured_peak": qb / qavg / 1e6 / peak, "frac_of_nominal_8000": qb / qavg / 1e6 / 8000.0,
                                "algorithmic_bytes_per_quant_elem": 5}
+        # and back: value(code) * scale to the flat fp32 positions (bf16 tensors widened), where a second flat buffer fits
+        free_q, _ = torch.cuda.mem_get_info()
+        if free_q > info.src_bytes * 1.05:
+            qflat = torch.empty(n_src, dtype=torch.int32, device=dev)
+            for _ in range(args.warmup):
+                qplan.reshard_inverse(qarena, qflat)
+            qe = [torch.cuda.Event(enable_timing=True) for _ in range(args.steps + 1)]
+            qe[0].record()
+            for i in range(args.steps):
+                qplan.reshard_inverse(qarena, qflat)
+                qe[i + 1].record()
+            torch.cuda.synchronize()
+            ims = [qe[i].elapsed_time(qe[i + 1]) for i in range(args.steps)]
+            iavg, ib = sum(ims) / len(ims), qplan.info.bytes_moved_inv
+            # round trip on a window of a quantised tensor: |code * scale - x| <= |x| / 16 or half a subnormal code step
+            t1 = [t for t in qplan.tensors() if t.quantised][0]
+            line["fp8_inverse"] = {"what": "dr_reshard_inverse on the same plan (widening kernel + dequantisation kernel)",
+                                   "bytes": int(ib), "gbs_avg": ib / iavg / 1e6, "gbs_best": ib / min(ims) / 1e6, "ms_avg": iavg,
+                                   "ms_best": min(ims), "frac_of_measured_peak": ib / iavg / 1e6 / peak,
+                                   "frac_of_nominal_8000": ib / iavg / 1e6 / 8000.0, "first_quantised_tensor": t1.name.decode()}
+            del qflat
         qplan.close()
         del qarena
         torch.cuda.empty_cache()

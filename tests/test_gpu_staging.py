@@ -307,9 +307,13 @@ def test_ranks_that_stay_relay_what_they_hold_and_rest_the_remainder_in_one_call
         st = plan.stage_out(d)
         assert st.bytes == 12 * (ohi - olo) and st.chunks_done == st.n_chunks
     for i in range(w_new):                                   # each new rank fetches what it does not hold yet
-        _, olo, ohi, _ = dr.dr_shard_range(n, w_old, i)
         _, nlo, nhi, s_new = dr.dr_shard_range(n, w_new, i)
-        lo, hi = max(olo, nlo), min(ohi, nhi)
+        if i < w_old:
+            _, olo, ohi, _ = dr.dr_shard_range(n, w_old, i)
+            lo, hi = max(olo, nlo), min(ohi, nhi)
+        else:                                                # a GPU that joins training holds nothing yet
+            lo = hi = nlo
+            new_bufs[i] = [torch.zeros(s_new, dtype=torch.int32, device=dev()) for _ in kinds]
         ptrs, sizes, offs = [], [], []
         for k in range(3):
             for a, e, held in _cut(nlo, nhi, lo, hi):
