@@ -12,8 +12,10 @@
 // wherever that provably gives the same code: t and the true quotient differ by at most 2 ulp, so they can
 // round to different e4m3 codes only if t lies within a few ulp of a midpoint between two codes (its 20 dropped
 // mantissa bits within 4 of 0x80000) or below 2^-6, where the e4m3 grid is no longer 3 mantissa bits wide.
-// A thread's eight values take the exact division together when any of them is in doubt (about one group in
-// 10^3 for weight-like data).
+// A thread's eight values of a row take the exact division together when any of them is in doubt (about one
+// group in 10^3 for weight-like data).  Whole, aligned blocks (nearly all of them) run a predicate-free body.
+// Parking part of the block in shared memory (cp.async) to raise the CTAs per SM was measured and is slower:
+// the block stays in registers, 256 threads x 64 values, three CTAs per SM.
 #include <cuda_runtime.h>
 
 #include "dr_internal.h"
@@ -58,86 +60,54 @@ __device__ __forceinline__ uint32_t cvt_e4m3x2(float lo, float hi)
     asm("cvt.rn.satfinite.e4m3x2.f32 %0, %1, %2;" : "=h"(d) : "f"(hi), "f"(lo));
     return d;
 }
-// x[k] / scale for a group of one thread's values, as far as the e4m3 codes are concerned: the products with the
-// reciprocal, unless one of them could round to a different code than the true quotient (see the header of
-// this file), in which case the whole group is divided exactly.  The midpoint test is one multiply-add and one
-// compare: shifting the 20 dropped mantissa bits to the top and subtracting (0x80000 - 4) << 12 leaves a
-// value <= 8 << 12 exactly when the bits lie within 4 of 0x80000.
-#ifndef DR_Q_GROUP
-#define DR_Q_GROUP 8  // values sharing one "in doubt" branch
-#endif
-#ifndef DR_Q_TREE
-#define DR_Q_TREE 1  // 1: reduce the group's tests with min trees (short dependency chains); 0: chained predicates
-#endif
-__device__ __forceinline__ void quotients(const float* x, float* t, float scale, float recip, float exact_below)
+// Eight values of one block row -> eight e4m3 codes of x / scale, packed into two words.
+// The codes are first taken from the products with the reciprocal.  Product and true quotient differ by at most
+// 2 ulp, so they can round to different codes only (A) next to a midpoint between two codes: the 20 mantissa bits
+// e4m3 drops lie within 4 of 0x80000, tested with one multiply-add per value (shifting the 20 bits to the top and
+// subtracting (0x80000 - 4) << 12 leaves a value <= 8 << 12) and a min tree; or (B) below 2^-6, where the e4m3
+// grid is no longer 3 mantissa bits wide: tested on the packed codes, four at a time (a code of magnitude
+// <= small_code = 8 means the product rounded to 2^-6 or less).  In either case all eight are redone with the
+// correctly rounded division.  small_code = 0x7F sends every group there (blocks whose reciprocal is not normal).
+__device__ __forceinline__ uint2 pack8(const float* t)
 {
-    bool near = false;
-#if DR_Q_TREE
-    uint32_t d[DR_Q_GROUP];
-    float a[DR_Q_GROUP];
+    const uint32_t h0 = cvt_e4m3x2(t[0], t[1]), h1 = cvt_e4m3x2(t[2], t[3]);
+    const uint32_t h2 = cvt_e4m3x2(t[4], t[5]), h3 = cvt_e4m3x2(t[6], t[7]);
+    return make_uint2(h0 | (h1 << 16), h2 | (h3 << 16));
+}
+__device__ __forceinline__ uint2 quantise8(const float* x, float scale, float recip, uint32_t small_code)
+{
+    float t[8];
+    uint32_t d[8];
 #pragma unroll
-    for (int k = 0; k < DR_Q_GROUP; ++k) {
+    for (int k = 0; k < 8; ++k) {
         t[k] = __fmul_rn(x[k], recip);
         d[k] = __float_as_uint(t[k]) * 4096u - 0x7FFFC000u;
-        a[k] = fabsf(t[k]);
     }
 #pragma unroll
-    for (int w = DR_Q_GROUP / 2; w >= 1; w /= 2)
+    for (int w = 4; w >= 1; w /= 2)  // min tree (three-input minima were measured and are slower)
 #pragma unroll
-        for (int k = 0; k < w; ++k) {
-            d[k] = min(d[k], d[k + w]);
-            a[k] = fminf(a[k], a[k + w]);  // a NaN operand is dropped: a NaN needs no exact division
-        }
-    near = (d[0] <= 0x8000u) | (a[0] < exact_below);
-#else
+        for (int k = 0; k < w; ++k) d[k] = min(d[k], d[k + w]);
+    const uint32_t dmin = d[0];
+    uint2 q = pack8(t);
+    // per byte: magnitude + (0x7F - small_code) reaches bit 7 exactly when the magnitude exceeds small_code
+    const uint32_t bias = (0x7Fu - small_code) * 0x01010101u;
+    const uint32_t big = ((q.x & 0x7F7F7F7Fu) + bias) & ((q.y & 0x7F7F7F7Fu) + bias) & 0x80808080u;
+    if (dmin <= 0x8000u || big != 0x80808080u) {
 #pragma unroll
-    for (int k = 0; k < DR_Q_GROUP; ++k) {
-        t[k] = __fmul_rn(x[k], recip);
-        const uint32_t d = __float_as_uint(t[k]) * 4096u - 0x7FFFC000u;
-        near |= (d <= 0x8000u) | (fabsf(t[k]) < exact_below);
+        for (int k = 0; k < 8; ++k) t[k] = __fdiv_rn(x[k], scale);
+        q = pack8(t);
     }
-#endif
-    if (near) {
-#pragma unroll
-        for (int k = 0; k < DR_Q_GROUP; ++k) t[k] = __fdiv_rn(x[k], scale);
-    }
+    return q;
 }
-__global__ void __launch_bounds__(kQThreads, DR_Q_MIN_BLOCKS)
-    quant_kernel(const QTensor* __restrict__ tensors, uint32_t n_tensors, const QPart* __restrict__ parts,
-                 const uint32_t* __restrict__ hints, uint32_t hint_shift, const char* __restrict__ flat,
-                 char* __restrict__ arena, int allow256, uint64_t block_begin)
+
+// One 128 x 128 block.  FAST: the block is whole (128 rows, 128 columns inside the tensor), its rows allow
+// 256-bit loads and the buffers' bases are 32-byte aligned, so no access needs a predicate.
+template <bool FAST>
+__device__ __forceinline__ void quant_block(const QTensor& T, uint32_t bi, uint32_t bj, uint32_t nrows,
+                                            const uint64_t* row_src, float* warp_max, float* s_scale,
+                                            const char* __restrict__ flat, char* __restrict__ arena, int allow256)
 {
-    __shared__ uint64_t row_src[128];  // flat element offset of (row, first column of the tensor)
-    __shared__ float warp_max[kQThreads / 32];
-    __shared__ float s_scale;
-
-    const uint64_t b = block_begin + blockIdx.x;
-    // block -> tensor: hint plus a short walk (all threads, same addresses: broadcast loads)
-    uint32_t ti = hints[b >> hint_shift];
-    while (ti + 1 < n_tensors && tensors[ti + 1].block0 <= b) ++ti;
-    const QTensor T = tensors[ti];
-    const uint32_t lb = (uint32_t)(b - T.block0);
-    const uint32_t bi = lb / T.nbc, bj = lb - bi * T.nbc;
     const uint32_t r0 = bi * 128, c0 = bj * 128;
-    const uint32_t nrows = min(128u, T.rows - r0);
-
-    // each of the first 128 threads finds the source row of one block row (binary search over the parts)
-    if (threadIdx.x < 128) {
-        uint64_t off = 0;
-        const uint32_t r = r0 + threadIdx.x;
-        if (threadIdx.x < nrows) {
-            uint32_t lo = T.part0, hi = T.part0 + T.n_parts;  // last part with dst_row0 <= r
-            while (hi - lo > 1) {
-                uint32_t mid = lo + (hi - lo) / 2;
-                if (parts[mid].dst_row0 <= r) lo = mid; else hi = mid;
-            }
-            const QPart P = parts[lo];
-            off = P.src_off + (uint64_t)(r - P.dst_row0) * P.src_stride;
-        }
-        row_src[threadIdx.x] = off;
-    }
-    __syncthreads();
-
     const uint32_t cu = threadIdx.x & 15;   // 8-column unit inside the block row
     const uint32_t rb = threadIdx.x >> 4;   // row inside a pass
     const uint32_t col = c0 + cu * 8;
@@ -146,21 +116,25 @@ __global__ void __launch_bounds__(kQThreads, DR_Q_MIN_BLOCKS)
 #pragma unroll
     for (int p = 0; p < kPasses; ++p) {
         const uint32_t row = p * kRowsPerPass + rb;
+        if (FAST) {
+            ld256f(flat + (row_src[row] + col) * 4, v[p]);
+        } else {
 #pragma unroll
-        for (int k = 0; k < 8; ++k) v[p][k] = 0.0f;
-        if (row < nrows && col < T.cols) {
-            const char* src = flat + (row_src[row] + col) * 4;
-            // T.aligned speaks of offsets from the flat base; the base itself is only promised to be 16-byte
-            // aligned, so the 256-bit form also needs a 32-byte aligned base (allow256)
-            if (T.aligned && allow256) {
-                ld256f(src, v[p]);
-            } else if (T.aligned) {
-                ld128f(src, &v[p][0]);
-                ld128f(src + 16, &v[p][4]);
-            } else {
+            for (int k = 0; k < 8; ++k) v[p][k] = 0.0f;
+            if (row < nrows && col < T.cols) {
+                const char* src = flat + (row_src[row] + col) * 4;
+                // T.aligned speaks of offsets from the flat base; the base itself is only promised to be 16-byte
+                // aligned, so the 256-bit form also needs a 32-byte aligned base (allow256)
+                if (T.aligned && allow256) {
+                    ld256f(src, v[p]);
+                } else if (T.aligned) {
+                    ld128f(src, &v[p][0]);
+                    ld128f(src + 16, &v[p][4]);
+                } else {
 #pragma unroll
-                for (int k = 0; k < 8; ++k)
-                    if (col + k < T.cols) v[p][k] = ld32f(src + 4 * k);
+                    for (int k = 0; k < 8; ++k)
+                        if (col + k < T.cols) v[p][k] = ld32f(src + 4 * k);
+                }
             }
         }
     }
@@ -179,44 +153,72 @@ __global__ void __launch_bounds__(kQThreads, DR_Q_MIN_BLOCKS)
         // amax / 448, held inside the normal fp32 range: 2^-126 for blocks whose amax / 448 underflows (the
         // all-zero block among them), FLT_MAX for a block holding an infinity
         float scale = fminf(fmaxf(__fdiv_rn(m, 448.0f), 1.17549435e-38f), 3.40282347e+38f);
-        s_scale = scale;
+        *s_scale = scale;
         *(float*)(arena + T.scale_off + ((uint64_t)bi * T.nbc + bj) * 4) = scale;
     }
     __syncthreads();
-    const float scale = s_scale;
+    const float scale = *s_scale;
     const float recip = __frcp_rn(scale);
     // the product form needs a normal reciprocal (scale <= 2^126: always, except for the infinity block);
-    // otherwise every element takes the exact division
-    const float exact_below = recip >= 1.17549435e-38f ? 0.015625f : __int_as_float(0x7F800000);
+    // otherwise every group takes the exact division
+    const uint32_t small_code = recip >= 1.17549435e-38f ? 8u : 0x7Fu;
 
 #pragma unroll
     for (int p = 0; p < kPasses; ++p) {
         const uint32_t row = p * kRowsPerPass + rb;
-        if (row >= nrows || col >= T.cols) continue;
-        uint32_t q[8];
-        float t[8];
-#pragma unroll
-        for (int k = 0; k < 8; k += DR_Q_GROUP) quotients(&v[p][k], &t[k], scale, recip, exact_below);
-#pragma unroll
-        for (int k = 0; k < 8; k += 2) {
-            const uint32_t two = cvt_e4m3x2(t[k], t[k + 1]);
-            q[k] = two & 0xFF;
-            q[k + 1] = two >> 8;
-        }
+        if (!FAST && (row >= nrows || col >= T.cols)) continue;
+        const uint2 q = quantise8(v[p], scale, recip, small_code);
         char* dst = arena + T.payload_off + (uint64_t)(r0 + row) * T.cols + col;
-        if (T.aligned) {
-            uint2 w;
-            w.x = q[0] | (q[1] << 8) | (q[2] << 16) | (q[3] << 24);
-            w.y = q[4] | (q[5] << 8) | (q[6] << 16) | (q[7] << 24);
-            asm volatile("st.global.L1::no_allocate.v2.b32 [%0], {%1,%2};" ::"l"(dst), "r"(w.x), "r"(w.y) : "memory");
+        if (FAST || T.aligned) {
+            asm volatile("st.global.L1::no_allocate.v2.b32 [%0], {%1,%2};" ::"l"(dst), "r"(q.x), "r"(q.y) : "memory");
         } else {
 #pragma unroll
             for (int k = 0; k < 8; ++k)
-                if (col + k < T.cols) dst[k] = (char)q[k];
+                if (col + k < T.cols) dst[k] = (char)(((k < 4 ? q.x : q.y) >> (8 * (k & 3))) & 0xFF);
         }
     }
 }
 
+__global__ void __launch_bounds__(kQThreads, DR_Q_MIN_BLOCKS)
+    quant_kernel(const QTensor* __restrict__ tensors, uint32_t n_tensors, const QPart* __restrict__ parts,
+                 const uint32_t* __restrict__ hints, uint32_t hint_shift, const char* __restrict__ flat,
+                 char* __restrict__ arena, int allow256, uint64_t block_begin)
+{
+    __shared__ uint64_t row_src[128];  // flat element offset of (row, first column of the tensor)
+    __shared__ float warp_max[kQThreads / 32];
+    __shared__ float s_scale;
+
+    const uint64_t b = block_begin + blockIdx.x;
+    // block -> tensor: hint plus a short walk (all threads, same addresses: broadcast loads)
+    uint32_t ti = hints[b >> hint_shift];
+    while (ti + 1 < n_tensors && tensors[ti + 1].block0 <= b) ++ti;
+    const QTensor T = tensors[ti];
+    const uint32_t lb = (uint32_t)(b - T.block0);
+    const uint32_t bi = lb / T.nbc, bj = lb - bi * T.nbc;
+    const uint32_t r0 = bi * 128;
+    const uint32_t nrows = min(128u, T.rows - r0);
+
+    // each of the first 128 threads finds the source row of one block row (binary search over the parts)
+    if (threadIdx.x < 128) {
+        uint64_t off = 0;
+        const uint32_t r = r0 + threadIdx.x;
+        if (threadIdx.x < nrows) {
+            uint32_t lo = T.part0, hi = T.part0 + T.n_parts;  // last part with dst_row0 <= r
+            while (hi - lo > 1) {
+                uint32_t mid = lo + (hi - lo) / 2;
+                if (parts[mid].dst_row0 <= r) lo = mid; else hi = mid;
+            }
+            const QPart P = parts[lo];
+            off = P.src_off + (uint64_t)(r - P.dst_row0) * P.src_stride;
+        }
+        row_src[threadIdx.x] = off;
+    }
+    __syncthreads();
+    if (nrows == 128 && bj * 128 + 128 <= T.cols && T.aligned && allow256)
+        quant_block<true>(T, bi, bj, nrows, row_src, warp_max, &s_scale, flat, arena, allow256);
+    else
+        quant_block<false>(T, bi, bj, nrows, row_src, warp_max, &s_scale, flat, arena, allow256);
+}
 
 // ---- the inverse: e4m3 codes times the block's scale, back to the flat fp32 positions ----------------------
 // Same decomposition (one CTA per 128 x 128 block, 16 threads per block row, eight values per thread and row),
