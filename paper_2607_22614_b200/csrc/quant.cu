@@ -261,6 +261,7 @@ __global__ void __launch_bounds__(kQThreads)
         row_src[threadIdx.x] = off;
     }
     const float scale = *(const float*)(arena + T.scale_off + ((uint64_t)bi * T.nbc + bj) * 4);
+    const bool finite_scale = (__float_as_uint(scale) & 0x7F800000u) != 0x7F800000u;
     __syncthreads();
 
     const uint32_t cu = threadIdx.x & 15, rb = threadIdx.x >> 4;
@@ -286,14 +287,23 @@ __global__ void __launch_bounds__(kQThreads)
         const uint32_t row = p * kRowsPerPass + rb;
         if (row >= nrows || col >= T.cols) continue;
         uint32_t y[8];
+        // A product can only be NaN if a code is a NaN code (magnitude 0x7F: + 1 reaches bit 7) or the scale is not
+        // finite; without either, the eight products need no NaN check.
+        const uint32_t nan_code = (((q[p][0] & 0x7F7F7F7Fu) + 0x01010101u) | ((q[p][1] & 0x7F7F7F7Fu) + 0x01010101u)) & 0x80808080u;
+        const bool check = nan_code != 0 || !finite_scale;
 #pragma unroll
         for (int k = 0; k < 8; k += 2) {
             float lo, hi;
             e4m3x2_to_f32((q[p][k >> 2] >> (8 * (k & 3))) & 0xFFFF, lo, hi);
             lo = __fmul_rn(lo, scale);
             hi = __fmul_rn(hi, scale);
-            y[k] = lo != lo ? 0x7FC00000u : __float_as_uint(lo);
-            y[k + 1] = hi != hi ? 0x7FC00000u : __float_as_uint(hi);
+            y[k] = __float_as_uint(lo);
+            y[k + 1] = __float_as_uint(hi);
+        }
+        if (check) {
+#pragma unroll
+            for (int k = 0; k < 8; ++k)
+                if ((y[k] & 0x7FFFFFFFu) > 0x7F800000u) y[k] = 0x7FC00000u;
         }
         char* dst = flat + (row_src[row] + col) * 4;
         if (T.aligned && allow256) {
