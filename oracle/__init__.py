@@ -85,7 +85,7 @@ def _l():
         lib.orc_forward_fp8.restype = ctypes.c_int
         lib.orc_forward_fp8.argtypes = [p, p, p, i64]
         lib.orc_inverse_fp8.restype = ctypes.c_int
-        lib.orc_inverse_fp8.argtypes = [p, p, p]
+        lib.orc_inverse_fp8.argtypes = [p, p, p, i64]
         lib.orc_restage_out.restype = None
         lib.orc_restage_out.argtypes = [p, u64, u64, u64, p]
         lib.orc_restage_in.restype = None
@@ -210,11 +210,11 @@ class Model:
         assert arena_u8.dtype == np.uint8 and arena_u8.size >= self.fp8_layout()[0]
         _l().orc_forward_fp8(self._h, src_u32.ctypes.data, arena_u8.ctypes.data, only)
 
-    def inverse_fp8(self, arena_u8: np.ndarray, flat_u32: np.ndarray) -> None:
+    def inverse_fp8(self, arena_u8: np.ndarray, flat_u32: np.ndarray, only: int = -1) -> None:
         """Inverse of D7: codes times block scales (and widened bf16 tensors) back to their flat positions."""
         assert flat_u32.dtype == np.uint32 and flat_u32.flags.c_contiguous and flat_u32.size >= self.flat_elems
         assert arena_u8.dtype == np.uint8 and arena_u8.flags.c_contiguous and arena_u8.size >= self.fp8_layout()[0]
-        _l().orc_inverse_fp8(self._h, arena_u8.ctypes.data, flat_u32.ctypes.data)
+        _l().orc_inverse_fp8(self._h, arena_u8.ctypes.data, flat_u32.ctypes.data, only)
 
     def inverse(self, arena_u8: np.ndarray, flat_u32: np.ndarray, *, gathered: bool = True, rank: int = 0) -> None:
         assert flat_u32.dtype == np.uint32 and flat_u32.flags.c_contiguous

@@ -827,13 +827,14 @@ int orc_forward_fp8(const orc_model *m, const uint32_t *src, uint8_t *arena, int
  * exact e4m3 value, one fp32 multiplication (round to nearest); a NaN code, or a NaN product (a scale
  * that is itself NaN, or 0 * Inf), becomes the quiet NaN 0x7FC00000.  Positions no rollout element maps
  * to keep their words. */
-int orc_inverse_fp8(const orc_model *m, const uint8_t *arena, uint32_t *flat)
+int orc_inverse_fp8(const orc_model *m, const uint8_t *arena, uint32_t *flat, int64_t only)
 {
     uint64_t i, p, r, c;
     for (i = 0; i < m->n_dst; ++i) {
         const orc_dst *d = &m->dst[i];
         int qz;
         uint64_t off, soff, nbc = (d->cols + 127) / 128;
+        if (only >= 0 && (uint64_t)only != i) continue; /* the same loop over one rollout tensor */
         if (d->alias_of >= 0) continue;
         orc_fp8_layout(m, i, &qz, &off, &soff);
         for (p = 0; p < d->n_parts; ++p) {

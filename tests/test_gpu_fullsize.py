@@ -317,3 +317,72 @@ def test_cfg1_streamed_repack_equals_resident_repack():
     assert torch.equal(arena, ref)
     assert torch.equal(h_dst, ref.cpu())
     plan.close()
+
+
+def test_cfg1_eight_ranks_push_into_two_arenas_equals_oracle():
+    """The Qwen3-1.7B-shaped flat buffer cut into its eight FSDP shards: every rank repacks its own shard and
+    stores the pieces into two rollout arenas with dr_reshard_push (ranks one after the other on this GPU).
+    Both arenas must equal the oracle's gathered forward, all 1.72 GB of each."""
+    _need(14)
+    cfg = CONFIGS[1]
+    _, om = _models(cfg)
+    seed = seed_of(1)
+    S = om.shard_elems
+    arenas = [torch.full((om.arena_bytes,), 0xA5, dtype=torch.uint8, device=DEV) for _ in range(2)]
+    shard = torch.empty(S, dtype=torch.int32, device=DEV)
+    moved = 0
+    for r in range(cfg["world"]):
+        plan = dr.Plan(cfg["spec"], world=cfg["world"], rank=r, gathered=False, tp=cfg["tp"], tp_rank=cfg["tp_rank"])
+        synth.cuda_fill_f32(shard, seed, synth.BUF_MASTER, start=r * S)
+        plan.reshard_push(shard, arenas)
+        moved += plan.info.elems_moved
+        torch.cuda.synchronize()
+        plan.close()
+    assert moved == 860_349_440
+    flat = synth.fill_f32(seed, synth.BUF_MASTER, 0, om.world * S)
+    want = np.full(om.arena_bytes, 0xA5, dtype=np.uint8)
+    om.forward(flat, want)
+    for a in arenas:
+        assert np.array_equal(a.cpu().numpy(), want)
+
+
+def test_cfg2_fp8_inverse_full_size_sampled_tensors():
+    """Qwen3-8B-shaped fp8 arena (random codes, scales of weight-like size) back to the 32.8 GB flat buffer:
+    the oracle's inverse on every tensor of layers 0 and 35 (the layers' whole flat ranges are compared)."""
+    _need(50)
+    cfg = CONFIGS[2]
+    plan = dr.Plan(cfg["spec"], dtype=dr.DR_FP8_E4M3_B128)
+    om = oracle.Model(cfg["spec"])
+    total, lay = om.fp8_layout()
+    assert plan.info.dst_bytes == total
+    arena = torch.empty(total, dtype=torch.uint8, device=DEV)
+    synth.cuda_fill_bf16(arena[:total // 2 * 2].view(torch.int16), seed_of(2), synth.BUF_ROLLOUT)   # every byte value occurs
+    dst = om.dst_tensors()
+    rng = np.random.default_rng(4)
+    for d, (qz, off, soff) in zip(dst, lay):                      # sane block scales for the quantised tensors
+        if qz and d.alias_of < 0:
+            nb = (-(-d.rows // 128)) * (-(-d.cols // 128))
+            sc = np.exp(rng.uniform(-12, -6, nb)).astype(np.float32)
+            arena[soff:soff + 4 * nb] = torch.from_numpy(sc.view(np.uint8)).to(DEV)
+    flat = torch.full((om.flat_elems,), 0x5A5A5A5A, dtype=torch.int32, device=DEV)
+    plan.reshard_inverse(arena, flat)
+    torch.cuda.synchronize()
+    host_arena = np.empty(total, dtype=np.uint8)                   # lazily committed; only the tested tensors are filled
+    want = np.empty(om.flat_elems, dtype=np.uint32)
+    srcs = {s.name: s for s in om.src_tensors()}
+    for layer in (0, 35):
+        names = [n for n in srcs if n.startswith(f"layers.{layer}.")]
+        lo = min(srcs[n].flat_off for n in names)
+        hi = max(srcs[n].flat_off + srcs[n].rows * srcs[n].cols for n in names)
+        want[lo:hi] = 0x5A5A5A5A
+        for i, (d, (qz, off, soff)) in enumerate(zip(dst, lay)):
+            if d.name.startswith(f"layers.{layer}."):
+                nbytes = d.rows * d.cols * (1 if qz else 2)
+                host_arena[off:off + nbytes] = arena[off:off + nbytes].cpu().numpy()
+                if qz:
+                    nb = 4 * (-(-d.rows // 128)) * (-(-d.cols // 128))
+                    host_arena[soff:soff + nb] = arena[soff:soff + nb].cpu().numpy()
+                om.inverse_fp8(host_arena, want, only=i)   # the oracle's loop over this rollout tensor alone
+        got = flat[lo:hi].cpu().numpy().view(np.uint32)
+        assert np.array_equal(got, want[lo:hi]), layer
+    plan.close()
