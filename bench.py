@@ -614,6 +614,37 @@ def main():
         del qarena
         torch.cuda.empty_cache()
 
+    # the exchange fused into the repack, as far as one GPU can time it: rank 0 of a world of two repacks its shard
+    # and stores the pieces into two arenas of this GPU (the second stands for a peer's; over NVLink the stores to it
+    # would be bound by the link instead of HBM)
+    if cfg["gathered"] and halves == 1 and not args.no_fp8:
+        xplan = dr.Plan(cfg["spec"], world=2, rank=0, gathered=False, tp=cfg["tp"], tp_rank=cfg["tp_rank"])
+        free_x, _ = torch.cuda.mem_get_info()
+        if free_x > info.dst_bytes * 1.1:
+            arena2 = torch.empty(info.dst_bytes, dtype=torch.uint8, device=dev)
+            shard = master[:xplan.info.src_bytes // 4]
+            for _ in range(args.warmup):
+                xplan.reshard_push(shard, [arena, arena2])
+            xe = [torch.cuda.Event(enable_timing=True) for _ in range(args.steps + 1)]
+            xe[0].record()
+            for i in range(args.steps):
+                xplan.reshard_push(shard, [arena, arena2])
+                xe[i + 1].record()
+            torch.cuda.synchronize()
+            xms = [xe[i].elapsed_time(xe[i + 1]) for i in range(args.steps)]
+            xavg = sum(xms) / len(xms)
+            xb = xplan.info.elems_moved * (4 + 2 * 2)
+            same = bool(torch.equal(arena[:1 << 24], arena2[:1 << 24]))
+            line["exchange_local"] = {"what": "dr_reshard_push: rank 0 of 2 repacks its shard into two arenas of this GPU in one kernel "
+                                              "(4 B read + 2 x 2 B written per element); multi-GPU rate unmeasured in this run",
+                                      "elements": int(xplan.info.elems_moved), "n_dst": 2, "bytes": int(xb),
+                                      "ranges_of_this_rank": len(xplan.ranges()), "gbs_avg": xb / xavg / 1e6, "ms_avg": xavg,
+                                      "ms_best": min(xms), "arenas_agree_on_window": same}
+            del arena2
+            plans[0].reshard(master, arena)  # put the whole arena back
+        xplan.close()
+        torch.cuda.empty_cache()
+
     # ---- host-link sections ---------------------------------------------------------------------
     if not args.no_staging:
         try:
@@ -830,7 +861,13 @@ def staging_sections(args, cfg, plan, master, arena, seed, base, dev, world, lin
 
         eight = ring(budget, budget // 8 // 4096 * 4096)          # the workload's budget as eight slots
         two = ring(budget, budget // 2 // 4096 * 4096)            # ... and as two
-        small = ring(256 << 20, 16 << 20) if 4 * n >= (1 << 30) else None
+        # a ring small enough to stay in the host's last-level cache (it uses 64 MiB of the budget): the chunks are
+        # copied out right behind the DMA that delivered them, and filled right before the DMA that reads them
+        small = ring(64 << 20, 8 << 20) if 4 * n >= (1 << 30) else None
+        small16 = ring(64 << 20, 4 << 20) if 4 * n >= (1 << 30) else None
+        rings = [x for x in (eight, two, small, small16) if x]
+        best_out = max(rings, key=lambda x: x["stage_out_gbs"])
+        best_in = max(rings, key=lambda x: x["stage_in_gbs"])
         # CPU baseline of this path: the engine's multi-threaded host copy on its own, and the same copy while the
         # link moves data in the same direction beside it (what the ring path has to share the host's memory with)
         hb = min(4 * n, GiB)
@@ -882,12 +919,11 @@ def staging_sections(args, cfg, plan, master, arena, seed, base, dev, world, lin
         c_in, dma_in = beside_dma(p1, pg, False)
         del p1, p2, scratch
         out["staging"]["through_ring_to_pageable"] = {
-            "bytes": int(4 * n), "eight_slots": eight, "two_slots": two, "with_256MiB_budget_16MiB_chunks": small,
-            "stage_out_gbs": max(eight["stage_out_gbs"], two["stage_out_gbs"]),
-            "stage_in_gbs": max(eight["stage_in_gbs"], two["stage_in_gbs"]),
-            "stage_out_frac_of_link": max(eight["stage_out_frac_of_link"], two["stage_out_frac_of_link"]),
-            "stage_in_frac_of_link": max(eight["stage_in_frac_of_link"], two["stage_in_frac_of_link"]),
-            "bytes_match": bool(eight["bytes_match"] and two["bytes_match"]),
+            "bytes": int(4 * n), "eight_slots": eight, "two_slots": two, "ring_64MiB_8x8MiB": small, "ring_64MiB_16x4MiB": small16,
+            "stage_out_gbs": best_out["stage_out_gbs"], "stage_in_gbs": best_in["stage_in_gbs"],
+            "stage_out_frac_of_link": best_out["stage_out_frac_of_link"], "stage_in_frac_of_link": best_in["stage_in_frac_of_link"],
+            "best_geometry": {"stage_out": [best_out["slots"], best_out["chunk_bytes"]], "stage_in": [best_in["slots"], best_in["chunk_bytes"]]},
+            "bytes_match": bool(all(x["bytes_match"] for x in rings)),
             "cpu_baseline_host_copy": {
                 "what": "dr_host_copy, the engine's multi-threaded copy (non-temporal stores), 1 GiB, this box's host cores",
                 "threads": min(16, os.cpu_count() or 1),

@@ -332,6 +332,13 @@ typedef int (*dr_chunk_fn)(void* user, uint64_t chunk_idx, uint64_t stream_off, 
  *                        stream image, or host_offset[i] with DR_STAGE_HOST_OFFSETS); a pinned arena is
  *                        copied to directly (still chunk by chunk), a pageable one through the ring by
  *                        worker threads
+ * A pageable arena is served by worker threads behind the pump (ring slot -> arena on the way out, arena ->
+ * ring slot on the way in, in tasks of 1 MiB), so several chunks are in flight on the host side as well.
+ * For such an arena a small ring is the fast one: about eight slots of 4 - 8 MiB stay in the host's
+ * last-level cache, so a chunk is copied out right behind the DMA that delivered it (and filled right
+ * before the DMA that reads it) without a round trip through host DRAM; measured 0.85 - 0.97 of the link
+ * against 0.70 - 0.88 with slots of 256 MiB - 1 GiB.  Rings of at most 64 MiB are filled with ordinary
+ * stores on the way in, larger ones with non-temporal stores.
  * One stage-out call may mix relay and arena buffers: a rank that keeps training under a new world size
  * relays the part of its new shard it already holds and rests the remainder of its old shard on the
  * host in the same pass.  A non-empty buffer with neither place to go is DR_ERR_INVALID.

@@ -119,7 +119,10 @@ void CopyPool::loop(unsigned i)
     }
 }
 
-Drainer::Drainer(CopyPool* pool) : pool_(pool), th_([this] { loop(); }) {}
+Drainer::Drainer(unsigned n_threads)
+{
+    for (unsigned i = 0; i < (n_threads ? n_threads : 1); ++i) th_.emplace_back([this] { loop(); });
+}
 
 Drainer::~Drainer()
 {
@@ -128,47 +131,48 @@ Drainer::~Drainer()
         stop_ = true;
     }
     work_.notify_all();
-    th_.join();
+    for (auto& t : th_) t.join();
 }
 
-void Drainer::submit(const Part* parts, unsigned n_parts)
+void Drainer::submit(const Part* parts, unsigned n_parts, std::atomic<uint32_t>* pending)
 {
+    uint32_t n_tasks = 0;
+    for (unsigned i = 0; i < n_parts; ++i) n_tasks += (uint32_t)((parts[i].n + kTaskBytes - 1) / kTaskBytes);
+    pending->store(n_tasks, std::memory_order_release);
+    if (n_tasks == 0) return;
     {
         std::lock_guard<std::mutex> l(mu_);
-        q_.emplace_back(parts, parts + n_parts);
+        for (unsigned i = 0; i < n_parts; ++i)
+            for (uint64_t off = 0; off < parts[i].n; off += kTaskBytes)
+                q_.push_back(Task{parts[i].dst + off, parts[i].src + off, std::min(kTaskBytes, parts[i].n - off), parts[i].cached,
+                                 pending});
     }
-    work_.notify_one();
+    if (n_tasks == 1) work_.notify_one(); else work_.notify_all();
 }
 
-uint64_t Drainer::completed()
+bool Drainer::wait_zero(const std::atomic<uint32_t>* pending, std::chrono::steady_clock::time_point deadline)
 {
-    std::lock_guard<std::mutex> l(mu_);
-    return completed_;
-}
-
-bool Drainer::wait_completed(uint64_t count, std::chrono::steady_clock::time_point deadline)
-{
+    if (pending->load(std::memory_order_acquire) == 0) return true;
     std::unique_lock<std::mutex> l(mu_);
-    return done_.wait_until(l, deadline, [&] { return completed_ >= count; });
+    return done_.wait_until(l, deadline, [&] { return pending->load(std::memory_order_acquire) == 0; });
 }
 
 void Drainer::loop()
 {
     for (;;) {
-        std::vector<Part> job;
+        Task t;
         {
             std::unique_lock<std::mutex> l(mu_);
             work_.wait(l, [&] { return stop_ || !q_.empty(); });
             if (q_.empty()) return;  // stop requested and nothing left to copy
-            job.swap(q_.front());
+            t = q_.front();
             q_.pop_front();
         }
-        for (const Part& p : job) pool_->copy(p.dst, p.src, p.n);
-        {
-            std::lock_guard<std::mutex> l(mu_);
-            ++completed_;
+        if (t.cached) memcpy(t.dst, t.src, t.n); else copy_bytes(t.dst, t.src, t.n);
+        if (t.pending->fetch_sub(1, std::memory_order_acq_rel) == 1) {  // the chunk's last task
+            std::lock_guard<std::mutex> l(mu_);                          // pairs with the waiter's predicate check
+            done_.notify_all();
         }
-        done_.notify_all();
     }
 }
 

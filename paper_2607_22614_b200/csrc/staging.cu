@@ -1,5 +1,5 @@
 // Bounded chunked host staging: a pinned ring of chunk slots, a copy stream and a relay stream,
-// and a small worker pool that moves chunks between the ring and a pageable host arena.
+// and worker threads that move chunks between the ring and a pageable host arena behind the pump.
 // Every wait is a bounded host-side poll; there is no device-side waiting anywhere.
 #include <cuda_runtime.h>
 
@@ -23,6 +23,12 @@ using Clock = std::chrono::steady_clock;
 
 double ms_since(Clock::time_point t0) { return std::chrono::duration<double, std::milli>(Clock::now() - t0).count(); }
 
+// Rings up to this size are filled with ordinary (cached) stores on stage-in.
+#ifndef DR_CACHED_RING_BYTES
+#define DR_CACHED_RING_BYTES (64ull << 20)
+#endif
+constexpr uint64_t kCachedRingBytes = DR_CACHED_RING_BYTES;
+
 // A single core cannot keep up with the host link; beyond 16 threads the copy is bound by memory, not cores.
 unsigned default_copy_threads()
 {
@@ -34,13 +40,15 @@ unsigned default_copy_threads()
 
 struct Ring {
     cudaStream_t s_copy = nullptr, s_relay = nullptr;
-    char* base = nullptr;  // pinned, slots * chunk bytes
+    char* base = nullptr;  // pinned, at least slots * chunk bytes
+    uint64_t capacity = 0; // bytes allocated at base
     uint64_t chunk = 0;
     uint32_t slots = 0;
     std::vector<cudaEvent_t> ev_copy, ev_relay;  // one per slot
     cudaEvent_t ev_entry = nullptr;              // recorded on the caller's stream when a call begins
-    std::unique_ptr<CopyPool> pool;
     std::unique_ptr<Drainer> drainer;  // started by the first stage-out into a pageable arena
+    std::unique_ptr<std::atomic<uint32_t>[]> pending;  // per slot: host-copy tasks of the chunk in it still to run
+    uint32_t pending_slots = 0;
 };
 
 void ring_destroy(Ring* r)
@@ -95,7 +103,7 @@ int geometry(const dr_stage_desc* d, Geometry* g)
     return DR_OK;
 }
 
-int ensure_ring(dr_plan* p, const Geometry& g, bool need_memory)
+int ensure_ring(dr_plan* p, const Geometry& g, bool need_memory, uint64_t budget)
 {
     if (!p->ring) {
         Ring* r = new (std::nothrow) Ring();
@@ -104,12 +112,6 @@ int ensure_ring(dr_plan* p, const Geometry& g, bool need_memory)
         DR_CUDA(cudaStreamCreateWithFlags(&r->s_copy, cudaStreamNonBlocking));
         DR_CUDA(cudaStreamCreateWithFlags(&r->s_relay, cudaStreamNonBlocking));
         DR_CUDA(cudaEventCreateWithFlags(&r->ev_entry, cudaEventDisableTiming));
-        try {
-            r->pool.reset(new CopyPool(default_copy_threads()));
-        } catch (const std::exception& e) {
-            set_error("cannot start the host copy threads: %s", e.what());
-            return DR_ERR_NOMEM;
-        }
     }
     Ring* r = p->ring;
     while (r->ev_copy.size() < g.slots) {
@@ -119,19 +121,39 @@ int ensure_ring(dr_plan* p, const Geometry& g, bool need_memory)
         DR_CUDA(cudaEventCreateWithFlags(&b, cudaEventDisableTiming));
         r->ev_relay.push_back(b);
     }
-    if (need_memory && (r->chunk != g.chunk || r->slots != g.slots)) {
+    // a ring that is large enough, and not larger than this call's budget, is kept and re-cut
+    if (need_memory && (g.chunk * g.slots > r->capacity || r->capacity > budget)) {
         if (r->base) {
             DR_CUDA(cudaStreamSynchronize(r->s_copy));
             DR_CUDA(cudaStreamSynchronize(r->s_relay));
             cudaFreeHost(r->base);
             r->base = nullptr;
-            r->chunk = 0;
-            r->slots = 0;
+            r->capacity = 0;
         }
         DR_CUDA(cudaHostAlloc((void**)&r->base, g.chunk * g.slots, cudaHostAllocDefault));
+        r->capacity = g.chunk * g.slots;
+    }
+    if (need_memory) {
         r->chunk = g.chunk;
         r->slots = g.slots;
     }
+    return DR_OK;
+}
+
+// Worker threads and per-slot task counters for copies between the ring and a pageable arena.
+int ensure_drainer(Ring* r, uint32_t slots)
+{
+    try {
+        if (!r->drainer) r->drainer.reset(new Drainer(default_copy_threads()));
+        if (r->pending_slots < slots) {
+            r->pending.reset(new std::atomic<uint32_t>[slots]);
+            r->pending_slots = slots;
+        }
+    } catch (const std::exception& e) {
+        set_error("cannot start the host copy threads: %s", e.what());
+        return DR_ERR_NOMEM;
+    }
+    for (uint32_t i = 0; i < slots; ++i) r->pending[i].store(0);
     return DR_OK;
 }
 
@@ -271,7 +293,7 @@ extern "C" int dr_stage_out(dr_plan* plan, const dr_stage_desc* d, dr_stage_stat
     const bool pinned_arena = any_host && is_pinned_host(d->host_arena);  // DMA straight into the arena
     const bool via_drainer = any_host && !pinned_arena;                   // pageable arena: drainer thread copies out
     const bool need_ring = d->callback || any_relay || via_drainer;
-    if ((rc = ensure_ring(plan, g, need_ring))) return rc;
+    if ((rc = ensure_ring(plan, g, need_ring, d->budget_bytes))) return rc;
     Ring* r = plan->ring;
     const auto t0 = Clock::now();
     const auto limit = std::chrono::milliseconds(d->timeout_ms ? d->timeout_ms : 60000);
@@ -309,17 +331,9 @@ extern "C" int dr_stage_out(dr_plan* plan, const dr_stage_desc* d, dr_stage_stat
         }
         return DR_OK;
     };
-    // A pageable arena is filled by the drainer thread: the pump hands it a chunk as soon as the chunk has
-    // arrived in its ring slot and goes on issuing copies; the slot is free again once the chunk is copied out.
-    if (via_drainer && !r->drainer) {
-        try {
-            r->drainer.reset(new Drainer(r->pool.get()));
-        } catch (const std::exception& e) {
-            set_error("cannot start the host copy thread: %s", e.what());
-            return DR_ERR_NOMEM;
-        }
-    }
-    const uint64_t drained0 = via_drainer ? r->drainer->completed() : 0;
+    // A pageable arena is filled by the drainer's worker threads: the pump hands them a chunk as soon as the chunk
+    // has arrived in its ring slot and goes on issuing copies; the slot is free again once the chunk is copied out.
+    if (via_drainer && (rc = ensure_drainer(r, g.slots))) return rc;
     uint64_t handed = 0;  // chunks given to the drainer by this call
 
     // wait for chunk k and hand it to the sink
@@ -343,9 +357,9 @@ extern "C" int dr_stage_out(dr_plan* plan, const dr_stage_desc* d, dr_stage_stat
                     parts[np++] = Drainer::Part{(char*)d->host_arena + g.host_at[b] + (a - g.prefix[b]), slot_ptr(k) + (a - lo),
                                                 e - a};
             }
-            r->drainer->submit(parts, np);  // possibly empty (a chunk of relay bytes only): keeps the count in step
+            r->drainer->submit(parts, np, &r->pending[s]);  // possibly nothing to copy (a chunk of relay bytes only)
             ++handed;
-            return DR_OK;  // counted as done once the drainer has copied it out
+            return DR_OK;  // counted as done once the workers have copied it out
         }
         st.bytes += n;
         return DR_OK;
@@ -361,26 +375,27 @@ extern "C" int dr_stage_out(dr_plan* plan, const dr_stage_desc* d, dr_stage_stat
         }
     } else {
         uint64_t out = first;  // chunks below this index rest in the arena; their slots are free
-        auto refresh = [&] {
-            const uint64_t now = first + (r->drainer->completed() - drained0);
-            for (; out < now; ++out) st.bytes += chunk_bytes_of(out);
+        auto refresh = [&] {   // chunks leave in order: chunk `out` is out once it was handed over and its tasks are done
+            while (out < first + handed && r->pending[out % g.slots].load(std::memory_order_acquire) == 0)
+                st.bytes += chunk_bytes_of(out++);
             st.chunks_done = out;
         };
         while (rc == DR_OK && out < g.n_chunks) {
             refresh();
             while (rc == DR_OK && next_issue < g.n_chunks && next_issue - out < g.slots) rc = issue(next_issue++);
-            if (rc != DR_OK) break;
+            if (rc != DR_OK || out >= g.n_chunks) break;
             if (next_done < next_issue) {
                 if ((rc = complete(next_done)) == DR_OK) ++next_done;
-            } else if (out < g.n_chunks) {  // every issued chunk is with the drainer: wait for a slot to come back
-                if (!r->drainer->wait_completed(drained0 + (out - first) + 1, Clock::now() + limit)) {
+            } else {  // every issued chunk is with the workers: wait for the oldest slot to come back
+                if (!r->drainer->wait_zero(&r->pending[out % g.slots], Clock::now() + limit)) {
                     set_error("staging wait timed out (host copy)");
                     rc = DR_ERR_TIMEOUT;
                 }
             }
         }
         // whatever happened, no host copy of this call may still be running when it returns
-        r->drainer->wait_completed(drained0 + handed, Clock::now() + std::chrono::seconds(60));
+        for (uint64_t k = out; k < first + handed; ++k)
+            r->drainer->wait_zero(&r->pending[k % g.slots], Clock::now() + std::chrono::seconds(60));
         refresh();
     }
     if (rc) drain(r);
@@ -412,7 +427,7 @@ extern "C" int dr_stage_in(dr_plan* plan, const dr_stage_desc* d, dr_stage_stats
     }
     std::lock_guard<std::mutex> lock(plan->stage_mu);
     const bool direct = !d->callback && is_pinned_host(d->host_arena);
-    if ((rc = ensure_ring(plan, g, !direct))) return rc;
+    if ((rc = ensure_ring(plan, g, !direct, d->budget_bytes))) return rc;
     Ring* r = plan->ring;
     const auto t0 = Clock::now();
     const auto limit = std::chrono::milliseconds(d->timeout_ms ? d->timeout_ms : 60000);
@@ -451,9 +466,7 @@ extern "C" int dr_stage_in(dr_plan* plan, const dr_stage_desc* d, dr_stage_stats
                     set_error("chunk callback failed at piece %llu", (unsigned long long)i);
                     return DR_ERR_SINK;
                 }
-            } else {
-                r->pool->copy(slot, (const char*)d->host_arena + at, pc.n);
-            }
+            }  // (a pageable arena does not come here: its slots are filled by the worker threads, see below)
             host = slot;
         }
         DR_CUDA(cudaMemcpyAsync((char*)d->dev_ptr[pc.buf] + pc.pos, host, pc.n, cudaMemcpyHostToDevice, r->s_copy));
@@ -470,9 +483,58 @@ extern "C" int dr_stage_in(dr_plan* plan, const dr_stage_desc* d, dr_stage_stats
     };
 
     uint64_t next_issue = st.chunks_done, next_done = st.chunks_done;
-    while (rc == DR_OK && next_done < pieces.size()) {
-        if (next_issue < pieces.size() && next_issue - next_done < g.slots) rc = issue(next_issue++);
-        else if ((rc = complete(next_done)) == DR_OK) st.chunks_done = ++next_done;
+    const bool via_filler = !direct && !d->callback;  // pageable arena: worker threads fill the ring slots
+    if (!via_filler) {
+        while (rc == DR_OK && next_done < pieces.size()) {
+            if (next_issue < pieces.size() && next_issue - next_done < g.slots) rc = issue(next_issue++);
+            else if ((rc = complete(next_done)) == DR_OK) st.chunks_done = ++next_done;
+        }
+    } else if ((rc = ensure_drainer(r, g.slots)) == DR_OK) {
+        // Three cursors: pieces below next_fill have been given to the workers (pageable arena -> ring slot), pieces
+        // below next_issue are on their way to the device, pieces below next_done have arrived.  A slot is refilled
+        // once its previous piece has arrived.  A small ring is filled with ordinary stores, so that the device can
+        // read it from the last-level cache; a large one with non-temporal stores.
+        const bool cached = g.chunk * g.slots <= kCachedRingBytes;
+        uint64_t next_fill = next_issue;
+        auto fill = [&](uint64_t i) {
+            const Piece& pc = pieces[i];
+            const uint32_t s = (uint32_t)(i % g.slots);
+            Drainer::Part part{r->base + (uint64_t)s * g.chunk, (const char*)d->host_arena + g.host_at[pc.buf] + pc.pos, pc.n, cached};
+            r->drainer->submit(&part, 1, &r->pending[s]);
+        };
+        auto send = [&](uint64_t i) -> int {
+            const Piece& pc = pieces[i];
+            const uint32_t s = (uint32_t)(i % g.slots);
+            DR_CUDA(cudaMemcpyAsync((char*)d->dev_ptr[pc.buf] + pc.pos, r->base + (uint64_t)s * g.chunk, pc.n,
+                                    cudaMemcpyHostToDevice, r->s_copy));
+            DR_CUDA(cudaEventRecord(r->ev_copy[s], r->s_copy));
+            if (pc.last && d->ready_events[pc.buf])
+                DR_CUDA(cudaEventRecord((cudaEvent_t)d->ready_events[pc.buf], r->s_copy));
+            return DR_OK;
+        };
+        while (rc == DR_OK && next_done < pieces.size()) {
+            // retire arrivals without blocking, so that their slots can be refilled at once
+            while (next_done < next_issue && cudaEventQuery(r->ev_copy[next_done % g.slots]) == cudaSuccess) {
+                st.bytes += pieces[next_done].n;
+                if (pieces[next_done].last) st.ready_ms[pieces[next_done].buf] = ms_since(t0);
+                st.chunks_done = ++next_done;
+            }
+            while (next_fill < pieces.size() && next_fill - next_done < g.slots) fill(next_fill++);
+            while (rc == DR_OK && next_issue < next_fill &&
+                   r->pending[next_issue % g.slots].load(std::memory_order_acquire) == 0)
+                rc = send(next_issue++);
+            if (rc != DR_OK || next_done >= pieces.size()) break;
+            if (next_issue < next_fill) {  // a fill is under way: it ends within milliseconds
+                if (!r->drainer->wait_zero(&r->pending[next_issue % g.slots], Clock::now() + limit)) {
+                    set_error("staging wait timed out (host copy)");
+                    rc = DR_ERR_TIMEOUT;
+                }
+            } else if ((rc = complete(next_done)) == DR_OK) {
+                st.chunks_done = ++next_done;
+            }
+        }
+        for (uint64_t k = next_issue; k < next_fill; ++k)  // no host copy of this call may outlive it
+            r->drainer->wait_zero(&r->pending[k % g.slots], Clock::now() + std::chrono::seconds(60));
     }
     if (rc) drain(r);
     if (d->done_event) cudaEventRecord((cudaEvent_t)d->done_event, r->s_copy);
