@@ -525,9 +525,10 @@ int dr_probe_stream(uint32_t mode, const void* a_dev, void* b_dev, uint64_t n_by
 
 /*
  * dr_host_copy -- measurement aid (the paper has no counterpart): the multi-threaded host copy that the
- * staging engine uses between its pinned ring and a pageable arena, run on its own, so that a benchmark
- * can state what the host's cores sustain without the link (the CPU baseline of staging through pageable
- * memory).  threads = 0 takes the engine's own count (at most 16).  Blocking.  DR_ERR_INVALID on NULL.
+ * staging engine uses between its pinned ring and a pageable arena (worker threads taking 1 MiB tasks,
+ * non-temporal stores), run on its own, so that a benchmark can state what the host's cores sustain
+ * without the link (the CPU baseline of staging through pageable memory).  threads = 0 takes the
+ * engine's own count (at most 16).  Blocking.  DR_ERR_INVALID on NULL.
  */
 int dr_host_copy(void* dst_host, const void* src_host, uint64_t n_bytes, uint32_t threads);
 

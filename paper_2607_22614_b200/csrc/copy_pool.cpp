@@ -56,69 +56,6 @@ void copy_bytes(char* dst, const char* src, uint64_t n)
 
 }  // namespace
 
-CopyPool::CopyPool(unsigned n) : n_(n ? n : 1)
-{
-    for (unsigned i = 1; i < n_; ++i) th_.emplace_back([this, i] { loop(i); });
-}
-
-CopyPool::~CopyPool()
-{
-    {
-        std::lock_guard<std::mutex> l(mu_);
-        stop_ = true;
-        ++gen_;
-    }
-    cv_.notify_all();
-    for (auto& t : th_) t.join();
-}
-
-void CopyPool::copy(void* dst, const void* src, uint64_t n)
-{
-    if (n_ == 1 || n < (1u << 20)) {
-        copy_bytes((char*)dst, (const char*)src, n);
-        return;
-    }
-    {
-        std::lock_guard<std::mutex> l(mu_);
-        dst_ = (char*)dst;
-        src_ = (const char*)src;
-        len_ = n;
-        pending_ = n_ - 1;
-        ++gen_;
-    }
-    cv_.notify_all();
-    part(0);
-    std::unique_lock<std::mutex> l(mu_);
-    done_.wait(l, [this] { return pending_ == 0; });
-}
-
-void CopyPool::part(unsigned i)
-{
-    uint64_t per = (len_ / n_ + 4095) / 4096 * 4096;
-    uint64_t a = std::min<uint64_t>(len_, per * i), b = std::min<uint64_t>(len_, a + per);
-    if (i == n_ - 1) b = len_;
-    if (b > a) copy_bytes(dst_ + a, src_ + a, b - a);
-}
-
-void CopyPool::loop(unsigned i)
-{
-    uint64_t seen = 0;
-    for (;;) {
-        {
-            std::unique_lock<std::mutex> l(mu_);
-            cv_.wait(l, [&] { return gen_ != seen; });
-            seen = gen_;
-            if (stop_) return;
-        }
-        part(i);
-        {
-            std::lock_guard<std::mutex> l(mu_);
-            --pending_;
-        }
-        done_.notify_one();
-    }
-}
-
 Drainer::Drainer(unsigned n_threads)
 {
     for (unsigned i = 0; i < (n_threads ? n_threads : 1); ++i) th_.emplace_back([this] { loop(); });

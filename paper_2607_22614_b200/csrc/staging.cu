@@ -550,9 +550,13 @@ extern "C" int dr_host_copy(void* dst_host, const void* src_host, uint64_t n_byt
         set_error("NULL host pointer");
         return DR_ERR_INVALID;
     }
-    try {
-        CopyPool pool(threads ? threads : default_copy_threads());
-        pool.copy(dst_host, src_host, n_bytes);
+    try {  // the engine's own workers and task size, on one copy
+        Drainer workers(threads ? threads : default_copy_threads());
+        std::atomic<uint32_t> pending{0};
+        Drainer::Part part{(char*)dst_host, (const char*)src_host, n_bytes, false};
+        workers.submit(&part, 1, &pending);
+        while (!workers.wait_zero(&pending, Clock::now() + std::chrono::seconds(60))) {
+        }
     } catch (const std::exception& e) {
         set_error("cannot start the host copy threads: %s", e.what());
         return DR_ERR_NOMEM;

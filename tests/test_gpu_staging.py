@@ -328,6 +328,32 @@ def test_ranks_that_stay_relay_what_they_hold_and_rest_the_remainder_in_one_call
             assert np.array_equal(new_bufs[i][k].cpu().numpy().view(np.uint32), want[k][i]), (i, k)
 
 
+@pytest.mark.parametrize("chunk,slots", [(2_500_001, 3), (1 << 20, 5), (32 << 20, 3), (7 << 20, 8)])
+def test_pageable_arena_with_chunks_of_several_host_copy_tasks(plan, chunk, slots):
+    """Chunks larger than the 1 MiB host-copy task, of odd sizes, straddling buffers: the worker threads behind
+    the pump cut them into tasks.  Rings of at most 64 MiB are filled with ordinary stores on the way in, larger
+    ones (the 3 x 32 MiB case) with non-temporal stores.  The image is the oracle's concatenation and stage-in
+    (v first) restores every byte."""
+    sizes = [50_000_003, 4_099, 71_000_001]
+    host = [synth.fill_f32(61 + i, synth.BUF_ADAM_M, 0, -(-n // 4)).view(np.uint8)[:n].copy() for i, n in enumerate(sizes)]
+    devs = [torch.from_numpy(h).to(dev()) for h in host]
+    total = sum(sizes)
+    image = np.full(total + 64, 0x5A, dtype=np.uint8)
+    d = dr.stage_desc([t.data_ptr() for t in devs], sizes, budget=chunk * slots, chunk=chunk, host_arena=image.ctypes.data,
+                      host_arena_bytes=total)
+    st = plan.stage_out(d)
+    assert st.n_chunks == st.chunks_done == -(-total // chunk) and st.bytes == total
+    assert st.pinned_high_water_bytes == chunk * slots
+    assert np.array_equal(image[:total], np.concatenate(host)) and (image[total:] == 0x5A).all()
+    back = [torch.zeros_like(t) for t in devs]
+    d = dr.stage_desc([t.data_ptr() for t in back], sizes, budget=chunk * slots, chunk=chunk, host_arena=image.ctypes.data,
+                      host_arena_bytes=total, order=[2, 0, 1])
+    st = plan.stage_in(d)
+    assert st.chunks_done == st.n_chunks == sum(-(-n // chunk) for n in sizes) and st.bytes == total
+    assert all(torch.equal(a, b) for a, b in zip(back, devs))
+    assert 0 < st.ready_ms[2] <= st.ready_ms[0] <= st.ready_ms[1]
+
+
 def test_host_offset_errors(plan):
     t = torch.zeros(2048, dtype=torch.int32, device=dev())
     host = np.zeros(16384, dtype=np.uint8)

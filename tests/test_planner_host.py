@@ -158,6 +158,20 @@ def test_error_codes():
     assert dr.dr_plan_destroy(None) == 0
 
 
+def test_host_copy_workers_copy_every_byte():
+    """The staging engine's host-copy workers (1 MiB tasks taken by several threads), run on their own through
+    dr_host_copy: odd sizes, sizes below and above one task, one and many threads, unaligned ends."""
+    rng = np.random.default_rng(0)
+    for n, threads in ((0, 2), (1, 1), (4097, 3), ((1 << 20) - 1, 2), ((1 << 20) + 1, 16), (5 * (1 << 20) + 12345, 4), (33_333_333, 0)):
+        src = rng.integers(0, 256, size=n + 64, dtype=np.uint64).astype(np.uint8)
+        dst = np.full(n + 128, 0x5A, dtype=np.uint8)
+        rc = dr.dr_host_copy(dst.ctypes.data + 31, src.ctypes.data + 7, n, threads)
+        assert rc == 0
+        assert np.array_equal(dst[31:31 + n], src[7:7 + n])
+        assert (dst[:31] == 0x5A).all() and (dst[31 + n:] == 0x5A).all()
+    assert dr.dr_host_copy(None, 4096, 16, 1) == dr.binding.DR_ERR_INVALID
+
+
 def test_shard_range():
     assert dr.dr_shard_range(1000, 6, 0) == (0, 0, 167, 167)
     assert dr.dr_shard_range(1000, 6, 5) == (0, 835, 1000, 167)      # last shard holds 165 real elements
