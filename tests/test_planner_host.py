@@ -113,6 +113,44 @@ def test_full_size_plans_match_quoted_sizes():
         p.close()
 
 
+def test_plans_far_larger_than_the_workloads_keep_64_bit_arithmetic_and_segment_limits():
+    """A 70B-class dense shape (6.9e10 elements) and a 235B-class MoE shape (2.3e11 elements): element counts
+    equal the closed form, every segment stays inside the buffers and below the per-segment unit limit, and
+    sampled elements agree with the oracle's map.  Host only: nothing is allocated."""
+    shapes = [dict(n_layers=80, hidden=8192, n_q_heads=64, n_kv_heads=8, head_dim=128, ffn=28672, vocab=128256,
+                   n_experts=0, moe_ffn=0, tied=0, qk_norm=0),
+              dict(n_layers=94, hidden=4096, n_q_heads=64, n_kv_heads=4, head_dim=128, ffn=0, vocab=151936,
+                   n_experts=128, moe_ffn=1536, tied=0, qk_norm=1)]
+    for spec, T in zip(shapes, (8, 4)):
+        H, hd, nq, nkv, V, L = (spec[k] for k in ("hidden", "head_dim", "n_q_heads", "n_kv_heads", "vocab", "n_layers"))
+        mlp = 3 * H * spec["ffn"] if not spec["n_experts"] else spec["n_experts"] * H + 3 * spec["n_experts"] * H * spec["moe_ffn"]
+        closed = 2 * V * H + L * (2 * H + 2 * hd * spec["qk_norm"] + 2 * H * nq * hd + 2 * H * nkv * hd + mlp) + H
+        p = dr.Plan(spec, world=16, rank=5, gathered=True, tp=T, tp_rank=T - 1, host_only=True)
+        assert p.info.flat_elems == closed > (1 << 36)
+        om = oracle.Model(spec, world=16, tp=T, tp_rank=T - 1)
+        assert p.info.dst_bytes == om.arena_bytes and p.info.src_bytes == 4 * 16 * om.shard_elems
+        segs = p.segments()
+        n_src = p.info.src_bytes // 4
+        assert sum(s.rows * s.row_len for s in segs) == p.info.elems_moved
+        for s in segs:
+            assert s.src_off + (s.rows - 1) * s.src_row_stride + s.row_len <= n_src
+            assert s.dst_off + ((s.rows - 1) * s.dst_row_stride + s.row_len) * 2 <= p.info.dst_bytes
+            assert s.rows * -(-s.row_len // 8) < (1 << 32)
+        dst = om.dst_tensors()
+        starts = np.array([d.arena_off if d.alias_of < 0 else -1 for d in dst])
+        own = np.flatnonzero(starts >= 0)
+        rng = np.random.default_rng(2)
+        for s in [segs[i] for i in rng.integers(0, len(segs), size=40)] + [segs[0], segs[-1]]:
+            for _ in range(5):
+                i, j = int(rng.integers(0, s.rows)), int(rng.integers(0, s.row_len))
+                byte = s.dst_off + (i * s.dst_row_stride + j) * 2
+                ti = int(own[np.searchsorted(starts[own], byte, side="right") - 1])
+                d = dst[ti]
+                slot = (byte - d.arena_off) // 2
+                assert om.map(ti, slot // d.cols, slot % d.cols) == s.src_off + i * s.src_row_stride + j
+        p.close()
+
+
 def test_library_exports_every_declared_symbol():
     header = open(os.path.join(ROOT, "include", "dynaresize.h")).read()
     declared = set(re.findall(r"\b(dr_[a-z_]+)\s*\(", header)) - {"dr_chunk_fn"}
