@@ -75,3 +75,47 @@ def test_push_into_one_arena_is_dr_reshard_and_argument_errors():
     assert torch.equal(a, b)
     for p in (plan, q, host):
         p.close()
+
+
+def test_push_into_an_arena_owned_by_another_process():
+    """Two processes on this GPU play FSDP ranks 0 and 1.  Rank 0 (this process) owns a rollout arena and hands it
+    to rank 1 through CUDA IPC; rank 1 repacks its shard and pushes the pieces into that arena, which it reaches
+    only through the IPC mapping, as it would reach a peer GPU's arena.  The processes are ordered on the host
+    (rank 1 synchronises and reports before rank 0 reads), no kernel waits for another.  After rank 0's own push the
+    arena must equal the oracle's gathered forward."""
+    import torch.multiprocessing as mp
+
+    import synth
+    from push_peer_worker import run
+
+    spec, W, T, t, seed = MID[0]["spec"], 2, 2, 1, 4242
+    om = oracle.Model(spec, world=W, tp=T, tp_rank=t)
+    S = om.shard_elems
+    arena = torch.full((om.arena_bytes,), SENT8, dtype=torch.uint8, device=dev())
+    torch.cuda.synchronize()
+    ctx = mp.get_context("spawn")
+    q = ctx.Queue()
+    child = ctx.Process(target=run, args=(arena, spec, W, T, t, seed, q))
+    child.start()
+    try:
+        status, n_ranges, digest = q.get(timeout=300)
+    finally:
+        child.join(timeout=60)
+        if child.is_alive():
+            child.kill()
+    assert status == "ok", n_ranges
+    # what rank 1 left in this process's memory: exactly its plan's ranges, everything else still sentinel
+    flat = synth.fill_f32(seed, synth.BUF_MASTER, 0, W * S)
+    after_one = np.full(om.arena_bytes, SENT8, dtype=np.uint8)
+    om.forward(flat[S:2 * S].copy(), after_one, gathered=False, rank=1)
+    assert first_diff(arena.cpu().numpy(), after_one) is None
+    assert digest == int(after_one.astype(np.int64).sum()) and n_ranges > 0
+    plan = dr.Plan(spec, world=W, rank=0, gathered=False, tp=T, tp_rank=t)
+    plan.reshard_push(torch.from_numpy(flat[:S].copy().view(np.int32)).to(dev()), [arena])
+    torch.cuda.synchronize()
+    want = np.full(om.arena_bytes, SENT8, dtype=np.uint8)
+    om.forward(flat, want, gathered=True)
+    assert first_diff(arena.cpu().numpy(), want) is None
+    plan.close()
+    del arena
+    torch.cuda.ipc_collect()
