@@ -486,8 +486,11 @@ extern "C" int dr_stage_in(dr_plan* plan, const dr_stage_desc* d, dr_stage_stats
     const bool via_filler = !direct && !d->callback;  // pageable arena: worker threads fill the ring slots
     if (!via_filler) {
         while (rc == DR_OK && next_done < pieces.size()) {
-            if (next_issue < pieces.size() && next_issue - next_done < g.slots) rc = issue(next_issue++);
-            else if ((rc = complete(next_done)) == DR_OK) st.chunks_done = ++next_done;
+            if (next_issue < pieces.size() && next_issue - next_done < g.slots) {
+                if ((rc = issue(next_issue)) == DR_OK) ++next_issue;  // a piece whose source failed was not issued
+            } else if ((rc = complete(next_done)) == DR_OK) {
+                st.chunks_done = ++next_done;
+            }
         }
     } else if ((rc = ensure_drainer(r, g.slots)) == DR_OK) {
         // Three cursors: pieces below next_fill have been given to the workers (pageable arena -> ring slot), pieces
@@ -522,7 +525,7 @@ extern "C" int dr_stage_in(dr_plan* plan, const dr_stage_desc* d, dr_stage_stats
             while (next_fill < pieces.size() && next_fill - next_done < g.slots) fill(next_fill++);
             while (rc == DR_OK && next_issue < next_fill &&
                    r->pending[next_issue % g.slots].load(std::memory_order_acquire) == 0)
-                rc = send(next_issue++);
+                if ((rc = send(next_issue)) == DR_OK) ++next_issue;
             if (rc != DR_OK || next_done >= pieces.size()) break;
             if (next_issue < next_fill) {  // a fill is under way: it ends within milliseconds
                 if (!r->drainer->wait_zero(&r->pending[next_issue % g.slots], Clock::now() + limit)) {
@@ -536,7 +539,15 @@ extern "C" int dr_stage_in(dr_plan* plan, const dr_stage_desc* d, dr_stage_stats
         for (uint64_t k = next_issue; k < next_fill; ++k)  // no host copy of this call may outlive it
             r->drainer->wait_zero(&r->pending[k % g.slots], Clock::now() + std::chrono::seconds(60));
     }
-    if (rc) drain(r);
+    if (rc) {
+        drain(r);
+        // pieces that were on their way when the call failed have landed during the drain: they count as done
+        while (next_done < next_issue && cudaEventQuery(r->ev_copy[next_done % g.slots]) == cudaSuccess) {
+            st.bytes += pieces[next_done].n;
+            if (pieces[next_done].last) st.ready_ms[pieces[next_done].buf] = ms_since(t0);
+            st.chunks_done = ++next_done;
+        }
+    }
     if (d->done_event) cudaEventRecord((cudaEvent_t)d->done_event, r->s_copy);
     st.elapsed_ms = ms_since(t0);
     st.link_gbs = st.elapsed_ms > 0 ? (double)st.bytes / st.elapsed_ms * 1e-6 : 0;

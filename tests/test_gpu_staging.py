@@ -127,6 +127,43 @@ def test_callback_sink_failure_and_resume(plan):
     assert [b for b, _, _ in walk][:16] == [2] * 16      # 250 001 bytes of buffer 2 = 16 pieces, before anything else
 
 
+def test_stage_in_failure_reports_the_pieces_done_and_resumes_from_there(plan):
+    """A source callback that fails at piece 6: the call stops with DR_ERR_SINK, reports six pieces done (those are
+    on the device, byte-exact), and a second call with first_chunk = 6 asks for exactly the remaining pieces of the
+    oracle's walk and completes the state."""
+    sizes = [70_001, 30_000, 55_555]
+    rng = np.random.default_rng(9)
+    host = [rng.integers(0, 256, size=n, dtype=np.uint64).astype(np.uint8) for n in sizes]
+    stream = np.concatenate(host)
+    prefix = np.concatenate([[0], np.cumsum(sizes)])
+    order, chunk = [1, 2, 0], 16 * 1024
+    asked, fail_at = [], [6]
+
+    @dr.dr_chunk_fn
+    def source(user, k, off, ptr, n):
+        if k == fail_at[0]:
+            return 7
+        asked.append((k, off, n))
+        C.memmove(ptr, stream.ctypes.data + off, n)
+        return 0
+
+    back = [torch.full((n,), 0xEE, dtype=torch.uint8, device=dev()) for n in sizes]
+    d = dr.stage_desc([t.data_ptr() for t in back], sizes, budget=4 * chunk, chunk=chunk, callback=source, order=order)
+    rc, st = dr.dr_stage_in(plan.handle, d)
+    assert rc == B.DR_ERR_SINK and st.chunks_done == 6 and "piece 6" in dr.dr_last_error()
+    ob = [np.zeros(n, dtype=np.uint8) for n in sizes]
+    n_pieces, _, walk = oracle.stage_in(ob, stream, 4 * chunk, chunk, order=order, pieces=True)
+    torch.cuda.synchronize()
+    for b, pos, nb in walk[:6]:                       # what was reported done is there
+        assert np.array_equal(back[b][pos:pos + nb].cpu().numpy(), host[b][pos:pos + nb])
+    fail_at[0] = -1
+    d.first_chunk = st.chunks_done
+    rc, st2 = dr.dr_stage_in(plan.handle, d)
+    assert rc == 0 and st2.chunks_done == st2.n_chunks == n_pieces
+    assert asked == [(i, int(prefix[b]) + pos, nb) for i, (b, pos, nb) in enumerate(walk)]
+    assert all(np.array_equal(t.cpu().numpy(), h) for t, h in zip(back, host))
+
+
 def test_relay_sink_moves_state_to_other_device_buffers(plan):
     S = 1_000_003
     host, devs = _state(S, 11, bufs=(0, 1))
