@@ -550,8 +550,10 @@ def main():
                 "write_gbs": best(lambda: probe(dr.binding.DR_PROBE_WRITE, None, ap, nb), nb),
                 "copy_1to1_gbs": best(lambda: probe(dr.binding.DR_PROBE_COPY, mp, ap, nb), 2 * nb),
                 "narrow_2to1_gbs": best(lambda: probe(dr.binding.DR_PROBE_NARROW, mp, ap, nb), nb * 3 // 2)}
+        ceil["narrow_4to1_gbs"] = best(lambda: probe(dr.binding.DR_PROBE_NARROW4, mp, ap, nb), nb * 5 // 4)
         if flat_back is not None:
             ceil["widen_1to2_gbs"] = best(lambda: probe(dr.binding.DR_PROBE_WIDEN, ap, flat_back.data_ptr(), nb), nb * 3 // 2)
+            ceil["widen_1to4_gbs"] = best(lambda: probe(dr.binding.DR_PROBE_WIDEN4, ap, flat_back.data_ptr(), nb), nb * 5 // 4)
         w = min(n_src, 1 << 30)
         ceil["torch_read_sum_gbs"] = best(lambda: master.view(torch.float32)[:w].sum(), 4 * w, reps=3)
         if info.dst_bytes >= 2 * w:
@@ -589,6 +591,9 @@ def main():
                                "gbs_best": qb / min(qms) / 1e6, "ms_avg": qavg, "ms_best": min(qms),
                                "frac_of_measured_peak": qb / qavg / 1e6 / peak, "frac_of_nominal_8000": qb / qavg / 1e6 / 8000.0,
                                "algorithmic_bytes_per_quant_elem": 5}
+        c41 = line.get("context_ceilings", {}).get("narrow_4to1_gbs")
+        if c41:
+            line["fp8_forward"].update({"same_run_ceiling_for_this_mix": c41, "frac_of_same_run_ceiling": qb / qavg / 1e6 / c41})
         # and back: value(code) * scale to the flat fp32 positions (bf16 tensors widened), where a second flat buffer fits
         free_q, _ = torch.cuda.mem_get_info()
         if free_q > info.src_bytes * 1.05:
@@ -609,6 +614,9 @@ def main():
                                    "bytes": int(ib), "gbs_avg": ib / iavg / 1e6, "gbs_best": ib / min(ims) / 1e6, "ms_avg": iavg,
                                    "ms_best": min(ims), "frac_of_measured_peak": ib / iavg / 1e6 / peak,
                                    "frac_of_nominal_8000": ib / iavg / 1e6 / 8000.0, "first_quantised_tensor": t1.name.decode()}
+            c14 = line.get("context_ceilings", {}).get("widen_1to4_gbs")
+            if c14:
+                line["fp8_inverse"].update({"same_run_ceiling_for_this_mix": c14, "frac_of_same_run_ceiling": ib / iavg / 1e6 / c14})
             del qflat
         qplan.close()
         del qarena

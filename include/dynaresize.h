@@ -518,9 +518,12 @@ int dr_ctl_destroy(dr_ctl* ctl);
  *   DR_PROBE_COPY   copies n_bytes a_dev -> b_dev                (1 : 1)
  *   DR_PROBE_NARROW reads n_bytes of fp32, writes n_bytes / 2 of bf16 (2 : 1, the forward repack's mix)
  *   DR_PROBE_WIDEN  reads n_bytes / 2 of bf16, writes n_bytes of fp32 (1 : 2, the inverse map's mix)
+ *   DR_PROBE_NARROW4 reads n_bytes, writes n_bytes / 4                (4 : 1, the fp8 forward's mix)
+ *   DR_PROBE_WIDEN4  reads n_bytes / 4, writes n_bytes                (1 : 4, the fp8 inverse's mix)
  * Asynchronous on cuda_stream.  Errors: DR_ERR_INVALID, DR_ERR_ALIGN, DR_ERR_UNSUPPORTED, DR_ERR_CUDA.
  */
-enum { DR_PROBE_READ = 0, DR_PROBE_WRITE = 1, DR_PROBE_COPY = 2, DR_PROBE_NARROW = 3, DR_PROBE_WIDEN = 4 };
+enum { DR_PROBE_READ = 0, DR_PROBE_WRITE = 1, DR_PROBE_COPY = 2, DR_PROBE_NARROW = 3, DR_PROBE_WIDEN = 4,
+       DR_PROBE_NARROW4 = 5, DR_PROBE_WIDEN4 = 6 };
 int dr_probe_stream(uint32_t mode, const void* a_dev, void* b_dev, uint64_t n_bytes, void* cuda_stream);
 
 /*

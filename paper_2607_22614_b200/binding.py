@@ -314,7 +314,7 @@ def dr_reshard_stream(plan, desc):
     return lib().dr_reshard_stream(plan, C.byref(desc), C.byref(st)), st
 
 
-DR_PROBE_READ, DR_PROBE_WRITE, DR_PROBE_COPY, DR_PROBE_NARROW, DR_PROBE_WIDEN = range(5)
+DR_PROBE_READ, DR_PROBE_WRITE, DR_PROBE_COPY, DR_PROBE_NARROW, DR_PROBE_WIDEN, DR_PROBE_NARROW4, DR_PROBE_WIDEN4 = range(7)
 
 
 def dr_probe_stream(mode, a_dev, b_dev, n_bytes, cuda_stream):

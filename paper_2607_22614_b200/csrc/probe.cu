@@ -88,6 +88,31 @@ __global__ void __launch_bounds__(kT) probe_kernel(const char* __restrict__ a, c
                     : "f"(__uint_as_float(v[j].w[2 * i + 1])), "f"(__uint_as_float(v[j].w[2 * i])));
             st128(b + (u0 + j * kT) * 16, o);
         }
+    } else if (MODE == DR_PROBE_NARROW4) {  // 32 bytes in, 8 bytes out per unit (the fp8 forward's mix)
+        W8 v[kU];
+#pragma unroll
+        for (int j = 0; j < kU; ++j) v[j] = ld256(a + (u0 + j * kT) * 32);
+#pragma unroll
+        for (int j = 0; j < kU; ++j) {
+            const uint32_t lo = (v[j].w[0] & 0xFF) | ((v[j].w[1] & 0xFF) << 8) | ((v[j].w[2] & 0xFF) << 16) | (v[j].w[3] << 24);
+            const uint32_t hi = (v[j].w[4] & 0xFF) | ((v[j].w[5] & 0xFF) << 8) | ((v[j].w[6] & 0xFF) << 16) | (v[j].w[7] << 24);
+            asm volatile("st.global.L1::no_allocate.v2.b32 [%0], {%1,%2};" ::"l"(b + (u0 + j * kT) * 8), "r"(lo), "r"(hi) : "memory");
+        }
+    } else if (MODE == DR_PROBE_WIDEN4) {  // 8 bytes in, 32 bytes out per unit (the fp8 inverse's mix)
+        uint32_t lo[kU], hi[kU];
+#pragma unroll
+        for (int j = 0; j < kU; ++j)
+            asm volatile("ld.global.nc.L1::no_allocate.v2.b32 {%0,%1}, [%2];" : "=r"(lo[j]), "=r"(hi[j]) : "l"(a + (u0 + j * kT) * 8));
+#pragma unroll
+        for (int j = 0; j < kU; ++j) {
+            W8 o;
+#pragma unroll
+            for (int i = 0; i < 4; ++i) {
+                o.w[i] = (lo[j] >> (8 * i)) << 23;
+                o.w[4 + i] = (hi[j] >> (8 * i)) << 23;
+            }
+            st256(b + (u0 + j * kT) * 32, o);
+        }
     } else {  // DR_PROBE_WIDEN
         W4 v[kU];
 #pragma unroll
@@ -112,7 +137,7 @@ extern "C" int dr_probe_stream(uint32_t mode, const void* a_dev, void* b_dev, ui
 {
     using namespace dr;
     const uint64_t tile = (uint64_t)kT * kU * 32;  // bytes of the wider side per CTA
-    if (mode > DR_PROBE_WIDEN || n_bytes == 0 || n_bytes % tile || (mode != DR_PROBE_WRITE && !a_dev) ||
+    if (mode > DR_PROBE_WIDEN4 || n_bytes == 0 || n_bytes % tile || (mode != DR_PROBE_WRITE && !a_dev) ||
         (mode != DR_PROBE_READ && !b_dev)) {
         set_error("dr_probe_stream: bad mode, NULL buffer, or byte count not a multiple of %llu", (unsigned long long)tile);
         return DR_ERR_INVALID;
@@ -135,6 +160,8 @@ extern "C" int dr_probe_stream(uint32_t mode, const void* a_dev, void* b_dev, ui
     case DR_PROBE_WRITE: probe_kernel<DR_PROBE_WRITE><<<g, kT, 0, s>>>(a, b, nullptr); break;
     case DR_PROBE_COPY: probe_kernel<DR_PROBE_COPY><<<g, kT, 0, s>>>(a, b, nullptr); break;
     case DR_PROBE_NARROW: probe_kernel<DR_PROBE_NARROW><<<g, kT, 0, s>>>(a, b, nullptr); break;
+    case DR_PROBE_NARROW4: probe_kernel<DR_PROBE_NARROW4><<<g, kT, 0, s>>>(a, b, nullptr); break;
+    case DR_PROBE_WIDEN4: probe_kernel<DR_PROBE_WIDEN4><<<g, kT, 0, s>>>(a, b, nullptr); break;
     default: probe_kernel<DR_PROBE_WIDEN><<<g, kT, 0, s>>>(a, b, nullptr); break;
     }
     cudaError_t e = cudaGetLastError();
