@@ -145,6 +145,9 @@ typedef struct dr_plan_info {
     uint64_t quant_elems;     /* DR_FP8_E4M3_B128 plans: elements written as fp8 (counted in elems_moved) */
     uint64_t quant_blocks;    /* and the number of 128 x 128 blocks, one fp32 scale each              */
     uint64_t n_groups;        /* n_layers + 2: embed, every layer, final norm with lm_head            */
+    uint64_t bulk_forward;    /* 1: dr_reshard runs the kernel that moves tiles with the TMA unit's bulk
+                                 copies (plans with under 2 % of their elements in strided segments);
+                                 0: the kernel that moves them through registers.  Same result.       */
 } dr_plan_info;
 
 typedef struct dr_tensor_desc {
@@ -534,6 +537,15 @@ int dr_probe_stream(uint32_t mode, const void* a_dev, void* b_dev, uint64_t n_by
  * engine's own count (at most 16).  Blocking.  DR_ERR_INVALID on NULL.
  */
 int dr_host_copy(void* dst_host, const void* src_host, uint64_t n_bytes, uint32_t threads);
+
+/*
+ * dr_diag_bulk_wait_failures -- diagnostic (the paper has no counterpart).  The repack kernels move whole
+ * contiguous tiles with the TMA unit's bulk copies and wait for them on an mbarrier with an iteration
+ * limit; a wait that ran out makes the tile fall back to the register path (same result) and counts
+ * here.  *count = such events on the current device since the library was loaded; expected 0.
+ * Synchronous (reads a device counter).  DR_ERR_INVALID, DR_ERR_CUDA.
+ */
+int dr_diag_bulk_wait_failures(uint64_t* count);
 
 /* Synchronises the plan's own streams, frees its ring, table and streams.  NULL is accepted. */
 int dr_plan_destroy(dr_plan* plan);

@@ -125,6 +125,8 @@ int create(const dr_model_spec* s, const dr_src_layout* a, const dr_dst_layout* 
         if (e != cudaSuccess || p->grid <= 0) {
             set_error("plan upload: %s", cudaGetErrorString(e));
             rc = e == cudaErrorMemoryAllocation ? DR_ERR_NOMEM : DR_ERR_CUDA;
+        } else {
+            rc = ensure_bulk_smem(p->device);  // keeps its own error message
         }
     }
     if (rc) {
@@ -205,6 +207,7 @@ int dr_plan_window_host(const dr_plan* plan, uint64_t src_elem_lo, uint64_t src_
     w->tp = plan->tp;
     w->tp_rank = plan->tp_rank;
     w->elem_size = plan->elem_size;
+    w->bulk_forward = plan->bulk_forward;
     w->host_only = true;
     int rc = DR_OK;
     try {
@@ -219,6 +222,7 @@ int dr_plan_window_host(const dr_plan* plan, uint64_t src_elem_lo, uint64_t src_
             w->info = plan->info;
             w->info.src_bytes = 4 * (src_elem_hi - src_elem_lo);
             w->info.n_segments = w->segs.size();
+            w->info.bulk_forward = plan->info.bulk_forward;
             w->info.n_tiles = tb.n_tiles;
             w->info.elems_moved = tb.elems;
             w->info.bytes_moved_fwd = w->info.bytes_moved_inv = tb.elems * (4 + plan->elem_size);
@@ -413,6 +417,15 @@ int dr_plan_destroy(dr_plan* plan)
     if (plan->d_qhints) cudaFree(plan->d_qhints);
     delete plan;
     return DR_OK;
+}
+
+int dr_diag_bulk_wait_failures(uint64_t* count)
+{
+    if (!count) {
+        set_error("NULL argument");
+        return DR_ERR_INVALID;
+    }
+    return bulk_wait_failures(count);
 }
 
 const char* dr_strerror(int status)

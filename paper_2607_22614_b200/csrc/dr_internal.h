@@ -126,6 +126,9 @@ struct dr_plan {
     dr::QPart* d_qparts = nullptr;
     uint32_t* d_qhints = nullptr;
     int grid = 0;
+    // forward launches take the TMA bulk-copy kernel (see reshard.cu): set when next to none of the plan's elements
+    // sit in strided (column-sliced) segments, whose short per-row copies are slower that way than from registers
+    bool bulk_forward = false;
     // staging
     std::mutex stage_mu;
     dr::Ring* ring = nullptr;
@@ -154,6 +157,8 @@ int launch_reshard(const dr_plan* p, bool inverse, const void* flat, void* arena
 // Forward repack into several arenas at once (the fused exchange).
 int launch_push(const dr_plan* p, const void* flat, void* const* arenas, uint32_t n_dst, void* stream);
 std::vector<dr_range> plan_ranges(const dr_plan* p);  // planner.cpp: coalesced arena byte ranges the plan writes
+int ensure_bulk_smem(int device);          // once per device: lets the repack kernels ask for their tile buffers
+int bulk_wait_failures(uint64_t* out);     // bounded mbarrier waits that ran out since the library was loaded (expected: 0)
 int choose_grid(int device, uint32_t elem_size);  // resident CTAs of the reshard kernel on the whole GPU
 // Blocks [block_lo, min(block_hi, all)) of the plan's quantised tensors.
 int launch_quant(const dr_plan* p, const void* flat, void* arena, void* stream, uint64_t block_lo = 0,
@@ -165,6 +170,6 @@ int build_tables(const std::vector<HostSeg>& segs, Tables* out);
 std::vector<HostSeg> window_segments(const std::vector<HostSeg>& segs, uint64_t lo, uint64_t hi, uint32_t es);
 // Enqueue the forward kernel for an explicit table (used by the streamed repack).
 int launch_forward_tables(uint32_t elem_size, const DevSeg* d_segs, uint32_t n_segs, const uint32_t* d_hints,
-                          uint32_t hint_shift, uint64_t n_tiles, const void* flat, void* arena, void* stream);
+                          uint32_t hint_shift, uint64_t n_tiles, const void* flat, void* arena, void* stream, bool bulk);
 
 }  // namespace dr

@@ -503,6 +503,12 @@ int compile_plan(dr_plan* p)
         }
     }
 
+    {   // elements in strided segments: under 2 % of the plan, forward launches go through the bulk-copy kernel
+        uint64_t strided = 0;
+        for (const HostSeg& g : p->segs)
+            if (g.rows > 1) strided += g.rows * g.row_len;
+        p->bulk_forward = strided * 50 <= moved;
+    }
     dr_plan_info& I = p->info;
     I.flat_elems = N;
     I.shard_elems = S;
@@ -517,6 +523,7 @@ int compile_plan(dr_plan* p)
     I.n_groups = p->groups.size();
     I.quant_elems = qelems;
     I.quant_blocks = qblocks;
+    I.bulk_forward = p->bulk_forward ? 1 : 0;
 
     // Every access the kernels will make is checked here, so a launch cannot leave its buffers.
     const uint64_t src_elems = I.src_bytes / 4;

@@ -189,7 +189,7 @@ extern "C" int dr_reshard_stream(dr_plan* plan, const dr_stream_desc* d, dr_stre
             st.h2d_bytes += n;
             DR_CUDA(cudaStreamWaitEvent(s->s_kernel, s->ev_arrived[slot], 0));
             int krc = launch_forward_tables(plan->elem_size, s->d_segs + c.seg_off, c.n_segs, s->d_hints + c.hint_off,
-                                            c.hint_shift, c.n_tiles, win, d->dst_dev, s->s_kernel);
+                                            c.hint_shift, c.n_tiles, win, d->dst_dev, s->s_kernel, plan->bulk_forward);
             if (krc) return krc;
             if (c.n_tiles) ++st.kernels;
             DR_CUDA(cudaEventRecord(s->ev_done[slot], s->s_kernel));

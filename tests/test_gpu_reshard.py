@@ -45,6 +45,32 @@ def test_sixteen_byte_aligned_bases_take_the_narrow_path(misalign, dtype):
     plan.close()
 
 
+# A MoE shape whose column-sliced (strided) attention output is under 2 % of the elements: such plans run the kernel
+# that moves tiles with the TMA unit's bulk copies, strided rows and run tails included.
+MOE32 = dict(MID[2]["spec"], n_experts=32)
+
+
+@pytest.mark.parametrize("kw", [dict(tp=2, tp_rank=1), dict(tp=2, tp_rank=0, world=3, rank=1, gathered=False),
+                                dict(tp=2, tp_rank=1, align=4, dtype=dr.DR_F32), dict(tp=2, tp_rank=0, misalign=16),
+                                dict(tp=4, tp_rank=3, world=5, gathered=True, align=16)],
+                         ids=["tp2", "shard-local", "f32-align4", "base16", "tp4-w5"])
+def test_bulk_copy_kernel_with_strided_rows_tails_and_shard_cuts(kw):
+    kw = dict(kw)
+    got, want, plan, om, _ = forward_both(MOE32, seed=91, **kw)
+    assert plan.info.bulk_forward == 1
+    assert any(s.rows > 1 for s in plan.segments())          # column-sliced segments are there
+    assert first_diff(got, want) is None
+    plan.close()
+    # and the dense TP = 1 plans of the other mid-size shapes take the same kernel
+    for cfg in MID[:2]:
+        got, want, plan, _, _ = forward_both(cfg["spec"], seed=92)
+        assert plan.info.bulk_forward == 1 and first_diff(got, want) is None
+        plan.close()
+    got, want, plan, _, _ = forward_both(MID[0]["spec"], tp=2, tp_rank=1, seed=93)
+    assert plan.info.bulk_forward == 0 and first_diff(got, want) is None      # 30 % strided: the register kernel
+    plan.close()
+
+
 def test_cast_special_values_in_hardware():
     """Every hand-picked pattern (ties, carries, overflow, subnormals, NaNs) through the vector path and,
     via an odd-sized spec, through the scalar path."""

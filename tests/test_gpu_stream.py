@@ -108,3 +108,18 @@ def test_streamed_repack_is_ordered_after_pending_work_on_the_callers_stream():
     assert still_pending, "the fills finished before the call: the test did not exercise the ordering"
     assert first_diff(arena.cpu().numpy(), want) is None
     plan.close()
+
+
+def test_no_bounded_device_wait_ran_out():
+    """The repack kernels wait for their bulk copies on an mbarrier with an iteration limit and fall back to the
+    register path if the wait runs out.  After everything this process has launched so far that must never have
+    happened (a fallback would still give the right bytes, but would point at a broken pipeline)."""
+    plan = dr.Plan(MID[0]["spec"])
+    src = torch.zeros(plan.info.src_bytes // 4, dtype=torch.int32, device=dev())
+    arena = torch.zeros(plan.info.dst_bytes, dtype=torch.uint8, device=dev())
+    plan.reshard(src, arena)
+    plan.reshard_inverse(arena, src)
+    torch.cuda.synchronize()
+    rc, n = dr.dr_diag_bulk_wait_failures()
+    assert rc == 0 and n == 0
+    plan.close()

@@ -162,7 +162,7 @@ def test_library_exports_every_declared_symbol():
 
 def test_struct_sizes_match_the_header_layout():
     assert C.sizeof(dr.dr_model_spec) == 48 and C.sizeof(dr.dr_src_layout) == 28 and C.sizeof(dr.dr_dst_layout) == 36
-    assert C.sizeof(dr.dr_stage_desc) == 448 and C.sizeof(dr.dr_stream_desc) == 112 and C.sizeof(dr.dr_stage_stats) == 112 and C.sizeof(dr.dr_plan_info) == 104 and C.sizeof(dr.dr_tensor_desc) == 128 and C.sizeof(dr.dr_segment_desc) == 56
+    assert C.sizeof(dr.dr_stage_desc) == 448 and C.sizeof(dr.dr_stream_desc) == 112 and C.sizeof(dr.dr_stage_stats) == 112 and C.sizeof(dr.dr_plan_info) == 112 and C.sizeof(dr.dr_tensor_desc) == 128 and C.sizeof(dr.dr_segment_desc) == 56
 
 
 def test_error_codes():
