@@ -31,7 +31,7 @@ GiB = 1 << 30
 # DRAM bytes per element (dram__bytes_read.sum + dram__bytes_write.sum over elements moved) of the forward
 # kernel, from the committed ncu capture summary of this kernel (a 654 M-element case of the
 # same kernel; traffic grows in proportion to the elements, so it is scaled to the launch timed here).
-NCU_DRAM_BYTES_PER_ELEMENT_FWD = 5.948
+NCU_DRAM_BYTES_PER_ELEMENT_FWD = 5.951
 
 
 def load_peaks():
@@ -500,7 +500,7 @@ def main():
         "gpu_launches": args.steps * (len(plans) + (1 if do_inverse else 0)),
         "forward": {"gbs_avg": ach, "gbs_best": bytes_fwd / min(fwd_ms) / 1e6, "ms_avg": fwd_avg, "ms_best": min(fwd_ms),
                     "ms_median": median(fwd_ms), "frac_of_measured_peak": ach / peak, "frac_of_nominal_8000": ach / 8000.0},
-        "roofline": {"bound": "hbm", "kernel": "reshard_kernel<2,false> (dr_reshard)", "achieved": ach, "peak": peak,
+        "roofline": {"bound": "hbm", "kernel": "reshard_kernel<2,false> (dr_reshard), bulk-copy form" if plans[0].info.bulk_forward else "reshard_kernel<2,false> (dr_reshard), register form", "achieved": ach, "peak": peak,
                      "peak_kind": f"{peak_kind} copy bandwidth (burst)", "unit": "GB/s", "frac": ach / peak,
                      "traffic": None, "algorithmic_bytes": int(bytes_fwd // len(plans))},
     }

@@ -197,7 +197,7 @@ struct Peers {
 // A forward tile of a vector-class segment is moved by 1-D bulk asynchronous copies (cp.async.bulk: no tensor map,
 // no multicast): global -> shared memory, one copy per source row the tile touches (one in all for a contiguous
 // run), completion counted in bytes on an mbarrier; the cast runs from shared memory to shared memory; one bulk copy
-// shared -> global per destination arena (the rollout side of a segment is always dense).  On B200 this streams
+// shared -> global (the rollout side of a segment is always dense).  On B200 this streams
 // 1 % faster than 256-bit loads and stores from registers (7.17 against 7.10 TB/s on the 2 : 1 mix).  It is used for
 // the forward direction only: for the write-heavy inverse the register path is the faster one, and a kernel that
 // reserves the tile buffers (72 KB per CTA) leaves the register path too little L1 to keep its loads in flight, so
@@ -222,9 +222,9 @@ __device__ __forceinline__ bool mbar_wait_bounded(uint32_t bar, uint32_t parity)
 }
 
 // Units [ub, ub + n) of segment g, flat -> arena(s).  Returns false if the tile has to take the register path.
-template <int ES, bool PUSH>
+template <int ES>
 __device__ __forceinline__ bool bulk_forward_tile(const DevSeg& g, uint32_t ub, uint32_t n, const char* fbase, char* arena,
-                                                  const Peers& peers, char* smem, uint64_t* bar_ptr)
+                                                  char* smem, uint64_t* bar_ptr)
 {
     const bool contiguous = g.flags & kSegContiguous;
     // source pieces: piece 0 is the rest of the first row, the others are whole rows, the last may be cut short
@@ -277,14 +277,6 @@ __device__ __forceinline__ bool bulk_forward_tile(const DevSeg& g, uint32_t ub, 
         asm volatile("cp.async.bulk.global.shared::cta.bulk_group [%0], [%1], %2;" ::"l"(arena + off), "r"(out_s),
                      "r"(n * 8u * ES)
                      : "memory");
-        if (PUSH) {
-#pragma unroll
-            for (uint32_t q = 0; q < DR_MAX_PUSH_DST - 1; ++q)
-                if (q < peers.n)
-                    asm volatile("cp.async.bulk.global.shared::cta.bulk_group [%0], [%1], %2;" ::"l"(peers.a[q] + off),
-                                 "r"(out_s), "r"(n * 8u * ES)
-                                 : "memory");
-        }
         asm volatile("cp.async.bulk.commit_group;" ::: "memory");
         asm volatile("cp.async.bulk.wait_group.read 0;" ::: "memory");  // shared memory is read out before the CTA leaves
     }
@@ -332,12 +324,12 @@ __global__ void __launch_bounds__(kThreads, DR_MIN_BLOCKS)
         const bool contiguous = g.flags & kSegContiguous;
 
 #if DR_BULK
-        if (BULK && kOneTile && !INV && (g.flags & (kSegVec32 | kSegVec16))) {  // a forward tile whose rows are 16-byte aligned
+        if (BULK && kOneTile && !INV && !PUSH && (g.flags & (kSegVec32 | kSegVec16))) {  // a forward tile whose rows are 16-byte aligned
             extern __shared__ __align__(128) char bulk_smem[];
             __shared__ __align__(8) uint64_t bulk_bar;
             const uint32_t ub = (uint32_t)(tile - g.tile0) * kTileUnits;
             const uint32_t n = min(kTileUnits, g.n_units - ub);
-            if (bulk_forward_tile<ES, PUSH>(g, ub, n, fbase, arena, peers, bulk_smem, &bulk_bar)) return;
+            if (bulk_forward_tile<ES>(g, ub, n, fbase, arena, bulk_smem, &bulk_bar)) return;
         }
 #endif
 
@@ -460,8 +452,6 @@ int ensure_bulk_smem(int device)
     if (done[device]) return DR_OK;
     DR_CUDA(cudaFuncSetAttribute(reshard_kernel<2, false, DR_BLOCKED, false, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, DR_DYN_SMEM));
     DR_CUDA(cudaFuncSetAttribute(reshard_kernel<4, false, DR_BLOCKED, false, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, DR_DYN_SMEM));
-    DR_CUDA(cudaFuncSetAttribute(reshard_kernel<2, false, DR_BLOCKED, true, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, DR_DYN_SMEM));
-    DR_CUDA(cudaFuncSetAttribute(reshard_kernel<4, false, DR_BLOCKED, true, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, DR_DYN_SMEM));
     done[device] = true;
     return DR_OK;
 }
@@ -545,16 +535,13 @@ int launch_push(const dr_plan* p, const void* flat, void* const* arenas, uint32_
     dim3 grid((unsigned)n), block(kThreads);
     cudaStream_t s = (cudaStream_t)stream;
     const uint32_t n_segs = (uint32_t)p->dev_segs.size();
-#define DR_LAUNCH_PUSH(ES, BULK)                                                                                \
-    reshard_kernel<ES, false, DR_BLOCKED, true, BULK><<<grid, block, (BULK) ? DR_DYN_SMEM : DR_OCC_SMEM, s>>>(     \
-        p->d_segs, n_segs, p->d_hints, p->hint_shift, 0, n, (char*)flat, (char*)arenas[0], allow256, peers)
-    const bool bulk = DR_BULK && p->bulk_forward;
-    if (p->elem_size == 2) {
-        if (bulk) DR_LAUNCH_PUSH(2, true); else DR_LAUNCH_PUSH(2, false);
-    } else {
-        if (bulk) DR_LAUNCH_PUSH(4, true); else DR_LAUNCH_PUSH(4, false);
-    }
-#undef DR_LAUNCH_PUSH
+    // the register kernel: with several destinations the stream is write-heavy, where the bulk path does not pay
+    if (p->elem_size == 2)
+        reshard_kernel<2, false, DR_BLOCKED, true><<<grid, block, DR_OCC_SMEM, s>>>(
+            p->d_segs, n_segs, p->d_hints, p->hint_shift, 0, n, (char*)flat, (char*)arenas[0], allow256, peers);
+    else
+        reshard_kernel<4, false, DR_BLOCKED, true><<<grid, block, DR_OCC_SMEM, s>>>(
+            p->d_segs, n_segs, p->d_hints, p->hint_shift, 0, n, (char*)flat, (char*)arenas[0], allow256, peers);
     cudaError_t e = cudaGetLastError();
     if (e != cudaSuccess) {
         set_error("push kernel launch: %s", cudaGetErrorString(e));
