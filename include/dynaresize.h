@@ -547,6 +547,15 @@ int dr_host_copy(void* dst_host, const void* src_host, uint64_t n_bytes, uint32_
  */
 int dr_diag_bulk_wait_failures(uint64_t* count);
 
+/*
+ * dr_diag_bulk_starve -- test hook (the paper has no counterpart).  While `on` is non-zero, every tile of the
+ * bulk-copy kernel is told to expect 16 bytes more than its copies deliver on the current device, so its
+ * bounded wait (about 50 ms) has to run out and the tile is redone by the register path: the way to
+ * exercise that path and the counter above without faulting or hanging anything.  The result of
+ * dr_reshard stays correct; it is only slow.  Switch it off again with on = 0.  Synchronous.
+ */
+int dr_diag_bulk_starve(int on);
+
 /* Synchronises the plan's own streams, frees its ring, table and streams.  NULL is accepted. */
 int dr_plan_destroy(dr_plan* plan);
 

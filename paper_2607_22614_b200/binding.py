@@ -21,7 +21,7 @@ DR_STREAM_UNORDERED = 1
 
 EXPORTS = ["dr_plan_create", "dr_plan_create_host", "dr_plan_window_host", "dr_plan_query", "dr_plan_tensor", "dr_plan_segment",
            "dr_reshard", "dr_reshard_inverse", "dr_plan_group", "dr_reshard_groups", "dr_reshard_static", "dr_plan_ranges", "dr_reshard_push", "dr_reshard_stream", "dr_shard_range", "dr_stage_out", "dr_stage_in", "dr_plan_destroy", "dr_strerror",
-           "dr_last_error", "dr_probe_stream", "dr_host_copy", "dr_diag_bulk_wait_failures", "dr_ctl_create", "dr_ctl_observe", "dr_ctl_break_even", "dr_ctl_destroy"]
+           "dr_last_error", "dr_probe_stream", "dr_host_copy", "dr_diag_bulk_wait_failures", "dr_diag_bulk_starve", "dr_ctl_create", "dr_ctl_observe", "dr_ctl_break_even", "dr_ctl_destroy"]
 
 u8, u32, u64, i64, vp = C.c_uint8, C.c_uint32, C.c_uint64, C.c_int64, C.c_void_p
 
@@ -137,6 +137,7 @@ def lib() -> C.CDLL:
         L.dr_probe_stream.argtypes = [u32, vp, vp, u64, vp]
         L.dr_host_copy.argtypes = [vp, vp, u64, u32]
         L.dr_diag_bulk_wait_failures.argtypes = [P(u64)]
+        L.dr_diag_bulk_starve.argtypes = [C.c_int]
         L.dr_ctl_create.argtypes = [P(dr_ctl_config), P(vp)]
         L.dr_ctl_observe.argtypes = [vp, C.c_double, C.c_double, P(C.c_int32), P(u32)]
         L.dr_ctl_break_even.argtypes = [C.c_double, C.c_double, C.c_double, P(C.c_double)]
@@ -325,6 +326,10 @@ def dr_probe_stream(mode, a_dev, b_dev, n_bytes, cuda_stream):
 def dr_diag_bulk_wait_failures():
     n = u64()
     return lib().dr_diag_bulk_wait_failures(C.byref(n)), n.value
+
+
+def dr_diag_bulk_starve(on):
+    return lib().dr_diag_bulk_starve(int(on))
 
 
 def dr_host_copy(dst_host, src_host, n_bytes, threads=0):

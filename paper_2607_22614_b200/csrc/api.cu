@@ -428,6 +428,8 @@ int dr_diag_bulk_wait_failures(uint64_t* count)
     return bulk_wait_failures(count);
 }
 
+int dr_diag_bulk_starve(int on) { return bulk_starve(on); }
+
 const char* dr_strerror(int status)
 {
     switch (status) {

@@ -158,6 +158,7 @@ int launch_reshard(const dr_plan* p, bool inverse, const void* flat, void* arena
 int launch_push(const dr_plan* p, const void* flat, void* const* arenas, uint32_t n_dst, void* stream);
 std::vector<dr_range> plan_ranges(const dr_plan* p);  // planner.cpp: coalesced arena byte ranges the plan writes
 int ensure_bulk_smem(int device);          // once per device: lets the repack kernels ask for their tile buffers
+int bulk_starve(int on);                   // test hook: makes the bulk tiles' bounded waits run out
 int bulk_wait_failures(uint64_t* out);     // bounded mbarrier waits that ran out since the library was loaded (expected: 0)
 int choose_grid(int device, uint32_t elem_size);  // resident CTAs of the reshard kernel on the whole GPU
 // Blocks [block_lo, min(block_hi, all)) of the plan's quantised tensors.

@@ -208,16 +208,30 @@ constexpr uint32_t kTileFlatBytes = kTileUnits * 32;                      // 48 
 constexpr uint32_t kBulkSmemBytes = kTileFlatBytes + kTileFlatBytes / 2;  // + 24 KB of bf16
 constexpr uint32_t kBulkMaxRows = 32;                                     // source rows per tile the first warp can issue
 __device__ unsigned int g_bulk_wait_gave_up = 0;
+// Test hook: when set, every bulk tile expects 16 bytes more than its copies deliver, so its wait has to run out.
+__device__ unsigned int g_bulk_starve = 0;
 
+__device__ __forceinline__ uint64_t global_ns()
+{
+    uint64_t t;
+    asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(t));
+    return t;
+}
+
+// Waits for the barrier's phase `parity`, at most about 50 ms (and never more than 2^22 polls): a tile's copies take
+// microseconds, so a wait that long has failed.
 __device__ __forceinline__ bool mbar_wait_bounded(uint32_t bar, uint32_t parity)
 {
     uint32_t done = 0;
+    const uint64_t t0 = global_ns();
 #pragma unroll 1
-    for (uint32_t it = 0; it < (1u << 22) && !done; ++it)
+    for (uint32_t it = 0; it < (1u << 22) && !done; ++it) {
         asm volatile("{ .reg .pred p; mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2; selp.u32 %0, 1, 0, p; }"
                      : "=r"(done)
                      : "r"(bar), "r"(parity)
                      : "memory");
+        if (!done && (it & 63) == 63 && global_ns() - t0 > 50000000ull) break;
+    }
     return done != 0;
 }
 
@@ -240,7 +254,8 @@ __device__ __forceinline__ bool bulk_forward_tile(const DevSeg& g, uint32_t ub, 
     if (threadIdx.x == 0) {
         asm volatile("mbarrier.init.shared::cta.b64 [%0], 1;" ::"r"(bar));
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
-        asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(bar), "r"(n * 32u) : "memory");
+        asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(bar), "r"(n * 32u + (g_bulk_starve ? 16u : 0u))
+                     : "memory");
     }
     if (threadIdx.x < 32) {
         __syncwarp();  // the byte count is expected before the first copy can complete
@@ -453,6 +468,13 @@ int ensure_bulk_smem(int device)
     DR_CUDA(cudaFuncSetAttribute(reshard_kernel<2, false, DR_BLOCKED, false, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, DR_DYN_SMEM));
     DR_CUDA(cudaFuncSetAttribute(reshard_kernel<4, false, DR_BLOCKED, false, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, DR_DYN_SMEM));
     done[device] = true;
+    return DR_OK;
+}
+
+int bulk_starve(int on)
+{
+    const unsigned int v = on ? 1u : 0u;
+    DR_CUDA(cudaMemcpyToSymbol(g_bulk_starve, &v, sizeof v));
     return DR_OK;
 }
 

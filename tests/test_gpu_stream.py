@@ -123,3 +123,38 @@ def test_no_bounded_device_wait_ran_out():
     rc, n = dr.dr_diag_bulk_wait_failures()
     assert rc == 0 and n == 0
     plan.close()
+
+
+def test_a_bulk_wait_that_runs_out_falls_back_to_the_register_path():
+    """With the test hook on, every tile of the bulk-copy kernel waits for bytes that never come: the wait gives up
+    after about 50 ms, the counter goes up by one per tile, the tile is redone through registers and the arena is
+    still the oracle's.  Nothing faults or hangs; with the hook off again the next call is an ordinary one."""
+    import time
+    spec = CONFIGS[0]["spec"]                                  # 1.98 M elements at TP = 1: 161 tiles, all resident at once
+    om = oracle.Model(spec)
+    src = make_source(om.flat_elems, 12)
+    want = np.full(om.arena_bytes, SENT8, dtype=np.uint8)
+    om.forward(src, want)
+    plan = dr.Plan(spec)
+    assert plan.info.bulk_forward == 1
+    s_dev = torch.from_numpy(src.view(np.int32)).to(dev())
+    arena = torch.full((om.arena_bytes,), SENT8, dtype=torch.uint8, device=dev())
+    torch.cuda.synchronize()
+    rc, before = dr.dr_diag_bulk_wait_failures()
+    assert rc == 0 and dr.dr_diag_bulk_starve(1) == 0
+    try:
+        t0 = time.perf_counter()
+        plan.reshard(s_dev, arena)
+        torch.cuda.synchronize()
+        took = time.perf_counter() - t0
+    finally:
+        assert dr.dr_diag_bulk_starve(0) == 0
+    rc, after = dr.dr_diag_bulk_wait_failures()
+    assert first_diff(arena.cpu().numpy(), want) is None
+    assert after - before == plan.info.n_tiles and 0.05 < took < 5.0
+    arena.fill_(SENT8)
+    plan.reshard(s_dev, arena)                                  # hook off: the ordinary path, no new failures
+    torch.cuda.synchronize()
+    assert first_diff(arena.cpu().numpy(), want) is None
+    assert dr.dr_diag_bulk_wait_failures()[1] == after
+    plan.close()
