@@ -305,9 +305,8 @@ int dr_reshard_push(const dr_plan* plan, const void* src_dev, uint64_t src_bytes
  * 16 384 segments (dr_plan_query: n_segments).  Unlike dr_reshard the call is not purely an enqueue:
  * the table is uploaded from ordinary (pageable) host memory with cudaMemcpyAsync, which the driver may
  * stage and for which it may make the host wait until earlier work on cuda_stream has drained.  The
- * first call on each device looks up the table's device address; make that first call outside any
- * stream capture.  All calls share the one table and
- * it keeps the previous call's entries: each call rewrites the entries it uses, in stream order,
+ * first call on each device also looks up the table's device address.  All calls share the one table
+ * and it keeps the previous call's entries: each call rewrites the entries it uses, in stream order,
  * before its kernel reads them, so calls on one stream are safe back to back, while calls that can
  * overlap on the GPU (different streams, or different threads on different streams) race on the table
  * and must be ordered by the caller.
