@@ -262,6 +262,15 @@ def run_reference(args, cfg):
     print(json.dumps(line))
 
 
+def engine_copy_threads() -> int:
+    """The staging engine's worker count on this machine (its rule, restated for the report)."""
+    env = os.environ.get("DR_COPY_THREADS", "")
+    if env.isdigit() and 1 <= int(env) <= 64:
+        return int(env)
+    n = os.cpu_count() or 1
+    return max(1, min(16, n - 2 if n > 4 else n))
+
+
 def run_all(args):
     """The per-workload table: each workload in a process of its own (device memory is returned in between)."""
     for i in range(5):
@@ -952,7 +961,7 @@ def staging_sections(args, cfg, plan, master, arena, seed, base, dev, world, lin
             "bytes_match": bool(all(x["bytes_match"] for x in rings)),
             "cpu_baseline_host_copy": {
                 "what": "dr_host_copy, the engine's multi-threaded copy (non-temporal stores), 1 GiB, this box's host cores",
-                "threads": min(16, os.cpu_count() or 1),
+                "threads": engine_copy_threads(),
                 "pinned_to_pageable_alone_gbs": alone_out, "pageable_to_pinned_alone_gbs": alone_in,
                 "pinned_to_pageable_beside_d2h_gbs": c_out, "d2h_beside_host_copy_gbs": dma_out,
                 "pageable_to_pinned_beside_h2d_gbs": c_in, "h2d_beside_host_copy_gbs": dma_in,

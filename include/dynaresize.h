@@ -336,9 +336,11 @@ typedef int (*dr_chunk_fn)(void* user, uint64_t chunk_idx, uint64_t stream_off, 
  *                        worker threads
  * A pageable arena is served by worker threads behind the pump (ring slot -> arena on the way out, arena ->
  * ring slot on the way in, in tasks of 1 MiB), so several chunks are in flight on the host side as well.
+ * There are min(16, cores - 2) workers (two cores stay free for the pump and the driver's thread; the
+ * environment variable DR_COPY_THREADS = 1..64, read when a plan first stages, overrides the count).
  * For such an arena a small ring is the fast one: about eight slots of 4 - 8 MiB stay in the host's
  * last-level cache, so a chunk is copied out right behind the DMA that delivered it (and filled right
- * before the DMA that reads it) without a round trip through host DRAM; measured 0.85 - 0.97 of the link
+ * before the DMA that reads it) without a round trip through host DRAM; measured 0.88 - 0.97 of the link
  * against 0.70 - 0.88 with slots of 256 MiB - 1 GiB.  Rings of at most 64 MiB are filled with ordinary
  * stores on the way in, larger ones with non-temporal stores.
  * One stage-out call may mix relay and arena buffers: a rank that keeps training under a new world size
@@ -533,7 +535,7 @@ int dr_probe_stream(uint32_t mode, const void* a_dev, void* b_dev, uint64_t n_by
  * staging engine uses between its pinned ring and a pageable arena (worker threads taking 1 MiB tasks,
  * non-temporal stores), run on its own, so that a benchmark can state what the host's cores sustain
  * without the link (the CPU baseline of staging through pageable memory).  threads = 0 takes the
- * engine's own count (at most 16).  Blocking.  DR_ERR_INVALID on NULL.
+ * engine's own count (see dr_stage_desc).  Blocking.  DR_ERR_INVALID on NULL.
  */
 int dr_host_copy(void* dst_host, const void* src_host, uint64_t n_bytes, uint32_t threads);
 
