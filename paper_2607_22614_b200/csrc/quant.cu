@@ -179,6 +179,15 @@ __device__ __forceinline__ void quant_block(const QTensor& T, uint32_t bi, uint3
     }
 }
 
+// The general form is a call, not inlined: compiled into the kernel body it costs the whole-block path registers
+// (156 instead of 32 bytes of spills at the 80 registers that three CTAs per SM allow).
+__device__ __noinline__ void quant_block_ragged(const QTensor& T, uint32_t bi, uint32_t bj, uint32_t nrows,
+                                                const uint64_t* row_src, float* warp_max, float* s_scale,
+                                                const char* __restrict__ flat, char* __restrict__ arena, int allow256)
+{
+    quant_block<false>(T, bi, bj, nrows, row_src, warp_max, s_scale, flat, arena, allow256);
+}
+
 __global__ void __launch_bounds__(kQThreads, DR_Q_MIN_BLOCKS)
     quant_kernel(const QTensor* __restrict__ tensors, uint32_t n_tensors, const QPart* __restrict__ parts,
                  const uint32_t* __restrict__ hints, uint32_t hint_shift, const char* __restrict__ flat,
@@ -217,7 +226,7 @@ __global__ void __launch_bounds__(kQThreads, DR_Q_MIN_BLOCKS)
     if (nrows == 128 && bj * 128 + 128 <= T.cols && T.aligned && allow256)
         quant_block<true>(T, bi, bj, nrows, row_src, warp_max, &s_scale, flat, arena, allow256);
     else
-        quant_block<false>(T, bi, bj, nrows, row_src, warp_max, &s_scale, flat, arena, allow256);
+        quant_block_ragged(T, bi, bj, nrows, row_src, warp_max, &s_scale, flat, arena, allow256);
 }
 
 // ---- the inverse: e4m3 codes times the block's scale, back to the flat fp32 positions ----------------------
