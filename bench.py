@@ -28,6 +28,7 @@ if ROOT not in sys.path:
 
 METRIC = "role-switch transform GB/s (% of HBM peak); stage-out/in GB/s; switch ms"
 GiB = 1 << 30
+MiB = 1 << 20
 # DRAM bytes per element (dram__bytes_read.sum + dram__bytes_write.sum over elements moved) of the forward
 # kernel, from the committed ncu capture summary of this kernel (a 654 M-element case of the
 # same kernel; traffic grows in proportion to the elements, so it is scaled to the launch timed here).
@@ -736,7 +737,29 @@ def staging_sections(args, cfg, plan, master, arena, seed, base, dev, world, lin
 
     link_d2h, link_h2d = link(GiB, True), link(GiB, False)
     link_d2h_c, link_h2d_c = link(chunk, True), link(chunk, False)
-    del pin, scratch
+
+    # both directions at once (what a relay through the ring can reach): four 1 GiB copies each way on two streams
+    pin2 = torch.empty(GiB, dtype=torch.uint8, pin_memory=True)
+    scratch2 = torch.empty(GiB, dtype=torch.uint8, device=dev)
+    s_out, s_in = torch.cuda.Stream(), torch.cuda.Stream()
+    duplex = []
+    for _ in range(3):
+        torch.cuda.synchronize()
+        ev = [torch.cuda.Event(enable_timing=True) for _ in range(4)]
+        with torch.cuda.stream(s_out):
+            ev[0].record()
+            for _ in range(4):
+                pin[:GiB].copy_(scratch[:GiB], non_blocking=True)
+            ev[1].record()
+        with torch.cuda.stream(s_in):
+            ev[2].record()
+            for _ in range(4):
+                scratch2.copy_(pin2, non_blocking=True)
+            ev[3].record()
+        torch.cuda.synchronize()
+        duplex.append((4 * GiB / ev[0].elapsed_time(ev[1]) / 1e6, 4 * GiB / ev[2].elapsed_time(ev[3]) / 1e6))
+    duplex_d2h, duplex_h2d = max(duplex, key=lambda x: min(x))
+    del pin, scratch, pin2, scratch2
     torch.cuda.empty_cache()
 
     # which state buffers fit: device memory for m and v, host memory for the image
@@ -874,6 +897,28 @@ def staging_sections(args, cfg, plan, master, arena, seed, base, dev, world, lin
                           "weights_resident_ms": best.ready_ms[0], "all_state_resident_ms": best.elapsed_ms,
                           "matches_generator": bool(ok4)}
         plan.stage_in(desc(ptrs, image, order=order))
+
+    # Relay (Sec. 3.3, old rank -> new rank through bounded host buffers): one state buffer goes device -> pinned ring
+    # -> another device buffer, both directions of the link busy at once; the target is the last state buffer,
+    # which is regenerated afterwards.
+    if len(bufs) >= 2:
+        relay = {}
+        for label, b_b, c_b in (("two_slots", budget, budget // 2), ("eight_slots", budget, budget // 8),
+                                ("ring_64MiB_16x4MiB", 64 * MiB, 4 * MiB)):
+            dd = dr.stage_desc(ptrs[:1], sizes[:1], budget=b_b, chunk=c_b, relay_dev=[ptrs[-1]])
+            runs = [plan.stage_out(dd) for _ in range(2)]
+            best = max(runs, key=lambda x: x.link_gbs)
+            relay[label] = {"budget_bytes": b_b, "chunk_bytes": c_b, "gbs": best.link_gbs, "ms": best.elapsed_ms,
+                            "frac_of_duplex_link": best.link_gbs / min(duplex_d2h, duplex_h2d),
+                            "pinned_high_water_bytes": int(best.pinned_high_water_bytes)}
+        torch.cuda.synchronize()
+        relay["target_matches_source"] = bool(torch.equal(bufs[0], bufs[-1]))
+        synth.cuda_fill_f32(bufs[-1], seed, ids[-1], start=base)
+        torch.cuda.synchronize()
+        out["relay"] = {"what": "dr_stage_out with a relay target: device buffer -> pinned ring -> second device buffer, "
+                                f"{sizes[0]} bytes", "bytes": sizes[0],
+                        "link_duplex_d2h_gbs": duplex_d2h, "link_duplex_h2d_gbs": duplex_h2d, **relay,
+                        "gbs": max(relay[k]["gbs"] for k in ("two_slots", "eight_slots", "ring_64MiB_16x4MiB"))}
 
     # the same engine with a pageable resting place: chunks go through the pinned ring and worker threads
     if mem_available_bytes() > 4 * n * 1.5:
