@@ -904,7 +904,7 @@ def staging_sections(args, cfg, plan, master, arena, seed, base, dev, world, lin
     if len(bufs) >= 2:
         relay = {}
         for label, b_b, c_b in (("two_slots", budget, budget // 2), ("eight_slots", budget, budget // 8),
-                                ("ring_64MiB_16x4MiB", 64 * MiB, 4 * MiB)):
+                                ("ring_64MiB_16x4MiB", 64 * MiB, 4 * MiB), ("no_chunk_size_given", budget, 0)):
             dd = dr.stage_desc(ptrs[:1], sizes[:1], budget=b_b, chunk=c_b, relay_dev=[ptrs[-1]])
             runs = [plan.stage_out(dd) for _ in range(2)]
             best = max(runs, key=lambda x: x.link_gbs)
@@ -918,7 +918,7 @@ def staging_sections(args, cfg, plan, master, arena, seed, base, dev, world, lin
         out["relay"] = {"what": "dr_stage_out with a relay target: device buffer -> pinned ring -> second device buffer, "
                                 f"{sizes[0]} bytes", "bytes": sizes[0],
                         "link_duplex_d2h_gbs": duplex_d2h, "link_duplex_h2d_gbs": duplex_h2d, **relay,
-                        "gbs": max(relay[k]["gbs"] for k in ("two_slots", "eight_slots", "ring_64MiB_16x4MiB"))}
+                        "gbs": max(relay[k]["gbs"] for k in ("two_slots", "eight_slots", "ring_64MiB_16x4MiB", "no_chunk_size_given"))}
 
     # the same engine with a pageable resting place: chunks go through the pinned ring and worker threads
     if mem_available_bytes() > 4 * n * 1.5:
@@ -935,7 +935,7 @@ def staging_sections(args, cfg, plan, master, arena, seed, base, dev, world, lin
             ri = [plan.stage_in(dd) for _ in range(2)]
             good &= synth.cuda_mismatch_f32(bufs[0], seed, ids[0], start=base) == 0
             o, i = max(x.link_gbs for x in ro), max(x.link_gbs for x in ri)
-            return {"budget_bytes": int(budget_b), "chunk_bytes": int(chunk_b), "slots": int(budget_b // chunk_b),
+            return {"budget_bytes": int(budget_b), "chunk_bytes": int(chunk_b), "slots": int(budget_b // chunk_b) if chunk_b else None,
                     "pinned_high_water_bytes": int(ro[0].pinned_high_water_bytes), "stage_out_gbs": o, "stage_in_gbs": i,
                     "stage_out_frac_of_link": o / link_d2h, "stage_in_frac_of_link": i / link_h2d, "bytes_match": good}
 
@@ -945,7 +945,15 @@ def staging_sections(args, cfg, plan, master, arena, seed, base, dev, world, lin
         # copied out right behind the DMA that delivered them, and filled right before the DMA that reads them
         small = ring(64 << 20, 8 << 20) if 4 * n >= (1 << 30) else None
         small16 = ring(64 << 20, 4 << 20) if 4 * n >= (1 << 30) else None
-        rings = [x for x in (eight, two, small, small16) if x]
+        # no chunk size given: the engine takes its small ring by itself (what a caller who only states a budget gets)
+        auto = ring(budget, 0)
+        rings = [x for x in (eight, two, small, small16, auto) if x]
+
+        def geometry_name(x):
+            if not x["chunk_bytes"]:
+                return "no chunk size given (the engine's own small ring)"
+            return f'{x["slots"]} x {x["chunk_bytes"] // MiB} MiB'
+
         best_out = max(rings, key=lambda x: x["stage_out_gbs"])
         best_in = max(rings, key=lambda x: x["stage_in_gbs"])
         # CPU baseline of this path: the engine's multi-threaded host copy on its own, and the same copy while the
@@ -1000,9 +1008,10 @@ def staging_sections(args, cfg, plan, master, arena, seed, base, dev, world, lin
         del p1, p2, scratch
         out["staging"]["through_ring_to_pageable"] = {
             "bytes": int(4 * n), "eight_slots": eight, "two_slots": two, "ring_64MiB_8x8MiB": small, "ring_64MiB_16x4MiB": small16,
+            "no_chunk_size_given": auto,
             "stage_out_gbs": best_out["stage_out_gbs"], "stage_in_gbs": best_in["stage_in_gbs"],
             "stage_out_frac_of_link": best_out["stage_out_frac_of_link"], "stage_in_frac_of_link": best_in["stage_in_frac_of_link"],
-            "best_geometry": {"stage_out": [best_out["slots"], best_out["chunk_bytes"]], "stage_in": [best_in["slots"], best_in["chunk_bytes"]]},
+            "best_geometry": {"stage_out": geometry_name(best_out), "stage_in": geometry_name(best_in)},
             "bytes_match": bool(all(x["bytes_match"] for x in rings)),
             "cpu_baseline_host_copy": {
                 "what": "dr_host_copy, the engine's multi-threaded copy (non-temporal stores), 1 GiB, this box's host cores",

@@ -341,8 +341,8 @@ typedef int (*dr_chunk_fn)(void* user, uint64_t chunk_idx, uint64_t stream_off, 
  * For such an arena a small ring is the fast one: about eight slots of 4 - 8 MiB stay in the host's
  * last-level cache, so a chunk is copied out right behind the DMA that delivered it (and filled right
  * before the DMA that reads it) without a round trip through host DRAM; measured 0.88 - 0.97 of the link
- * against 0.70 - 0.88 with slots of 256 MiB - 1 GiB (a relay gains in the same way: 1.0 against 0.8 - 0.9
- * of what the link gives with both directions busy).  Rings of at most 64 MiB are filled with ordinary
+ * against 0.70 - 0.88 with slots of 256 MiB - 1 GiB (a relay reaches what the link gives with both
+ * directions busy through the small ring on every box measured, through large slots only on some).  Rings of at most 64 MiB are filled with ordinary
  * stores on the way in, larger ones with non-temporal stores.
  * One stage-out call may mix relay and arena buffers: a rank that keeps training under a new world size
  * relays the part of its new shard it already holds and rests the remainder of its old shard on the
@@ -354,7 +354,10 @@ typedef struct dr_stage_desc {
     uint64_t bytes[DR_MAX_STAGE_BUFS];
     uint32_t order[DR_MAX_STAGE_BUFS];  /* stage-in priority, a permutation of 0..n_bufs-1            */
     uint64_t budget_bytes;
-    uint64_t chunk_bytes;               /* 0: budget / 2 rounded down to a multiple of 4096           */
+    uint64_t chunk_bytes;               /* 0: budget / 2 rounded down to a multiple of 4096; but where
+                                           the bytes pass through the ring (a relay target, a pageable
+                                           arena) at most 4 MiB on the way out and 8 MiB on the way in,
+                                           in a ring of at most 64 MiB (the fast geometry, see above)  */
     void* host_arena;
     uint64_t host_arena_bytes;
     dr_chunk_fn callback;

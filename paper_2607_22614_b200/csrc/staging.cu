@@ -85,7 +85,14 @@ struct Geometry {
     bool scattered = false;                      // host positions differ from stream positions
 };
 
-int geometry(const dr_stage_desc* d, Geometry* g)
+bool is_pinned_host(const void* p);
+
+// Chunk size a call gets when it names none and its bytes pass through the ring by DMA on one side and by DMA or
+// the worker threads on the other (relay target, pageable arena): slots this small keep the ring inside the host's
+// last-level cache, which is what makes that path fast (see the header).  Never more than the usual budget / 2.
+constexpr uint64_t kAutoChunkOut = 4ull << 20, kAutoChunkIn = 8ull << 20, kAutoRingBytes = 64ull << 20;
+
+int geometry(const dr_stage_desc* d, Geometry* g, bool out)
 {
     if (!d || d->struct_size != sizeof(dr_stage_desc) || d->n_bufs == 0 || d->n_bufs > DR_MAX_STAGE_BUFS) {
         set_error("bad staging descriptor");
@@ -101,13 +108,24 @@ int geometry(const dr_stage_desc* d, Geometry* g)
     g->total = g->prefix[d->n_bufs];
     g->scattered = (d->flags & DR_STAGE_HOST_OFFSETS) != 0;
     for (uint32_t i = 0; i < d->n_bufs; ++i) g->host_at[i] = g->scattered ? d->host_offset[i] : g->prefix[i];
-    g->chunk = d->chunk_bytes ? d->chunk_bytes : d->budget_bytes / 2 / 4096 * 4096;
-    if (g->chunk == 0 || d->budget_bytes / g->chunk < 2) {
+    uint64_t budget = d->budget_bytes;
+    g->chunk = d->chunk_bytes ? d->chunk_bytes : budget / 2 / 4096 * 4096;
+    if (!d->chunk_bytes && !d->callback) {
+        bool relay = false;
+        for (uint32_t i = 0; out && i < d->n_bufs; ++i) relay |= d->relay_dev[i] != nullptr && d->bytes[i] != 0;
+        const bool pageable = d->host_arena && !is_pinned_host(d->host_arena);
+        const uint64_t small = out ? kAutoChunkOut : kAutoChunkIn;
+        if ((relay || pageable) && g->chunk > small) {
+            g->chunk = small;
+            budget = std::min(budget, kAutoRingBytes);
+        }
+    }
+    if (g->chunk == 0 || budget / g->chunk < 2) {
         set_error("budget %llu cannot hold two slots of %llu bytes", (unsigned long long)d->budget_bytes,
                   (unsigned long long)g->chunk);
         return DR_ERR_BUDGET;
     }
-    g->slots = (uint32_t)std::min<uint64_t>(d->budget_bytes / g->chunk, 64);
+    g->slots = (uint32_t)std::min<uint64_t>(budget / g->chunk, 64);
     g->n_chunks = (g->total + g->chunk - 1) / g->chunk;
     return DR_OK;
 }
@@ -283,7 +301,7 @@ extern "C" int dr_stage_out(dr_plan* plan, const dr_stage_desc* d, dr_stage_stat
         return DR_ERR_INVALID;
     }
     Geometry g;
-    int rc = geometry(d, &g);
+    int rc = geometry(d, &g, true);
     if (rc) return rc;
     if ((rc = check_common(plan, d, g, true))) return rc;
     std::lock_guard<std::mutex> lock(plan->stage_mu);
@@ -422,7 +440,7 @@ extern "C" int dr_stage_in(dr_plan* plan, const dr_stage_desc* d, dr_stage_stats
         return DR_ERR_INVALID;
     }
     Geometry g;
-    int rc = geometry(d, &g);
+    int rc = geometry(d, &g, false);
     if (rc) return rc;
     if ((rc = check_common(plan, d, g, false))) return rc;
     {

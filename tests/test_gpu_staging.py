@@ -391,6 +391,44 @@ def test_pageable_arena_with_chunks_of_several_host_copy_tasks(plan, chunk, slot
     assert 0 < st.ready_ms[2] <= st.ready_ms[0] <= st.ready_ms[1]
 
 
+def test_no_chunk_size_given_takes_the_small_ring_where_bytes_pass_through_it(plan):
+    """chunk_bytes = 0 means budget / 2, except where the bytes pass through the ring (pageable arena, relay target) and
+    budget / 2 is large: then 4 MiB chunks on the way out and 8 MiB pieces on the way in, in a ring of at most 64 MiB.
+    A pinned arena and a callback keep budget / 2."""
+    sizes = [60_000_003, 4_099, 41_000_001]
+    host = [synth.fill_f32(71 + i, synth.BUF_ADAM_V, 0, -(-n // 4)).view(np.uint8)[:n].copy() for i, n in enumerate(sizes)]
+    devs = [torch.from_numpy(h).to(dev()) for h in host]
+    total = sum(sizes)
+    budget = 256 * MiB
+    image = np.full(total + 64, 0x5A, dtype=np.uint8)
+    st = plan.stage_out(dr.stage_desc([t.data_ptr() for t in devs], sizes, budget=budget, host_arena=image.ctypes.data,
+                                      host_arena_bytes=total))
+    assert st.n_chunks == st.chunks_done == -(-total // (4 * MiB)) and st.bytes == total
+    assert st.pinned_high_water_bytes == 64 * MiB
+    assert np.array_equal(image[:total], np.concatenate(host)) and (image[total:] == 0x5A).all()
+    back = [torch.zeros_like(t) for t in devs]
+    st = plan.stage_in(dr.stage_desc([t.data_ptr() for t in back], sizes, budget=budget, host_arena=image.ctypes.data,
+                                     host_arena_bytes=total, order=[1, 2, 0]))
+    assert st.chunks_done == st.n_chunks == sum(-(-n // (8 * MiB)) for n in sizes) and st.bytes == total
+    assert st.pinned_high_water_bytes == 64 * MiB
+    assert all(torch.equal(a, b) for a, b in zip(back, devs))
+    # relay: the same small chunks
+    relay = [torch.zeros_like(t) for t in devs]
+    st = plan.stage_out(dr.stage_desc([t.data_ptr() for t in devs], sizes, budget=budget,
+                                      relay_dev=[t.data_ptr() for t in relay]))
+    assert st.n_chunks == -(-total // (4 * MiB)) and st.pinned_high_water_bytes == 64 * MiB
+    torch.cuda.synchronize()
+    assert all(torch.equal(a, b) for a, b in zip(relay, devs))
+    # a pinned arena is copied to directly, in chunks of budget / 2; a small budget keeps budget / 2 everywhere
+    pinned = torch.empty(total, dtype=torch.uint8, pin_memory=True)
+    st = plan.stage_out(dr.stage_desc([t.data_ptr() for t in devs], sizes, budget=budget, host_arena=pinned.data_ptr(),
+                                      host_arena_bytes=total))
+    assert st.n_chunks == -(-total // (budget // 2)) and np.array_equal(pinned.numpy(), np.concatenate(host))
+    st = plan.stage_out(dr.stage_desc([t.data_ptr() for t in devs], sizes, budget=6 * MiB, host_arena=image.ctypes.data,
+                                      host_arena_bytes=total))
+    assert st.n_chunks == -(-total // (3 * MiB)) and st.pinned_high_water_bytes == 6 * MiB
+
+
 def test_host_offset_errors(plan):
     t = torch.zeros(2048, dtype=torch.int32, device=dev())
     host = np.zeros(16384, dtype=np.uint8)
