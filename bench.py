@@ -837,6 +837,38 @@ def staging_sections(args, cfg, plan, master, arena, seed, base, dev, world, lin
     restored_ok = all(synth.cuda_mismatch_f32(b, seed, bid, start=base) == 0 for b, bid in zip(bufs, ids))
     ins = [st_in.link_gbs] + [plan.stage_in(desc(ptrs, image, order=order)).link_gbs for _ in range(2)]
 
+    # The same switch with the deferred call (dr_stage_begin): the host thread is free at once, the weights are waited
+    # for on the caller's stream through their ready event, and the inverse map (rollout arena -> fp32 working copy,
+    # independent of the reload) is enqueued right behind the begin; optimizer state keeps arriving meanwhile.
+    deferred = None
+    free_b, _ = torch.cuda.mem_get_info()
+    if ids[0] == synth.BUF_MASTER and len(bufs) > 1 and free_b > 4 * n * 1.05:
+        work = torch.empty(n, dtype=torch.int32, device=dev)
+        for b in bufs:
+            b.zero_()
+        e0, e_inv = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        torch.cuda.synchronize()
+        t0 = time.perf_counter()
+        e0.record()
+        job = plan.stage_begin(desc(ptrs, image, order=order), dr.DR_STAGE_DIR_IN)
+        t_begin = (time.perf_counter() - t0) * 1e3
+        plan.reshard_inverse(arena, work)
+        e_inv.record()
+        job.wait_buffer(0)
+        e_inv.synchronize()
+        t_critical = (time.perf_counter() - t0) * 1e3
+        st_def = job.end()
+        t_all = (time.perf_counter() - t0) * 1e3
+        torch.cuda.synchronize()
+        ok_def = all(synth.cuda_mismatch_f32(b, seed, bid, start=base) == 0 for b, bid in zip(bufs, ids))
+        deferred = {"what": "dr_stage_begin(stage-in, weights first) + dr_reshard_inverse on the caller's stream + dr_stage_wait_buffer(weights) + dr_stage_end",
+                    "begin_returns_ms": t_begin, "inverse_map_done_ms": e0.elapsed_time(e_inv),
+                    "weights_resident_and_inverse_map_done_ms": t_critical, "weights_resident_ms": st_def.ready_ms[0],
+                    "all_state_resident_ms": t_all, "stage_in_gbs": st_def.link_gbs,
+                    "restored_state_matches_generator": bool(ok_def)}
+        del work
+        torch.cuda.empty_cache()
+
     out["staging"] = {
         "bytes": int(total), "buffers": [("master", "m", "v")[i] for i in ids], "budget_bytes": int(budget),
         "chunk_bytes": int(chunk), "chunks": int(st_out.n_chunks), "sink": "pinned host image, chunked direct copies, "
@@ -854,7 +886,8 @@ def staging_sections(args, cfg, plan, master, arena, seed, base, dev, world, lin
                              "until_state_staged_out": t_switch},
         "rollout_to_train": {"weights_resident": st_in.ready_ms[0] if ids[0] == synth.BUF_MASTER else None,
                              "inverse_map": line.get("inverse", {}).get("ms_avg"),
-                             "all_state_resident_deferred": st_in.elapsed_ms},
+                             "all_state_resident_deferred": st_in.elapsed_ms,
+                             "with_the_deferred_call": deferred},
     }
 
     # Re-shard across a changed training world size (Sec. 3.3; the paper's 6 -> 4 training GPUs): the device buffers

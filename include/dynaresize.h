@@ -413,7 +413,8 @@ typedef struct dr_stage_stats {
  * the master buffer).  Without wait_event the first copy waits for all of caller_stream's pending
  * work, the repack included.  On return every delivered chunk is complete and byte-exact.  Errors: DR_ERR_INVALID, DR_ERR_BUDGET, DR_ERR_SIZE (arena too small),
  * DR_ERR_NOMEM (pinned ring), DR_ERR_SINK, DR_ERR_TIMEOUT, DR_ERR_CUDA, DR_ERR_STATE.
- * Calls on one plan must not overlap in time (they share the ring).
+ * Stage calls on one plan share its ring and are serialised inside the library (a second thread's call
+ * waits for the first to return).
  */
 int dr_stage_out(dr_plan* plan, const dr_stage_desc* desc, dr_stage_stats* stats);
 
@@ -426,6 +427,35 @@ int dr_stage_out(dr_plan* plan, const dr_stage_desc* desc, dr_stage_stats* stats
  * Same pump, errors and threading as above.
  */
 int dr_stage_in(dr_plan* plan, const dr_stage_desc* desc, dr_stage_stats* stats);
+
+/*
+ * Deferred form of the two calls above (Sec. 3.3: only the weights are needed at the transition; the
+ * optimizer states are reloaded off the critical path, while the first step on the new topology is
+ * being prepared).  dr_stage_begin checks the descriptor, fixes the ordering point (everything enqueued
+ * on desc->caller_stream up to this call, or desc->wait_event) and starts the same pump on a thread the
+ * library owns; it returns at once.  The caller goes on (typically: runs dr_reshard_inverse, waits for the weights with
+ * dr_stage_wait_buffer, starts the step) and later collects the result:
+ *   dr_stage_wait_buffer : (stage-in) blocks the calling thread, at most timeout_ms (0 = 60 s), until
+ *                   buffer i is resident: its last copy has completed, so work enqueued afterwards on any
+ *                   stream may use it.  This is the way to wait for the weights here: ready_events[i] is
+ *                   recorded by the library's thread when the buffer's last copy is enqueued, and a
+ *                   cudaStreamWaitEvent on an event that has not been recorded yet does not wait at all.
+ *                   DR_ERR_TIMEOUT; the job's own error if the pump ended without the buffer.
+ *   dr_stage_poll : *done = 1 once the pump has returned (never blocks)
+ *   dr_stage_end  : waits for the pump, fills stats, returns the status dr_stage_out / dr_stage_in
+ *                   would have returned (with its message in dr_last_error) and frees the job
+ * direction: DR_STAGE_DIR_OUT or DR_STAGE_DIR_IN.  The descriptor is copied; the buffers, the arena, the
+ * events and the callback it names must stay valid until dr_stage_end.  A callback runs on the library's
+ * thread.  Every job must be ended before its plan is destroyed; jobs on one plan run one after the
+ * other.  Errors of dr_stage_begin: DR_ERR_INVALID, DR_ERR_BUDGET, DR_ERR_SIZE, DR_ERR_STATE (found
+ * before anything is started), DR_ERR_NOMEM, DR_ERR_CUDA.
+ */
+typedef struct dr_stage_job dr_stage_job;
+enum { DR_STAGE_DIR_OUT = 0, DR_STAGE_DIR_IN = 1 };
+int dr_stage_begin(dr_plan* plan, const dr_stage_desc* desc, int direction, dr_stage_job** job);
+int dr_stage_wait_buffer(dr_stage_job* job, uint32_t buffer, uint32_t timeout_ms);
+int dr_stage_poll(const dr_stage_job* job, int* done);
+int dr_stage_end(dr_stage_job* job, dr_stage_stats* stats);
 
 /*
  * Streamed repack: Training -> Rollout for a GPU that does not hold the fp32 master.  The flat source

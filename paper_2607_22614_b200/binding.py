@@ -18,9 +18,10 @@ DR_MAX_STAGE_BUFS = 8
 DR_STAGE_HOST_OFFSETS = 1
 DR_STAGE_UNORDERED = 2
 DR_STREAM_UNORDERED = 1
+DR_STAGE_DIR_OUT, DR_STAGE_DIR_IN = 0, 1
 
 EXPORTS = ["dr_plan_create", "dr_plan_create_host", "dr_plan_window_host", "dr_plan_query", "dr_plan_tensor", "dr_plan_segment",
-           "dr_reshard", "dr_reshard_inverse", "dr_plan_group", "dr_reshard_groups", "dr_reshard_static", "dr_plan_ranges", "dr_reshard_push", "dr_reshard_stream", "dr_shard_range", "dr_stage_out", "dr_stage_in", "dr_plan_destroy", "dr_strerror",
+           "dr_reshard", "dr_reshard_inverse", "dr_plan_group", "dr_reshard_groups", "dr_reshard_static", "dr_plan_ranges", "dr_reshard_push", "dr_reshard_stream", "dr_shard_range", "dr_stage_out", "dr_stage_in", "dr_stage_begin", "dr_stage_wait_buffer", "dr_stage_poll", "dr_stage_end", "dr_plan_destroy", "dr_strerror",
            "dr_last_error", "dr_probe_stream", "dr_host_copy", "dr_diag_bulk_wait_failures", "dr_diag_bulk_starve", "dr_ctl_create", "dr_ctl_observe", "dr_ctl_break_even", "dr_ctl_destroy"]
 
 u8, u32, u64, i64, vp = C.c_uint8, C.c_uint32, C.c_uint64, C.c_int64, C.c_void_p
@@ -131,6 +132,10 @@ def lib() -> C.CDLL:
         L.dr_reshard_groups.argtypes = [vp, u32, u32, vp, u64, vp, u64, vp]
         L.dr_stage_out.argtypes = [vp, P(dr_stage_desc), P(dr_stage_stats)]
         L.dr_stage_in.argtypes = [vp, P(dr_stage_desc), P(dr_stage_stats)]
+        L.dr_stage_begin.argtypes = [vp, P(dr_stage_desc), C.c_int, P(vp)]
+        L.dr_stage_wait_buffer.argtypes = [vp, u32, u32]
+        L.dr_stage_poll.argtypes = [vp, P(C.c_int)]
+        L.dr_stage_end.argtypes = [vp, P(dr_stage_stats)]
         L.dr_reshard_stream.argtypes = [vp, P(dr_stream_desc), P(dr_stream_stats)]
         L.dr_plan_destroy.argtypes = [vp]
         L.dr_shard_range.argtypes = [u64, u32, u32, P(u64), P(u64), P(u64)]
@@ -299,6 +304,26 @@ def dr_stage_in(plan, desc):
     return lib().dr_stage_in(plan, C.byref(desc), C.byref(st)), st
 
 
+def dr_stage_begin(plan, desc, direction):
+    """Starts dr_stage_out / dr_stage_in on a thread of the library's own; returns (status, job handle)."""
+    job = vp()
+    return lib().dr_stage_begin(plan, C.byref(desc), direction, C.byref(job)), job
+
+
+def dr_stage_wait_buffer(job, buffer, timeout_ms=0):
+    return lib().dr_stage_wait_buffer(job, buffer, timeout_ms)
+
+
+def dr_stage_poll(job):
+    done = C.c_int(0)
+    return lib().dr_stage_poll(job, C.byref(done)), bool(done.value)
+
+
+def dr_stage_end(job):
+    st = dr_stage_stats()
+    return lib().dr_stage_end(job, C.byref(st)), st
+
+
 def stream_desc(host_src, host_src_bytes, dst_dev, dst_bytes, window_dev, window_bytes, chunk_bytes=0, host_dst=None,
                 host_dst_bytes=0, timeout_ms=0, caller_stream=None, wait_event=None, done_event=None,
                 unordered=False) -> dr_stream_desc:
@@ -378,6 +403,36 @@ def dr_last_error() -> str:
 
 
 # ---- convenience wrapper (raises instead of returning codes; still marshalling only) -------------
+class StageJob:
+    """A deferred stage call (dr_stage_begin): poll() tells whether the pump has returned, end() collects it."""
+
+    def __init__(self, handle, desc):
+        self.handle, self.desc = handle, desc
+
+    def poll(self) -> bool:
+        rc, done = dr_stage_poll(self.handle)
+        if rc:
+            raise DrError(rc, "dr_stage_poll")
+        return done
+
+    def wait_buffer(self, buffer: int, timeout_ms: int = 0) -> None:
+        """Blocks until buffer `buffer` of a stage-in job is resident (dr_stage_wait_buffer)."""
+        rc = dr_stage_wait_buffer(self.handle, buffer, timeout_ms)
+        if rc:
+            raise DrError(rc, "dr_stage_wait_buffer")
+
+    def end(self):
+        if self.handle is None:
+            raise RuntimeError("job already ended")
+        rc, st = dr_stage_end(self.handle)
+        self.handle = None
+        if rc:
+            e = DrError(rc, "dr_stage_end")
+            e.stats = st
+            raise e
+        return st
+
+
 class Plan:
     """Owns one ``dr_plan``.  ``host_only=True`` builds the planner's tables without touching CUDA."""
 
@@ -489,3 +544,10 @@ class Plan:
             e.stats = st
             raise e
         return st
+
+    def stage_begin(self, desc, direction):
+        """dr_stage_begin: the pump runs on the library's thread; returns a StageJob (keep `desc` and its buffers alive)."""
+        rc, job = dr_stage_begin(self.handle, desc, direction)
+        if rc:
+            raise DrError(rc, "dr_stage_begin")
+        return StageJob(job, desc)

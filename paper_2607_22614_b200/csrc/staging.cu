@@ -11,6 +11,7 @@
 #include <cstring>
 #include <exception>
 #include <functional>
+#include <string>
 #include <thread>
 
 #include "copy_pool.h"
@@ -46,6 +47,9 @@ unsigned default_copy_threads()
 }
 
 }  // namespace
+
+// Set by the deferred form's thread: where dr_stage_in announces, buffer by buffer, that a buffer is resident.
+thread_local std::atomic<int>* tl_buffer_ready = nullptr;
 
 struct Ring {
     cudaStream_t s_copy = nullptr, s_relay = nullptr;
@@ -477,6 +481,12 @@ extern "C" int dr_stage_in(dr_plan* plan, const dr_stage_desc* d, dr_stage_stats
     st.chunks_done = std::min<uint64_t>(d->first_chunk, pieces.size());
     st.pinned_high_water_bytes = direct ? 0 : g.chunk * g.slots;
     if ((rc = order_after_caller(r, d))) return rc;
+    if (tl_buffer_ready) {  // buffers this call has nothing to do for: empty, or complete before first_chunk
+        bool pending[DR_MAX_STAGE_BUFS] = {false};
+        for (uint64_t i = st.chunks_done; i < pieces.size(); ++i) pending[pieces[i].buf] = true;
+        for (uint32_t b = 0; b < d->n_bufs; ++b)
+            if (!pending[b]) tl_buffer_ready[b].store(1, std::memory_order_release);
+    }
 
     auto issue = [&](uint64_t i) -> int {
         const Piece& pc = pieces[i];
@@ -505,7 +515,10 @@ extern "C" int dr_stage_in(dr_plan* plan, const dr_stage_desc* d, dr_stage_stats
         int w = wait_event(r->ev_copy[i % g.slots], Clock::now() + limit);
         if (w) return w;
         st.bytes += pieces[i].n;
-        if (pieces[i].last) st.ready_ms[pieces[i].buf] = ms_since(t0);
+        if (pieces[i].last) {
+            st.ready_ms[pieces[i].buf] = ms_since(t0);
+            if (tl_buffer_ready) tl_buffer_ready[pieces[i].buf].store(1, std::memory_order_release);
+        }
         return DR_OK;
     };
 
@@ -546,7 +559,10 @@ extern "C" int dr_stage_in(dr_plan* plan, const dr_stage_desc* d, dr_stage_stats
             // retire arrivals without blocking, so that their slots can be refilled at once
             while (next_done < next_issue && cudaEventQuery(r->ev_copy[next_done % g.slots]) == cudaSuccess) {
                 st.bytes += pieces[next_done].n;
-                if (pieces[next_done].last) st.ready_ms[pieces[next_done].buf] = ms_since(t0);
+                if (pieces[next_done].last) {
+                    st.ready_ms[pieces[next_done].buf] = ms_since(t0);
+                    if (tl_buffer_ready) tl_buffer_ready[pieces[next_done].buf].store(1, std::memory_order_release);
+                }
                 st.chunks_done = ++next_done;
             }
             while (next_fill < pieces.size() && next_fill - next_done < g.slots) fill(next_fill++);
@@ -571,7 +587,10 @@ extern "C" int dr_stage_in(dr_plan* plan, const dr_stage_desc* d, dr_stage_stats
         // pieces that were on their way when the call failed have landed during the drain: they count as done
         while (next_done < next_issue && cudaEventQuery(r->ev_copy[next_done % g.slots]) == cudaSuccess) {
             st.bytes += pieces[next_done].n;
-            if (pieces[next_done].last) st.ready_ms[pieces[next_done].buf] = ms_since(t0);
+            if (pieces[next_done].last) {
+                st.ready_ms[pieces[next_done].buf] = ms_since(t0);
+                if (tl_buffer_ready) tl_buffer_ready[pieces[next_done].buf].store(1, std::memory_order_release);
+            }
             st.chunks_done = ++next_done;
         }
     }
@@ -579,6 +598,121 @@ extern "C" int dr_stage_in(dr_plan* plan, const dr_stage_desc* d, dr_stage_stats
     st.elapsed_ms = ms_since(t0);
     st.link_gbs = st.elapsed_ms > 0 ? (double)st.bytes / st.elapsed_ms * 1e-6 : 0;
     if (stats) *stats = st;
+    return rc;
+}
+
+// ---- deferred form: the same pump on a thread of the library's own --------------------------------------------
+struct dr_stage_job {
+    std::thread th;
+    dr_plan* plan = nullptr;
+    dr_stage_desc desc{};
+    int direction = 0;
+    dr_stage_stats stats{};
+    int rc = DR_OK;
+    std::string err;
+    std::atomic<int> done{0};
+    std::atomic<int> ready[DR_MAX_STAGE_BUFS];  // stage-in: buffer i is resident (its last copy has completed)
+    cudaEvent_t entry = nullptr;  // the ordering point, recorded on the caller's stream by dr_stage_begin
+};
+
+extern "C" int dr_stage_begin(dr_plan* plan, const dr_stage_desc* d, int direction, dr_stage_job** out)
+{
+    if (!plan || !out || (direction != DR_STAGE_DIR_OUT && direction != DR_STAGE_DIR_IN)) {
+        set_error("NULL plan or job pointer, or unknown direction");
+        return DR_ERR_INVALID;
+    }
+    *out = nullptr;
+    Geometry g;
+    int rc = geometry(d, &g, direction == DR_STAGE_DIR_OUT);
+    if (rc) return rc;
+    if ((rc = check_common(plan, d, g, direction == DR_STAGE_DIR_OUT))) return rc;
+    dr_stage_job* job = new (std::nothrow) dr_stage_job();
+    if (!job) return DR_ERR_NOMEM;
+    for (auto& r : job->ready) r.store(0);
+    job->plan = plan;
+    job->desc = *d;
+    job->direction = direction;
+    // the pump would take its ordering point when it starts, some time after this call has returned: take it now
+    if (!d->wait_event && !(d->flags & DR_STAGE_UNORDERED)) {
+        cudaError_t e = cudaEventCreateWithFlags(&job->entry, cudaEventDisableTiming);
+        if (e == cudaSuccess) e = cudaEventRecord(job->entry, (cudaStream_t)d->caller_stream);
+        if (e != cudaSuccess) {
+            set_error("ordering event: %s", cudaGetErrorString(e));
+            if (job->entry) cudaEventDestroy(job->entry);
+            delete job;
+            return DR_ERR_CUDA;
+        }
+        job->desc.wait_event = job->entry;
+    }
+    try {
+        job->th = std::thread([job] {
+            if (cudaSetDevice(job->plan->device) != cudaSuccess) {
+                job->rc = DR_ERR_CUDA;
+                job->err = "cudaSetDevice on the staging thread failed";
+            } else {
+                tl_buffer_ready = job->ready;
+                job->rc = job->direction == DR_STAGE_DIR_OUT ? dr_stage_out(job->plan, &job->desc, &job->stats)
+                                                             : dr_stage_in(job->plan, &job->desc, &job->stats);
+                tl_buffer_ready = nullptr;
+                if (job->rc) job->err = dr_last_error();
+            }
+            job->done.store(1, std::memory_order_release);
+        });
+    } catch (const std::exception& e) {
+        set_error("cannot start the staging thread: %s", e.what());
+        if (job->entry) cudaEventDestroy(job->entry);
+        delete job;
+        return DR_ERR_NOMEM;
+    }
+    *out = job;
+    return DR_OK;
+}
+
+extern "C" int dr_stage_poll(const dr_stage_job* job, int* done)
+{
+    if (!job || !done) {
+        set_error("NULL job or result pointer");
+        return DR_ERR_INVALID;
+    }
+    *done = job->done.load(std::memory_order_acquire);
+    return DR_OK;
+}
+
+extern "C" int dr_stage_wait_buffer(dr_stage_job* job, uint32_t buffer, uint32_t timeout_ms)
+{
+    if (!job || buffer >= DR_MAX_STAGE_BUFS || buffer >= job->desc.n_bufs || job->direction != DR_STAGE_DIR_IN) {
+        set_error("NULL job, buffer index out of range, or not a stage-in job");
+        return DR_ERR_INVALID;
+    }
+    const auto deadline = Clock::now() + std::chrono::milliseconds(timeout_ms ? timeout_ms : 60000);
+    for (unsigned spins = 0;; ++spins) {
+        if (job->ready[buffer].load(std::memory_order_acquire)) return DR_OK;
+        if (job->done.load(std::memory_order_acquire)) {  // the pump has returned without this buffer: it failed
+            if (job->ready[buffer].load(std::memory_order_acquire)) return DR_OK;
+            set_error("the stage-in ended before buffer %u was resident: %s", buffer, job->err.c_str());
+            return job->rc ? job->rc : DR_ERR_STATE;
+        }
+        if (Clock::now() > deadline) {
+            set_error("buffer %u not resident within the time given", buffer);
+            return DR_ERR_TIMEOUT;
+        }
+        if (spins < 200) std::this_thread::yield();
+        else std::this_thread::sleep_for(std::chrono::microseconds(50));
+    }
+}
+
+extern "C" int dr_stage_end(dr_stage_job* job, dr_stage_stats* stats)
+{
+    if (!job) {
+        set_error("NULL job");
+        return DR_ERR_INVALID;
+    }
+    if (job->th.joinable()) job->th.join();
+    if (job->entry) cudaEventDestroy(job->entry);
+    if (stats) *stats = job->stats;
+    const int rc = job->rc;
+    if (rc) set_error("%s", job->err.c_str());
+    delete job;
     return rc;
 }
 

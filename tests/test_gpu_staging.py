@@ -515,3 +515,84 @@ def test_done_event_and_unordered_flag(plan):
     plan.stage_out(d)
     assert done.query()                                   # the call blocks until its copies are complete
     assert np.array_equal(image.view(np.uint32), host[0])
+
+
+def test_deferred_stage_in_weights_first_while_the_caller_goes_on(plan):
+    """dr_stage_begin / dr_stage_end (Sec. 3.3: only the weights at the transition, optimizer state deferred): the pump
+    runs on the library's thread; the caller waits for the weights' ready event on its own stream, works on them, and
+    collects the job later.  The ordering point is taken at begin: the zero-fills queued before it cannot land late."""
+    sizes = [24_000_004, 64_000_004, 64_000_004]
+    host = [synth.fill_f32(81 + i, synth.BUF_ADAM_M, 0, n // 4).view(np.uint8).copy() for i, n in enumerate(sizes)]
+    total = sum(sizes)
+    image = torch.empty(total, dtype=torch.uint8, pin_memory=True)
+    image.numpy()[:] = np.concatenate(host)
+    back = [torch.empty(n, dtype=torch.uint8, device=dev()) for n in sizes]
+    big = torch.empty(1 << 28, dtype=torch.int32, device=dev())
+    for _ in range(8):
+        big.fill_(1)                       # keeps the stream busy while begin is called
+    for b in back:
+        b.zero_()
+    ready = [torch.cuda.Event() for _ in sizes]
+    d = dr.stage_desc([b.data_ptr() for b in back], sizes, budget=8 * MiB, host_arena=image.data_ptr(),
+                      host_arena_bytes=total, order=[0, 1, 2], ready_events=[e.cuda_event for e in ready])
+    job = plan.stage_begin(d, dr.DR_STAGE_DIR_IN)
+    job.wait_buffer(0)                                         # the weights: resident, usable by anything enqueued from here on
+    doubled = back[0].to(torch.int32) * 2                      # the caller's work on them
+    still_running = not job.poll()
+    job.wait_buffer(1, timeout_ms=30000)
+    st = job.end()
+    assert isinstance(still_running, bool)
+    torch.cuda.synchronize()
+    assert st.bytes == total and st.chunks_done == st.n_chunks
+    assert 0 < st.ready_ms[0] <= st.ready_ms[1] <= st.ready_ms[2] <= st.elapsed_ms
+    assert all(np.array_equal(b.cpu().numpy(), h) for b, h in zip(back, host))
+    assert np.array_equal(doubled.cpu().numpy(), host[0].astype(np.int32) * 2)
+
+
+def test_deferred_stage_out_reports_a_failing_sink_at_end_and_jobs_on_one_plan_run_in_turn(plan):
+    n = 6_000_000
+    host = [synth.fill_f32(91 + i, synth.BUF_ADAM_V, 0, n // 4).view(np.uint8).copy() for i in range(2)]
+    devs = [torch.from_numpy(h).to(dev()) for h in host]
+    images = [np.zeros(n, dtype=np.uint8) for _ in range(2)]
+    torch.cuda.synchronize()
+    descs = [dr.stage_desc([devs[i].data_ptr()], [n], budget=2 * MiB, chunk=MiB, host_arena=images[i].ctypes.data,
+                           host_arena_bytes=n) for i in range(2)]
+    jobs = [plan.stage_begin(descs[i], dr.DR_STAGE_DIR_OUT) for i in range(2)]   # both started; the plan serialises them
+    stats = [j.end() for j in jobs]
+    assert all(j.handle is None for j in jobs)
+    for i in range(2):
+        assert stats[i].bytes == n and np.array_equal(images[i], host[i])
+
+    seen = []
+
+    def sink(user, k, off, ptr, nbytes):
+        seen.append(k)
+        return 1 if k == 3 else 0
+
+    cb = B.dr_chunk_fn(sink)
+    job = plan.stage_begin(dr.stage_desc([devs[0].data_ptr()], [n], budget=2 * MiB, chunk=MiB, callback=cb), dr.DR_STAGE_DIR_OUT)
+    with pytest.raises(dr.DrError) as w:
+        job.wait_buffer(0)                                    # not a stage-in job
+    assert w.value.status == B.DR_ERR_INVALID
+    with pytest.raises(dr.DrError) as e:
+        job.end()
+    assert e.value.status == B.DR_ERR_SINK and e.value.stats.chunks_done == 3 and seen == [0, 1, 2, 3]
+    assert "callback" in dr.dr_last_error()
+    # a stage-in whose source fails: the wait for a buffer that will not arrive ends with the job's own error
+    back = torch.zeros(n, dtype=torch.uint8, device=dev())
+
+    def source(user, k, off, ptr, nbytes):
+        return 1 if k == 2 else 0
+
+    cb2 = B.dr_chunk_fn(source)
+    job = plan.stage_begin(dr.stage_desc([back.data_ptr()], [n], budget=2 * MiB, chunk=MiB, callback=cb2), dr.DR_STAGE_DIR_IN)
+    with pytest.raises(dr.DrError) as w:
+        job.wait_buffer(0, timeout_ms=30000)
+    assert w.value.status == B.DR_ERR_SINK
+    with pytest.raises(dr.DrError) as e:
+        job.end()
+    assert e.value.status == B.DR_ERR_SINK and e.value.stats.chunks_done == 2
+    # errors that need nothing started are reported by begin itself
+    bad = dr.stage_desc([devs[0].data_ptr()], [n], budget=MiB, chunk=MiB, host_arena=images[0].ctypes.data, host_arena_bytes=n)
+    assert dr.dr_stage_begin(plan.handle, bad, dr.DR_STAGE_DIR_OUT)[0] == B.DR_ERR_BUDGET
+    assert dr.dr_stage_begin(plan.handle, descs[0], 7)[0] == B.DR_ERR_INVALID

@@ -191,6 +191,13 @@ def test_error_codes():
     d = dr.stage_desc([16], [4096], budget=4096, chunk=4096, host_arena=4096, host_arena_bytes=4096)
     rc, _ = dr.dr_stage_out(p.handle, d)
     assert rc == dr.binding.DR_ERR_BUDGET
+    # the deferred form checks the same things before it starts anything
+    rc, job = dr.dr_stage_begin(p.handle, d, dr.DR_STAGE_DIR_OUT)
+    assert rc == dr.binding.DR_ERR_BUDGET and not job
+    d = dr.stage_desc([16], [4096], budget=1 << 20, host_arena=4096, host_arena_bytes=4096)
+    assert dr.dr_stage_begin(p.handle, d, dr.DR_STAGE_DIR_IN)[0] == dr.binding.DR_ERR_STATE
+    assert dr.dr_stage_begin(p.handle, d, 2)[0] == dr.binding.DR_ERR_INVALID
+    assert dr.dr_stage_end(None)[0] == dr.binding.DR_ERR_INVALID and dr.dr_stage_poll(None)[0] == dr.binding.DR_ERR_INVALID
     assert dr.dr_plan_tensor(p.handle, 10_000)[0] == dr.binding.DR_ERR_INVALID
     assert "budget" in dr.dr_strerror(dr.binding.DR_ERR_BUDGET)
     assert dr.dr_plan_destroy(None) == 0
