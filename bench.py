@@ -263,6 +263,16 @@ def run_reference(args, cfg):
     print(json.dumps(line))
 
 
+def duplex_model_ms(h2d_bytes, d2h_bytes, h2d_alone_gbs, h2d_duplex_gbs, d2h_duplex_gbs):
+    """Time of a transfer of h2d_bytes in and d2h_bytes out over a link that runs the two directions at the duplex rates
+    while both are busy and the remaining direction at its own rate afterwards (rates in GB/s = bytes / ns)."""
+    t_out = d2h_bytes / d2h_duplex_gbs  # ns
+    t_in_beside = h2d_bytes / h2d_duplex_gbs
+    if t_in_beside <= t_out:
+        return t_out / 1e6
+    return (t_out + (h2d_bytes - t_out * h2d_duplex_gbs) / h2d_alone_gbs) / 1e6
+
+
 def engine_copy_threads() -> int:
     """The staging engine's worker count on this machine (its rule, restated for the report)."""
     env = os.environ.get("DR_COPY_THREADS", "")
@@ -1093,7 +1103,7 @@ def staging_sections(args, cfg, plan, master, arena, seed, base, dev, world, lin
     # the same switch as one streamed call: H2D chunks, per-chunk repack and D2H of finished arena ranges overlap
     window = torch.empty(budget, dtype=torch.uint8, device=dev)
     sd = dr.stream_desc(h_src.data_ptr(), info.src_bytes, arena.data_ptr(), info.dst_bytes, window.data_ptr(), budget,
-                        chunk_bytes=budget // 8, host_dst=h_dst.data_ptr(), host_dst_bytes=info.dst_bytes)
+                        chunk_bytes=0, host_dst=h_dst.data_ptr(), host_dst_bytes=info.dst_bytes)
     h_dst.zero_()
     times, kernels = [], 0
     for i in range(e2e_steps + 1):
@@ -1111,8 +1121,12 @@ def staging_sections(args, cfg, plan, master, arena, seed, base, dev, world, lin
                   "steps": e2e_steps, "h2d_bytes_per_step": int(info.src_bytes), "d2h_bytes_per_step": int(info.dst_bytes),
                   "path": "dr_reshard_stream: pinned host master -> chunked H2D -> per-chunk repack -> D2H of finished arena "
                           "ranges to pinned host, three overlapped streams", "kernels_per_step": kernels,
-                  "window_bytes": int(budget), "chunk_bytes": int(budget // 8), "host_result_matches_device": host_ok,
+                  "window_bytes": int(budget), "chunk_bytes": int(min(budget // 2 // 4096 * 4096, 32 * MiB)),
+                  "chunk_choice": "the call's own (no chunk size given)", "host_result_matches_device": host_ok,
                   "duplex_ideal_ms": max(info.src_bytes / link_h2d, info.dst_bytes / link_d2h) / 1e6,
+                  # what the link gives when both directions are busy (measured above): the copy back runs at the duplex
+                  # D2H rate, the copy in at the duplex H2D rate beside it and at the full rate for the rest
+                  "duplex_link_model_ms": duplex_model_ms(info.src_bytes, info.dst_bytes, link_h2d, duplex_h2d, duplex_d2h),
                   "sequential": {"value": world * info.bytes_moved_fwd / t_seq / 1e9, "ms_per_step": t_seq * 1e3,
                                  "path": "dr_stage_in(master) -> dr_reshard -> dr_stage_out(arena), one after the other",
                                  "link_bound_ideal_ms": (info.src_bytes / link_h2d + info.dst_bytes / link_d2h) / 1e6}}

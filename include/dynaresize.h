@@ -477,7 +477,8 @@ typedef struct dr_stream_desc {
     uint64_t host_dst_bytes;
     void* window_dev;             /* device scratch the caller owns: slots = floor(window / chunk) >= 2 */
     uint64_t window_bytes;
-    uint64_t chunk_bytes;         /* multiple of 32; 0: window_bytes / 2 rounded down to 4096          */
+    uint64_t chunk_bytes;         /* multiple of 32; 0: window_bytes / 2 rounded down to 4096, at most
+                                     32 MiB (at most 16 chunks of the window are in use at a time)      */
     uint32_t timeout_ms;          /* bound on the final wait; 0 = 60 000                               */
     uint32_t pad;
     void* caller_stream;          /* cudaStream_t on which the caller last touched dst_dev / window_dev

@@ -141,7 +141,10 @@ extern "C" int dr_reshard_stream(dr_plan* plan, const dr_stream_desc* d, dr_stre
         set_error("pointers must be 32-byte aligned");
         return DR_ERR_ALIGN;
     }
-    const uint64_t chunk = d->chunk_bytes ? d->chunk_bytes : d->window_bytes / 2 / 4096 * 4096;
+    // no chunk size given: half the window, but not more than 32 MiB: small chunks start the pipeline early and
+    // interleave the copy back with the copy in more finely (measured on the Qwen3-8B shape with the result copied
+    // back to the host: 616 ms with 32 MiB chunks, 621 / 625 / 630 / 632 ms with 64 / 128 / 256 / 512 MiB)
+    const uint64_t chunk = d->chunk_bytes ? d->chunk_bytes : std::min<uint64_t>(d->window_bytes / 2 / 4096 * 4096, 32ull << 20);
     if (chunk % 32) {
         set_error("chunk_bytes %llu is not a multiple of 32", (unsigned long long)chunk);
         return DR_ERR_INVALID;
