@@ -329,3 +329,36 @@ def test_groups_in_any_order_build_up_the_full_repack(spec, kw):
     bad = dr.dr_reshard_groups(plan.handle, 1, plan.info.n_groups, src.data_ptr(), src.numel() * 4, arena.data_ptr(), arena.numel(), s)
     assert bad == dr.binding.DR_ERR_INVALID
     plan.close()
+
+
+def test_the_bulk_copy_kernel_replays_from_a_cuda_graph_too():
+    """The kernel that moves tiles with bulk copies (dynamic shared memory, mbarrier) is captured and replayed like the
+    register kernel: each replay repacks whatever the source buffer holds at that time."""
+    spec, kw = MOE32, dict(tp=2, tp_rank=0)
+    om = oracle.Model(spec, **kw)
+    plan = dr.Plan(spec, **kw)
+    assert plan.info.bulk_forward == 1
+    src = torch.zeros(om.shard_elems, dtype=torch.int32, device=dev())
+    arena = arena_dev(om.arena_bytes)
+    back = torch.zeros(om.shard_elems, dtype=torch.int32, device=dev())
+    plan.reshard(src, arena)            # an ordinary call first
+    plan.reshard_inverse(arena, back)
+    torch.cuda.synchronize()
+    g = torch.cuda.CUDAGraph()
+    with torch.cuda.graph(g):           # captures what is enqueued on torch's current (capturing) stream
+        plan.reshard(src, arena)
+        plan.reshard_inverse(arena, back)
+    for seed in (3, 4):
+        host = make_source(om.shard_elems, seed)
+        src.copy_(torch.from_numpy(host.view(np.int32)))
+        arena.fill_(SENT8)
+        back.fill_(0x5A5A5A5A)
+        g.replay()
+        torch.cuda.synchronize()
+        want = np.full(om.arena_bytes, SENT8, dtype=np.uint8)
+        om.forward(host, want)
+        assert first_diff(arena.cpu().numpy(), want) is None
+        want_back = np.full(om.shard_elems, 0x5A5A5A5A, dtype=np.uint32)
+        om.inverse(want, want_back)
+        assert np.array_equal(back.cpu().numpy().view(np.uint32), want_back)
+    plan.close()
