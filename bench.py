@@ -65,20 +65,37 @@ class ClockSampler:
         self.proc = None
         self.path = None
 
+    def _lines(self) -> int:
+        try:
+            with open(self.path) as f:
+                return sum(1 for _ in f)
+        except OSError:
+            return 0
+
     def start(self):
+        """Starts nvidia-smi and waits (at most 5 s) for its first line: the tool needs a few hundred milliseconds to
+        come up, which is longer than a short timed region.  Call before the warm-up steps."""
         fd, self.path = tempfile.mkstemp(suffix=".csv")
         os.close(fd)
         try:
             self.proc = subprocess.Popen(
                 ["nvidia-smi", "-i", str(self.index), f"--query-gpu={self.FIELDS}", "--format=csv,noheader,nounits",
-                 "-lms", "100"], stdout=open(self.path, "w"), stderr=subprocess.DEVNULL)
+                 "-lms", "50"], stdout=open(self.path, "w"), stderr=subprocess.DEVNULL)
         except OSError:
             self.proc = None
+            return
+        t0 = time.time()
+        while self._lines() == 0 and time.time() - t0 < 5 and self.proc.poll() is None:
+            time.sleep(0.02)
+
+    def mark(self):
+        """The timed region starts here: earlier samples are not used."""
+        self.first = self._lines() if self.proc is not None else 0
 
     def stop(self) -> dict:
         if self.proc is None:
             return {"sm_mhz": None, "sm_max_mhz": None, "reasons": ["nvidia-smi unavailable"]}
-        time.sleep(0.15)
+        time.sleep(0.06)  # one more sample period, so that the region's last sample is written
         self.proc.terminate()
         try:
             self.proc.wait(timeout=5)
@@ -87,7 +104,9 @@ class ClockSampler:
         sm, mx, reasons = [], [], set()
         names = ["hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"]
         with open(self.path) as f:
-            for line in f:
+            for k, line in enumerate(f):
+                if k < getattr(self, "first", 0):
+                    continue
                 p = [x.strip() for x in line.split(",")]
                 if len(p) < 7:
                     continue
@@ -471,15 +490,16 @@ def main():
                 events.append(torch.cuda.Event(enable_timing=True))
                 events[-1].record()
 
+    sampler = ClockSampler(local)
+    sampler.start()
     for _ in range(args.warmup):
         step()
     barrier()
-    sampler = ClockSampler(local)
-    sampler.start()
     evs = []
     wall0 = torch.cuda.Event(enable_timing=True)
     wall1 = torch.cuda.Event(enable_timing=True)
     barrier()
+    sampler.mark()
     wall0.record()
     for _ in range(args.steps):
         step(evs)

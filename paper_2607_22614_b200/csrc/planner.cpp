@@ -1,6 +1,7 @@
 // Layout planner: compiles (model spec, flat source layout, rollout layout, tp, rank) into the
 // segment table the gather/cast kernel walks.  Host only.
 #include <algorithm>
+#include <cstdlib>
 #include <cstring>
 
 #include "dr_internal.h"
@@ -503,11 +504,17 @@ int compile_plan(dr_plan* p)
         }
     }
 
-    {   // elements in strided segments: under 2 % of the plan, forward launches go through the bulk-copy kernel
+    {   // forward launches go through the bulk-copy kernel when under 2 % of the plan's elements sit in strided
+        // segments and the plan has 2^28 elements or more (below that the register kernel's shorter tile latency wins)
         uint64_t strided = 0;
         for (const HostSeg& g : p->segs)
             if (g.rows > 1) strided += g.rows * g.row_len;
-        p->bulk_forward = strided * 50 <= moved;
+        p->bulk_forward = strided * 50 <= moved && moved >= (1ull << 28);
+        // DR_FORWARD_KERNEL = bulk | register overrides the choice (for measurements; both give the same bytes)
+        if (const char* e = std::getenv("DR_FORWARD_KERNEL")) {
+            if (!std::strcmp(e, "bulk")) p->bulk_forward = true;
+            else if (!std::strcmp(e, "register")) p->bulk_forward = false;
+        }
     }
     dr_plan_info& I = p->info;
     I.flat_elems = N;

@@ -194,18 +194,25 @@ struct Peers {
 };
 
 // ---- forward tiles through the TMA unit -------------------------------------------------------------------------
-// A forward tile of a vector-class segment is moved by 1-D bulk asynchronous copies (cp.async.bulk: no tensor map,
+// A forward tile of a vector-class segment comes in by 1-D bulk asynchronous copies (cp.async.bulk: no tensor map,
 // no multicast): global -> shared memory, one copy per source row the tile touches (one in all for a contiguous
-// run), completion counted in bytes on an mbarrier; the cast runs from shared memory to shared memory; one bulk copy
-// shared -> global (the rollout side of a segment is always dense).  On B200 this streams
-// 1 % faster than 256-bit loads and stores from registers (7.17 against 7.10 TB/s on the 2 : 1 mix).  It is used for
-// the forward direction only: for the write-heavy inverse the register path is the faster one, and a kernel that
-// reserves the tile buffers (72 KB per CTA) leaves the register path too little L1 to keep its loads in flight, so
+// run), completion counted in bytes on an mbarrier.  It leaves through registers: 16 bytes read from shared memory,
+// cast, one 64-bit (bf16) or 128-bit (fp32) global store per thread and step, every warp one contiguous request.
+// Measured on B200, the 8.19 G-element contiguous plan, per launch: from idle (SM clock 1965 MHz) 6.80-6.87 ms
+// against 6.90-6.95 ms for the register kernel; in a long run of launches, with the part at its power limit and the
+// SM clock near 1.6 GHz, 6.87-6.88 ms against 6.89 ms.  DR_BULK_STORE=1 keeps the earlier form, which also casts from
+// shared to shared memory and stores the tile with one bulk copy: 6.80-6.82 ms from idle, but 7.04-7.2 ms at the
+// power limit (it leans on the TMA unit twice per byte and follows the SM clock down), so it is not the default.
+// It is used for the forward direction only: for the write-heavy inverse the register path is the faster one, and a
+// kernel that reserves the tile buffers leaves the register path too little L1 to keep its loads in flight, so
 // the two are not mixed in one launch configuration.
 // The wait on the mbarrier is bounded.  If it ever ran out, the tile is redone by the register path (same result)
 // after the copies in flight have been given a second bounded wait, and a counter is raised for the host to read.
 constexpr uint32_t kTileFlatBytes = kTileUnits * 32;                      // 48 KB of fp32
-constexpr uint32_t kBulkSmemBytes = kTileFlatBytes + kTileFlatBytes / 2;  // + 24 KB of bf16
+#ifndef DR_BULK_STORE
+#define DR_BULK_STORE 0
+#endif
+constexpr uint32_t kBulkSmemBytes = DR_BULK_STORE ? kTileFlatBytes + kTileFlatBytes / 2 : kTileFlatBytes;  // (+ 24 KB of bf16)
 constexpr uint32_t kBulkMaxRows = 32;                                     // source rows per tile the first warp can issue
 __device__ unsigned int g_bulk_wait_gave_up = 0;
 // Test hook: when set, every bulk tile expects 16 bytes more than its copies deliver, so its wait has to run out.
@@ -277,6 +284,25 @@ __device__ __forceinline__ bool bulk_forward_tile(const DevSeg& g, uint32_t ub, 
         mbar_wait_bounded(bar, 0);  // the copies must not land in the shared memory of a CTA that has moved on
         return false;
     }
+#if !DR_BULK_STORE
+    {   // out of shared memory through registers: cast, and plain stores (each warp one contiguous 256 or 512 B request)
+        char* dst = arena + g.dst_off + (uint64_t)ub * 8 * ES;
+#pragma unroll 2
+        for (uint32_t q = threadIdx.x; q < n * 2; q += kThreads) {
+            const uint4 v = *reinterpret_cast<const uint4*>(in + q * 16);
+            if (ES == 2)
+                asm volatile("st.global.L1::no_allocate.v2.b32 [%0], {%1,%2};" ::"l"(dst + q * 8), "r"(cvt_pair(v.x, v.y)),
+                             "r"(cvt_pair(v.z, v.w))
+                             : "memory");
+            else
+                asm volatile("st.global.L1::no_allocate.v4.b32 [%0], {%1,%2,%3,%4};" ::"l"(dst + q * 16), "r"(v.x), "r"(v.y),
+                             "r"(v.z), "r"(v.w)
+                             : "memory");
+        }
+        (void)out_s;
+        return true;
+    }
+#endif
     if (ES == 2) {  // fp32 -> bf16: 16 bytes in, 8 bytes out per step, consecutive threads consecutive quads
 #pragma unroll 2
         for (uint32_t q = threadIdx.x; q < n * 2; q += kThreads) {
@@ -456,7 +482,7 @@ __global__ void __launch_bounds__(kThreads, DR_MIN_BLOCKS)
 // with them is told so once per device.
 int ensure_bulk_smem(int device)
 {
-    if (DR_DYN_SMEM <= 48 * 1024) return DR_OK;
+    if (DR_DYN_SMEM < 40 * 1024) return DR_OK;  // static shared memory counts against the 48 KB default too
     static std::mutex mu;
     static bool done[64] = {false};
     std::lock_guard<std::mutex> lock(mu);

@@ -45,30 +45,48 @@ def test_sixteen_byte_aligned_bases_take_the_narrow_path(misalign, dtype):
     plan.close()
 
 
-# A MoE shape whose column-sliced (strided) attention output is under 2 % of the elements: such plans run the kernel
-# that moves tiles with the TMA unit's bulk copies, strided rows and run tails included.
+# A MoE shape whose column-sliced (strided) attention output is under 2 % of the elements.  Plans of that kind with
+# 2^28 elements or more run the kernel that brings tiles in with the TMA unit's bulk copies; the tests ask for that
+# kernel on this small shape through the library's override, strided rows and run tails included.
 MOE32 = dict(MID[2]["spec"], n_experts=32)
+
+
+@pytest.fixture
+def bulk_kernel(monkeypatch):
+    monkeypatch.setenv("DR_FORWARD_KERNEL", "bulk")
 
 
 @pytest.mark.parametrize("kw", [dict(tp=2, tp_rank=1), dict(tp=2, tp_rank=0, world=3, rank=1, gathered=False),
                                 dict(tp=2, tp_rank=1, align=4, dtype=dr.DR_F32), dict(tp=2, tp_rank=0, misalign=16),
                                 dict(tp=4, tp_rank=3, world=5, gathered=True, align=16)],
                          ids=["tp2", "shard-local", "f32-align4", "base16", "tp4-w5"])
-def test_bulk_copy_kernel_with_strided_rows_tails_and_shard_cuts(kw):
+def test_bulk_copy_kernel_with_strided_rows_tails_and_shard_cuts(kw, bulk_kernel):
     kw = dict(kw)
     got, want, plan, om, _ = forward_both(MOE32, seed=91, **kw)
     assert plan.info.bulk_forward == 1
     assert any(s.rows > 1 for s in plan.segments())          # column-sliced segments are there
     assert first_diff(got, want) is None
     plan.close()
-    # and the dense TP = 1 plans of the other mid-size shapes take the same kernel
-    for cfg in MID[:2]:
-        got, want, plan, _, _ = forward_both(cfg["spec"], seed=92)
+    # the dense TP = 1 plans of the other mid-size shapes, and one with 30 % strided elements, through the same kernel
+    for cfg, more in ((MID[0], {}), (MID[1], {}), (MID[0], dict(tp=2, tp_rank=1))):
+        got, want, plan, _, _ = forward_both(cfg["spec"], seed=92, **more)
         assert plan.info.bulk_forward == 1 and first_diff(got, want) is None
         plan.close()
-    got, want, plan, _, _ = forward_both(MID[0]["spec"], tp=2, tp_rank=1, seed=93)
-    assert plan.info.bulk_forward == 0 and first_diff(got, want) is None      # 30 % strided: the register kernel
-    plan.close()
+
+
+def test_which_plans_take_the_bulk_copy_kernel(monkeypatch):
+    """Large plans with next to no strided work take it; small plans and plans with column-sliced matrices do not."""
+    monkeypatch.delenv("DR_FORWARD_KERNEL", raising=False)
+    want = {0: 0, 1: 0, 2: 1, 3: 0, 4: 1}   # tiny: small; 1.7B at TP=2 and 14B at TP=4: 27-31 % strided
+    for i, cfg in enumerate(CONFIGS):
+        p = dr.Plan(cfg["spec"], world=cfg["world"], rank=cfg["rank"], gathered=cfg["gathered"], tp=cfg["tp"],
+                    tp_rank=cfg["tp_rank"], host_only=True)
+        assert p.info.bulk_forward == want[i], i
+        p.close()
+    monkeypatch.setenv("DR_FORWARD_KERNEL", "register")
+    p = dr.Plan(CONFIGS[2]["spec"], host_only=True)
+    assert p.info.bulk_forward == 0
+    p.close()
 
 
 def test_cast_special_values_in_hardware():
@@ -331,7 +349,7 @@ def test_groups_in_any_order_build_up_the_full_repack(spec, kw):
     plan.close()
 
 
-def test_the_bulk_copy_kernel_replays_from_a_cuda_graph_too():
+def test_the_bulk_copy_kernel_replays_from_a_cuda_graph_too(bulk_kernel):
     """The kernel that moves tiles with bulk copies (dynamic shared memory, mbarrier) is captured and replayed like the
     register kernel: each replay repacks whatever the source buffer holds at that time."""
     spec, kw = MOE32, dict(tp=2, tp_rank=0)

@@ -125,7 +125,7 @@ def test_no_bounded_device_wait_ran_out():
     plan.close()
 
 
-def test_a_bulk_wait_that_runs_out_falls_back_to_the_register_path():
+def test_a_bulk_wait_that_runs_out_falls_back_to_the_register_path(monkeypatch):
     """With the test hook on, every tile of the bulk-copy kernel waits for bytes that never come: the wait gives up
     after about 50 ms, the counter goes up by one per tile, the tile is redone through registers and the arena is
     still the oracle's.  Nothing faults or hangs; with the hook off again the next call is an ordinary one."""
@@ -135,6 +135,7 @@ def test_a_bulk_wait_that_runs_out_falls_back_to_the_register_path():
     src = make_source(om.flat_elems, 12)
     want = np.full(om.arena_bytes, SENT8, dtype=np.uint8)
     om.forward(src, want)
+    monkeypatch.setenv("DR_FORWARD_KERNEL", "bulk")           # a plan this small would take the register kernel
     plan = dr.Plan(spec)
     assert plan.info.bulk_forward == 1
     s_dev = torch.from_numpy(src.view(np.int32)).to(dev())
