@@ -145,9 +145,11 @@ typedef struct dr_plan_info {
     uint64_t quant_elems;     /* DR_FP8_E4M3_B128 plans: elements written as fp8 (counted in elems_moved) */
     uint64_t quant_blocks;    /* and the number of 128 x 128 blocks, one fp32 scale each              */
     uint64_t n_groups;        /* n_layers + 2: embed, every layer, final norm with lm_head            */
-    uint64_t bulk_forward;    /* 1: dr_reshard runs the kernel that moves tiles with the TMA unit's bulk
-                                 copies (plans with under 2 % of their elements in strided segments);
-                                 0: the kernel that moves them through registers.  Same result.       */
+    uint64_t bulk_forward;    /* 1: dr_reshard runs the kernel that brings tiles in with the TMA unit's
+                                 bulk copies (plans of 2^28 elements or more with under 2 % of them in
+                                 strided segments); 0: the kernel that moves them through registers.
+                                 Same result.  The environment variable DR_FORWARD_KERNEL = bulk |
+                                 register, read when a plan is created, overrides the choice.          */
 } dr_plan_info;
 
 typedef struct dr_tensor_desc {
