@@ -25,7 +25,9 @@ def stale() -> bool:
 def build(force: bool = False, verbose: bool = False) -> str:
     if not (force or stale()):
         return LIB
-    cmd = ["nvcc", *NVCC_FLAGS, "-I", os.path.join(_ROOT, "include"), "-I", CSRC, "-shared", "-o", LIB,
+    # DR_NVCC_FLAGS adds flags, e.g. the kernels' compile-time options (-DDR_BULK_STORE=1, -DDR_BULK=0, ...)
+    extra = os.environ.get("DR_NVCC_FLAGS", "").split()
+    cmd = ["nvcc", *NVCC_FLAGS, *extra, "-I", os.path.join(_ROOT, "include"), "-I", CSRC, "-shared", "-o", LIB,
            *[os.path.join(CSRC, s) for s in SOURCES]]
     if verbose:
         cmd.insert(1, "-Xptxas=-v")
